@@ -1,0 +1,252 @@
+// gv_oracle.cpp -- TEST INFRASTRUCTURE, NOT PRODUCT CODE.
+//
+// Plain, slow, single-threaded CPU statement of what the batched output verifier computes:
+// the "tolerance based tensor comparison of output tensors produced by test functions" of the
+// paper's Section 3.1 (TritonBench-revised, second bullet), applied to one candidate output
+// against one reference output, as the inner step of the Evaluator's functionality test
+// (Section 4.1) whose verdict feeds Execution Accuracy (Section 3.3: a kernel passes when it
+// satisfies all unit tests, i.e. n_mismatch == 0 for every test tensor).
+//
+// The paper states the comparison in one phrase and prints no formula. The rule below is the
+// torch.isclose rule (reference inside the relative term), evaluated element by element in
+// IEEE binary32 after exact widening, with every rounding written out. It shares no code,
+// header, table or constant generator with the CUDA library and is only ever used by tests/,
+// the smoke check and the CPU-baseline leg of the benchmark.
+//
+// Build: g++ -std=c++17 -O2 -ffp-contract=off -fno-fast-math -fPIC -shared
+//        (no -march flags, no -ffast-math / -Ofast: those would fuse, reassociate or flush
+//         subnormals to zero and change results).
+//
+// Every function here is pinned by tests/test_oracle_*.py against values fixed outside this
+// file (published SplitMix64 outputs, a hand-derived truth table, torch.isclose / numpy on the
+// host, closed forms and by-construction counts).
+
+#include <cstdint>
+#include <cstring>
+
+namespace {
+
+// ---- element types ---------------------------------------------------------------------
+enum Dtype { F32 = 0, BF16 = 1, F16 = 2, I32 = 3, I64 = 4 };
+
+inline int elem_size(int dt) {
+    switch (dt) {
+        case F32: return 4;
+        case BF16: return 2;
+        case F16: return 2;
+        case I32: return 4;
+        case I64: return 8;
+        default: return 0;
+    }
+}
+
+inline float bits_to_float(uint32_t b) {
+    float f;
+    std::memcpy(&f, &b, 4);
+    return f;
+}
+inline uint32_t float_to_bits(float f) {
+    uint32_t b;
+    std::memcpy(&b, &f, 4);
+    return b;
+}
+
+// Exact widening of a bfloat16 bit pattern: bf16 is the top half of a binary32.
+inline float widen_bf16(uint16_t h) { return bits_to_float(static_cast<uint32_t>(h) << 16); }
+
+// Exact widening of an IEEE binary16 bit pattern (1 sign, 5 exponent, 10 fraction bits).
+inline float widen_f16(uint16_t h) {
+    const uint32_t sign = static_cast<uint32_t>(h >> 15) << 31;
+    const uint32_t e = (h >> 10) & 0x1Fu;
+    const uint32_t m = h & 0x3FFu;
+    if (e == 0x1Fu) {                      // Inf (m == 0) or NaN (payload kept, moved up)
+        return bits_to_float(sign | 0x7F800000u | (m << 13));
+    }
+    if (e == 0) {
+        if (m == 0) return bits_to_float(sign);           // +-0
+        // subnormal half: value = m * 2^-24, exactly representable as a normal binary32
+        float v = static_cast<float>(m) * bits_to_float(0x33800000u);  // 2^-24, exact product
+        return sign ? -v : v;
+    }
+    // normal: rebias exponent 15 -> 127
+    return bits_to_float(sign | ((e + 112u) << 23) | (m << 13));
+}
+
+inline bool is_nan(float f) { return (float_to_bits(f) & 0x7FFFFFFFu) > 0x7F800000u; }
+inline int inf_class(float f) {
+    const uint32_t b = float_to_bits(f);
+    if ((b & 0x7FFFFFFFu) != 0x7F800000u) return 0;
+    return (b >> 31) ? -1 : +1;
+}
+inline bool is_finite(float f) { return (float_to_bits(f) & 0x7F800000u) != 0x7F800000u; }
+inline float f_abs(float f) { return bits_to_float(float_to_bits(f) & 0x7FFFFFFFu); }
+
+}  // namespace
+
+extern "C" {
+
+// 64-byte result record, one per candidate. Field meaning as in the library's public header,
+// restated here because the two sides share no header.
+struct gvo_result {
+    uint64_t n_mismatch;        // elements that are not close
+    uint64_t first_mismatch;    // smallest such index, all-ones when there is none
+    uint64_t n_nan_disagree;    // isnan(c) != isnan(r)
+    uint64_t n_inf_disagree;    // infclass(c) != infclass(r)
+    uint64_t hash;              // content hash of the candidate's bytes
+    uint64_t max_abs_diff_int;  // integer dtypes: max |c - r|, exact
+    float max_abs_err;          // float dtypes: max |fl(c - r)| over finite pairs
+    float max_rel_err;          // float dtypes: max fl(|d| / |r|) over finite pairs with r != 0
+    uint64_t reserved;          // 0
+};
+
+// SplitMix64 output function (Steele, Lea, Flood 2014; public domain reference by Vigna):
+// add the golden-gamma, two xor-shift-multiply rounds, final xor-shift. All mod 2^64.
+uint64_t gvo_splitmix64(uint64_t x) {
+    uint64_t z = x + 0x9E3779B97F4A7C15ull;
+    z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+    z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+    return z ^ (z >> 31);
+}
+
+// Order-independent content hash: the byte image, zero-padded to a multiple of 8, is read as
+// little-endian 64-bit words W_k; hash = sum over k of splitmix64(k xor W_k), wrapping.
+// ("index" = word index, "raw bits" = the word; the length is not mixed in.)
+uint64_t gvo_hash(const void* buf, uint64_t nbytes) {
+    const unsigned char* p = static_cast<const unsigned char*>(buf);
+    const uint64_t nwords = (nbytes + 7) / 8;
+    uint64_t h = 0;
+    for (uint64_t k = 0; k < nwords; ++k) {
+        uint64_t w = 0;
+        for (int b = 0; b < 8; ++b) {
+            const uint64_t pos = 8 * k + static_cast<uint64_t>(b);
+            if (pos < nbytes) w |= static_cast<uint64_t>(p[pos]) << (8 * b);
+        }
+        h += gvo_splitmix64(k ^ w);
+    }
+    return h;
+}
+
+// Widening used by the compare; exported so a test can check it against numpy for all 2^16
+// patterns of both 16-bit types. Returns the binary32 bit pattern.
+uint32_t gvo_widen_bits(int dtype, uint32_t raw) {
+    if (dtype == BF16) return float_to_bits(widen_bf16(static_cast<uint16_t>(raw)));
+    if (dtype == F16) return float_to_bits(widen_f16(static_cast<uint16_t>(raw)));
+    return raw;
+}
+
+// One candidate against one reference. Returns 0, or 1 for an unknown dtype.
+// Float dtypes: atol and rtol are converted once to binary32 (round to nearest); integer
+// dtypes ignore them and compare exactly.
+int gvo_verify(const void* ref, const void* cand, uint64_t n, int dtype, double atol, double rtol,
+               int equal_nan, gvo_result* out) {
+    const int esz = elem_size(dtype);
+    if (esz == 0) return 1;
+
+    gvo_result res;
+    res.n_mismatch = 0;
+    res.first_mismatch = ~0ull;
+    res.n_nan_disagree = 0;
+    res.n_inf_disagree = 0;
+    res.hash = gvo_hash(cand, n * static_cast<uint64_t>(esz));
+    res.max_abs_diff_int = 0;
+    res.max_abs_err = 0.0f;
+    res.max_rel_err = 0.0f;
+    res.reserved = 0;
+
+    if (dtype == I32 || dtype == I64) {
+        for (uint64_t i = 0; i < n; ++i) {
+            int64_t c, r;
+            if (dtype == I32) {
+                int32_t c32, r32;
+                std::memcpy(&c32, static_cast<const char*>(cand) + 4 * i, 4);
+                std::memcpy(&r32, static_cast<const char*>(ref) + 4 * i, 4);
+                c = c32;
+                r = r32;
+            } else {
+                std::memcpy(&c, static_cast<const char*>(cand) + 8 * i, 8);
+                std::memcpy(&r, static_cast<const char*>(ref) + 8 * i, 8);
+            }
+            if (c != r) {
+                res.n_mismatch += 1;
+                if (i < res.first_mismatch) res.first_mismatch = i;
+                // |c - r| in unsigned arithmetic: exact even at the int64 extremes
+                const uint64_t diff = (c > r) ? static_cast<uint64_t>(c) - static_cast<uint64_t>(r)
+                                              : static_cast<uint64_t>(r) - static_cast<uint64_t>(c);
+                if (diff > res.max_abs_diff_int) res.max_abs_diff_int = diff;
+            }
+        }
+        *out = res;
+        return 0;
+    }
+
+    const float atol_f = static_cast<float>(atol);
+    const float rtol_f = static_cast<float>(rtol);
+    const float pos_inf = bits_to_float(0x7F800000u);
+
+    for (uint64_t i = 0; i < n; ++i) {
+        float c, r;
+        if (dtype == F32) {
+            std::memcpy(&c, static_cast<const char*>(cand) + 4 * i, 4);
+            std::memcpy(&r, static_cast<const char*>(ref) + 4 * i, 4);
+        } else {
+            uint16_t cb, rb;
+            std::memcpy(&cb, static_cast<const char*>(cand) + 2 * i, 2);
+            std::memcpy(&rb, static_cast<const char*>(ref) + 2 * i, 2);
+            c = (dtype == BF16) ? widen_bf16(cb) : widen_f16(cb);
+            r = (dtype == BF16) ? widen_bf16(rb) : widen_f16(rb);
+        }
+
+        const float d = c - r;                 // one rounding
+        const float ad = f_abs(d);             // NaN stays NaN
+        const float prod = rtol_f * f_abs(r);  // one rounding
+        const float tol = atol_f + prod;       // a second rounding: never a fused multiply-add
+
+        const bool c_nan = is_nan(c), r_nan = is_nan(r);
+        bool close = (c == r);                                    // IEEE ==: +0 == -0, Inf == Inf
+        if (equal_nan && c_nan && r_nan) close = true;
+        if (ad < pos_inf && ad <= tol) close = true;              // false for NaN or infinite ad
+
+        if (!close) {
+            res.n_mismatch += 1;
+            if (i < res.first_mismatch) res.first_mismatch = i;
+        }
+        if (c_nan != r_nan) res.n_nan_disagree += 1;
+        if (inf_class(c) != inf_class(r)) res.n_inf_disagree += 1;
+
+        if (is_finite(c) && is_finite(r)) {
+            if (ad > res.max_abs_err) res.max_abs_err = ad;       // ad in [0, +Inf]
+            if (r != 0.0f) {
+                const float rel = ad / f_abs(r);                  // IEEE division
+                if (rel > res.max_rel_err) res.max_rel_err = rel;
+            }
+        }
+    }
+    *out = res;
+    return 0;
+}
+
+// Ragged batch: T tensors, each with N candidates. Tensor t starts at ref_base + ref_off[t], has
+// element size given by dtypes[t] and n_elems[t] elements (when n_elems is null the tensors are
+// packed back to back and the count is (ref_off[t+1] - ref_off[t]) / element size); candidate
+// (t, j) starts at cand_base + cand_off[t*N + j]. results is tensor-major (t*N + j);
+// first_mismatch is relative to the tensor's own start. Nothing but a double loop over gvo_verify.
+int gvo_verify_ragged(const void* ref_base, const int64_t* ref_off, const void* cand_base,
+                      const int64_t* cand_off, const uint8_t* dtypes, const int64_t* n_elems,
+                      int64_t T, int32_t N, double atol, double rtol, int equal_nan,
+                      gvo_result* results) {
+    for (int64_t t = 0; t < T; ++t) {
+        const int esz = elem_size(dtypes[t]);
+        if (esz == 0) return 1;
+        const uint64_t n = n_elems ? static_cast<uint64_t>(n_elems[t])
+                                   : static_cast<uint64_t>(ref_off[t + 1] - ref_off[t]) / static_cast<uint64_t>(esz);
+        for (int32_t j = 0; j < N; ++j) {
+            const int rc = gvo_verify(static_cast<const char*>(ref_base) + ref_off[t],
+                                      static_cast<const char*>(cand_base) + cand_off[t * N + j], n,
+                                      dtypes[t], atol, rtol, equal_nan, &results[t * N + j]);
+            if (rc) return rc;
+        }
+    }
+    return 0;
+}
+
+}  // extern "C"

@@ -1,0 +1,159 @@
+"""ctypes loader for the CPU oracle (``gv_oracle.cpp``) -- TEST INFRASTRUCTURE ONLY.
+
+Only ``tests/``, the smoke check and the benchmark's CPU-baseline leg may import this module.
+It holds no arithmetic of its own: it compiles the C++ file beside it with the flags its header
+states and marshals numpy arrays to it. The record layout is restated here (the oracle and the
+CUDA library share no header).
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "gv_oracle.cpp")
+_LIB = os.path.join(_HERE, "libgv_oracle.so")
+
+# dtype codes of the oracle's own enum
+F32, BF16, F16, I32, I64 = 0, 1, 2, 3, 4
+ELEM_SIZE = {F32: 4, BF16: 2, F16: 2, I32: 4, I64: 8}
+
+# 64-byte record as a numpy structured dtype (little-endian, no padding)
+RESULT_DTYPE = np.dtype(
+    [
+        ("n_mismatch", "<u8"),
+        ("first_mismatch", "<u8"),
+        ("n_nan_disagree", "<u8"),
+        ("n_inf_disagree", "<u8"),
+        ("hash", "<u8"),
+        ("max_abs_diff_int", "<u8"),
+        ("max_abs_err", "<f4"),
+        ("max_rel_err", "<f4"),
+        ("reserved", "<u8"),
+    ]
+)
+assert RESULT_DTYPE.itemsize == 64
+
+NO_INDEX = 0xFFFFFFFFFFFFFFFF
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle into a shared object beside its source (a second or two with g++)."""
+    if not force and os.path.exists(_LIB) and os.path.getmtime(_LIB) >= os.path.getmtime(_SRC):
+        return _LIB
+    cmd = [
+        "g++", "-std=c++17", "-O2", "-ffp-contract=off", "-fno-fast-math", "-fPIC", "-shared",
+        "-o", _LIB + ".tmp", _SRC,
+    ]
+    subprocess.run(cmd, check=True)
+    os.replace(_LIB + ".tmp", _LIB)
+    return _LIB
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    global _lib
+    if _lib is None:
+        L = ctypes.CDLL(build())
+        L.gvo_splitmix64.restype = ctypes.c_uint64
+        L.gvo_splitmix64.argtypes = [ctypes.c_uint64]
+        L.gvo_hash.restype = ctypes.c_uint64
+        L.gvo_hash.argtypes = [ctypes.c_void_p, ctypes.c_uint64]
+        L.gvo_widen_bits.restype = ctypes.c_uint32
+        L.gvo_widen_bits.argtypes = [ctypes.c_int, ctypes.c_uint32]
+        L.gvo_verify.restype = ctypes.c_int
+        L.gvo_verify.argtypes = [
+            ctypes.c_void_p, ctypes.c_void_p, ctypes.c_uint64, ctypes.c_int,
+            ctypes.c_double, ctypes.c_double, ctypes.c_int, ctypes.c_void_p,
+        ]
+        L.gvo_verify_ragged.restype = ctypes.c_int
+        L.gvo_verify_ragged.argtypes = [
+            ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
+            ctypes.c_void_p, ctypes.c_int64, ctypes.c_int32, ctypes.c_double, ctypes.c_double, ctypes.c_int,
+            ctypes.c_void_p,
+        ]
+        _lib = L
+    return _lib
+
+
+def _as_bytes_array(a: np.ndarray) -> np.ndarray:
+    a = np.ascontiguousarray(a)
+    return a
+
+
+def splitmix64(x: int) -> int:
+    return int(lib().gvo_splitmix64(ctypes.c_uint64(x & NO_INDEX)))
+
+
+def hash_bytes(a) -> int:
+    """Content hash of a numpy array's byte image (or of a bytes object)."""
+    if isinstance(a, (bytes, bytearray)):
+        a = np.frombuffer(bytes(a), dtype=np.uint8)
+    a = _as_bytes_array(a)
+    return int(lib().gvo_hash(a.ctypes.data_as(ctypes.c_void_p), ctypes.c_uint64(a.nbytes)))
+
+
+def widen_bits(dtype: int, raw: int) -> int:
+    return int(lib().gvo_widen_bits(dtype, raw))
+
+
+def verify(ref: np.ndarray, cand: np.ndarray, dtype: int, atol: float = 0.0, rtol: float = 0.0,
+           equal_nan: bool = False) -> np.ndarray:
+    """One candidate against one reference; returns a 0-d structured record.
+
+    ``ref`` / ``cand`` are numpy arrays whose bytes are the tensors (16-bit float types are
+    passed as uint16 bit patterns); the element count is nbytes / element size.
+    """
+    ref = _as_bytes_array(ref)
+    cand = _as_bytes_array(cand)
+    assert ref.nbytes == cand.nbytes, "reference and candidate differ in size"
+    n = ref.nbytes // ELEM_SIZE[dtype]
+    out = np.zeros((), dtype=RESULT_DTYPE)
+    rc = lib().gvo_verify(ref.ctypes.data_as(ctypes.c_void_p), cand.ctypes.data_as(ctypes.c_void_p),
+                          ctypes.c_uint64(n), dtype, float(atol), float(rtol), int(bool(equal_nan)),
+                          out.ctypes.data_as(ctypes.c_void_p))
+    if rc != 0:
+        raise ValueError(f"oracle rejected dtype {dtype}")
+    return out
+
+
+def verify_batch(ref: np.ndarray, cands, dtype: int, atol: float = 0.0, rtol: float = 0.0,
+                 equal_nan: bool = False) -> np.ndarray:
+    """N candidates against one reference: a plain loop over ``verify``."""
+    out = np.zeros(len(cands), dtype=RESULT_DTYPE)
+    for j, c in enumerate(cands):
+        out[j] = verify(ref, c, dtype, atol, rtol, equal_nan)
+    return out
+
+
+def verify_ragged(ref_buf: np.ndarray, ref_off: np.ndarray, cand_buf: np.ndarray,
+                  cand_off: np.ndarray, dtypes: np.ndarray, N: int, atol: float, rtol: float,
+                  equal_nan: bool = False, n_elems: np.ndarray | None = None) -> np.ndarray:
+    """Ragged batch (byte offsets; results tensor-major, shape [T*N]). ``n_elems`` (int64 [T])
+    gives the element counts; without it they are read off consecutive ``ref_off`` entries."""
+    ref_buf = _as_bytes_array(ref_buf)
+    cand_buf = _as_bytes_array(cand_buf)
+    ref_off = np.ascontiguousarray(ref_off, dtype=np.int64)
+    cand_off = np.ascontiguousarray(cand_off, dtype=np.int64)
+    dtypes = np.ascontiguousarray(dtypes, dtype=np.uint8)
+    T = len(dtypes)
+    assert ref_off.shape == (T + 1,) and cand_off.shape == (T * N,)
+    ne_ptr = None
+    if n_elems is not None:
+        n_elems = np.ascontiguousarray(n_elems, dtype=np.int64)
+        assert n_elems.shape == (T,)
+        ne_ptr = n_elems.ctypes.data_as(ctypes.c_void_p)
+    out = np.zeros(T * N, dtype=RESULT_DTYPE)
+    rc = lib().gvo_verify_ragged(
+        ref_buf.ctypes.data_as(ctypes.c_void_p), ref_off.ctypes.data_as(ctypes.c_void_p),
+        cand_buf.ctypes.data_as(ctypes.c_void_p), cand_off.ctypes.data_as(ctypes.c_void_p),
+        dtypes.ctypes.data_as(ctypes.c_void_p), ne_ptr, ctypes.c_int64(T), ctypes.c_int32(N),
+        float(atol), float(rtol), int(bool(equal_nan)), out.ctypes.data_as(ctypes.c_void_p))
+    if rc != 0:
+        raise ValueError("oracle rejected a dtype code in the ragged batch")
+    return out

@@ -1,0 +1,162 @@
+/* gv.h -- C ABI of the batched candidate-vs-reference output verifier (NVIDIA B200, sm_100a).
+ *
+ * What it computes. The GEAK paper's Evaluator runs a "functionality test" on every generated
+ * kernel (Section 4.1): the candidate's unit-test outputs are checked against the reference
+ * kernel's by a "tolerance based tensor comparison of output tensors" (Section 3.1), and a
+ * kernel counts towards Execution Accuracy when all its tests pass (Section 3.3). Parallel and
+ * sequential scaling (Section 4.2, Section 5.2) produce many candidates per reference output;
+ * this library verifies N candidates against one reference in a single pass over the data.
+ *
+ * Per candidate it returns a 64-byte record: number of elements that are not close, the first
+ * such index, NaN / Inf disagreement counts, maximum absolute and relative error, an exact
+ * maximum difference for integer outputs, and an order-independent 64-bit content hash of the
+ * candidate's bytes (for de-duplicating identical candidates).
+ *
+ * Per-element rule (float dtypes; c = candidate, r = reference, both widened exactly to
+ * binary32; fl() = one round-to-nearest-even binary32 operation; subnormals are preserved):
+ *     d = fl(c - r), ad = |d|, tol = fl(atol_f + fl(rtol_f * |r|))        (two roundings, no FMA)
+ *     close = (c == r) or (equal_nan and isnan(c) and isnan(r)) or (ad < +Inf and ad <= tol)
+ *     n_nan_disagree counts isnan(c) != isnan(r); n_inf_disagree counts infclass(c) != infclass(r)
+ *     over pairs with c and r both finite: max_abs_err = max ad;  where also r != 0:
+ *     max_rel_err = max fl(ad / |r|)                                       (IEEE division)
+ *   atol_f = (float)atol, rtol_f = (float)rtol. torch.allclose(c.float(), r.float(), rtol, atol,
+ *   equal_nan) is true exactly when n_mismatch == 0.
+ * Integer dtypes are always compared exactly (tolerances ignored): close = (c == r),
+ *   max_abs_diff_int = max |c - r| computed without overflow.
+ * Content hash: the tensor's byte image, zero-padded to a multiple of 8 bytes, read as
+ *   little-endian 64-bit words W_k; hash = sum_k splitmix64(k xor W_k) mod 2^64. The length is
+ *   not mixed in. Equal hashes indicate *candidate* duplicates (k xor W_k is a weak combiner: e.g.
+ *   int64 [0,0] and [1,1] collide); confirm with the other fields or a byte compare.
+ * Every field has exactly one correct value; all reductions are integer sums / minima / maxima,
+ * so results do not depend on scheduling.
+ *
+ * Conventions for every entry point below.
+ *  - Pointers marked "device" must be device-accessible memory of the current CUDA device;
+ *    "host" pointers are ordinary host memory. The library allocates and frees no memory.
+ *  - Calls enqueue work on `cuda_stream` (a cudaStream_t passed as void*; NULL = default stream)
+ *    and return without synchronising. Outputs are valid once the stream reaches that point.
+ *    Host arrays passed in (the candidate pointer list) are consumed before the call returns.
+ *  - Errors are reported by return code only. When a call returns anything but GV_OK because of
+ *    its arguments, nothing was enqueued and no output was touched.
+ *  - Inputs are read-only. Tensors are contiguous. Base addresses must be multiples of the
+ *    element size; 16-byte aligned bases take the fast path, others a slower path with the same
+ *    results.
+ */
+#ifndef GV_H_
+#define GV_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum gv_dtype { GV_F32 = 0, GV_BF16 = 1, GV_F16 = 2, GV_I32 = 3, GV_I64 = 4 } gv_dtype;
+
+typedef enum gv_status {
+    GV_OK = 0,
+    GV_ERR_INVALID_ARG = 1,    /* null pointer, negative count, non-finite or negative tolerance */
+    GV_ERR_UNSUPPORTED = 2,    /* dtype code out of range                                       */
+    GV_ERR_MISALIGNED = 3,     /* a base address is not a multiple of the element size          */
+    GV_ERR_WORKSPACE = 4,      /* workspace missing, misaligned or smaller than gv_workspace_bytes */
+    GV_ERR_CUDA = 5,           /* a CUDA runtime call failed; see gv_last_cuda_error()           */
+    GV_ERR_DEVICE_TIMEOUT = 6, /* a bounded device-side wait expired (reported by gv_check)      */
+    GV_ERR_BAD_TABLE = 7       /* ragged tables inconsistent (reported by gv_check)              */
+} gv_status;
+
+#define GV_NO_INDEX 0xFFFFFFFFFFFFFFFFull
+
+/* One record per candidate. 64 bytes, little-endian, comparable with memcmp. */
+typedef struct gv_result {
+    uint64_t n_mismatch;       /* elements that are not close                                   */
+    uint64_t first_mismatch;   /* smallest flat index that is not close, else GV_NO_INDEX        */
+    uint64_t n_nan_disagree;   /* float dtypes; 0 for integer dtypes                             */
+    uint64_t n_inf_disagree;   /* float dtypes; 0 for integer dtypes                             */
+    uint64_t hash;             /* content hash of the candidate's bytes                          */
+    uint64_t max_abs_diff_int; /* integer dtypes: exact max |c - r|; float dtypes: 0             */
+    float max_abs_err;         /* float dtypes; integer dtypes: 0. Never NaN, never -0           */
+    float max_rel_err;         /* float dtypes; integer dtypes: 0. Never NaN, never -0           */
+    uint64_t reserved;         /* 0                                                              */
+} gv_result;
+
+/* Tolerances of the comparison (Section 3.1 names them without values; callers choose). */
+typedef struct gv_tol {
+    double atol;       /* finite, >= 0 */
+    double rtol;       /* finite, >= 0 */
+    int32_t equal_nan; /* nonzero: NaN in both c and r counts as close */
+    int32_t reserved;  /* 0 */
+} gv_tol;
+
+/* Dense batch: N candidates, each n_elems elements of dtype dt, against one reference
+ * (the Evaluator's functionality test of Section 4.1 applied to one unit-test output).
+ *   ref        device, n_elems elements.
+ *   cands      HOST array of N device pointers (copied before return).
+ *   tol        host; ignored (may be NULL) for integer dtypes.
+ *   results    device, N records, fully overwritten.
+ *   ref_hash   device, one uint64, receives the reference's content hash; may be NULL.
+ *   workspace  device, >= gv_workspace_bytes(0, N) bytes, 16-byte aligned; must stay untouched
+ *              until the stream has passed this call. It carries a status word for gv_check().
+ * N == 0 or n_elems == 0 is legal (no records / zero records: all fields 0, first_mismatch
+ * GV_NO_INDEX, hash 0). The paper notes that an earlier harness silently compared empty outputs
+ * (Section 3.1); deciding that an empty test output is an error is left to the caller, who can
+ * see it from n_elems. */
+gv_status gv_verify_batch(const void* ref, const void* const* cands, int32_t N, uint64_t n_elems,
+                          gv_dtype dt, const gv_tol* tol, gv_result* results, uint64_t* ref_hash,
+                          void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* Ragged batch: T test tensors of mixed dtype and size packed into one reference buffer, each
+ * with N candidates packed into one candidate buffer (many small unit-test outputs, cf. the
+ * handful of unit tests per kernel noted in the paper's Appendix B).
+ *   ref_off    device, int64[T+1]: byte offset of tensor t in ref_base; entry T is the end of the
+ *              last tensor.
+ *   cand_off   device, int64[T*N], tensor-major: byte offset of candidate (t, j) in cand_base.
+ *   dtypes     device, uint8[T]: gv_dtype code of tensor t.
+ *   n_elems    device, int64[T]: element count of tensor t; may be NULL when tensors are packed
+ *              back to back, in which case it is (ref_off[t+1] - ref_off[t]) / element size.
+ *   results    device, T*N records, tensor-major; first_mismatch is relative to the tensor.
+ *   workspace  device, >= gv_workspace_bytes(T, N) bytes, 16-byte aligned.
+ * Offsets must be multiples of the tensor's element size. The tables live on the device and are
+ * checked there: a bad entry (negative size, misaligned offset, unknown dtype) makes that tensor's
+ * records stay zero records and sets GV_ERR_BAD_TABLE in the status word read by gv_check(). */
+gv_status gv_verify_ragged(const void* ref_base, const int64_t* ref_off, const void* cand_base,
+                           const int64_t* cand_off, const uint8_t* dtypes, const int64_t* n_elems,
+                           int64_t T, int32_t N, const gv_tol* tol, gv_result* results,
+                           void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* Content hash of nbytes bytes at buf (device) into *out (device). buf needs no alignment.
+ * The same function the verifier applies to each candidate (used to de-duplicate candidates). */
+gv_status gv_hash(const void* buf, uint64_t nbytes, uint64_t* out, void* cuda_stream);
+
+/* Host-buffer convenience for callers whose outputs live in host memory: copies the reference and
+ * the candidates host->device in slabs through `staging` (device, staging_bytes), verifies them and
+ * copies the N records (and the reference hash) back to host memory. Copies and kernels are
+ * enqueued on cuda_stream; the call returns after synchronising that stream, so results are valid
+ * on return. Same computation as gv_verify_batch.
+ *   ref_host, cands_host[j]   host memory (pinned memory makes the copies fast)
+ *   results_host              host, N records;  ref_hash_host host, may be NULL
+ *   staging                   device, 256-byte aligned, >= gv_host_staging_bytes(n_elems, dt, 1) */
+gv_status gv_verify_batch_host(const void* ref_host, const void* const* cands_host, int32_t N,
+                               uint64_t n_elems, gv_dtype dt, const gv_tol* tol,
+                               gv_result* results_host, uint64_t* ref_hash_host, void* staging,
+                               size_t staging_bytes, void* cuda_stream);
+
+/* Bytes of staging needed by gv_verify_batch_host to hold the reference plus `slab` candidates
+ * (slab >= 1; larger slabs amortise launches), including records and workspace. */
+size_t gv_host_staging_bytes(uint64_t n_elems, gv_dtype dt, int32_t slab);
+
+/* Upper bound on the workspace either verify call needs (T = 0 for the dense call). */
+size_t gv_workspace_bytes(int64_t T, int32_t N);
+
+/* Synchronises cuda_stream, reads the status word of `workspace` and returns GV_OK,
+ * GV_ERR_DEVICE_TIMEOUT or GV_ERR_BAD_TABLE (or GV_ERR_CUDA). Optional. */
+gv_status gv_check(const void* workspace, void* cuda_stream);
+
+const char* gv_status_string(gv_status s);
+const char* gv_last_cuda_error(void); /* text of the last CUDA error seen by this thread, or "" */
+uint32_t gv_version(void);            /* major << 16 | minor << 8 | patch */
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GV_H_ */

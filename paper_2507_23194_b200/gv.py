@@ -1,0 +1,196 @@
+"""Thin Python binding of the C ABI in ``include/gv.h`` (argument marshalling only).
+
+Every function here has the name and meaning of the C entry point it wraps; all computation runs
+in the CUDA kernels of ``libgv.so``. PyTorch only supplies device memory (``data_ptr()``) and the
+current stream. There is no CPU fallback: if the library is missing, importing this module fails.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Sequence
+
+import numpy as np
+import torch
+
+from . import build as _build
+
+GV_F32, GV_BF16, GV_F16, GV_I32, GV_I64 = 0, 1, 2, 3, 4
+GV_OK = 0
+GV_ERR_INVALID_ARG, GV_ERR_UNSUPPORTED, GV_ERR_MISALIGNED, GV_ERR_WORKSPACE = 1, 2, 3, 4
+GV_ERR_CUDA, GV_ERR_DEVICE_TIMEOUT, GV_ERR_BAD_TABLE = 5, 6, 7
+GV_NO_INDEX = 0xFFFFFFFFFFFFFFFF
+
+DTYPE_OF = {torch.float32: GV_F32, torch.bfloat16: GV_BF16, torch.float16: GV_F16,
+            torch.int32: GV_I32, torch.int64: GV_I64}
+
+#: gv_result as a numpy structured dtype (64 bytes)
+RESULT_DTYPE = np.dtype([
+    ("n_mismatch", "<u8"), ("first_mismatch", "<u8"), ("n_nan_disagree", "<u8"), ("n_inf_disagree", "<u8"),
+    ("hash", "<u8"), ("max_abs_diff_int", "<u8"), ("max_abs_err", "<f4"), ("max_rel_err", "<f4"),
+    ("reserved", "<u8")])
+assert RESULT_DTYPE.itemsize == 64
+
+
+class gv_tol(ctypes.Structure):
+    _fields_ = [("atol", ctypes.c_double), ("rtol", ctypes.c_double),
+                ("equal_nan", ctypes.c_int32), ("reserved", ctypes.c_int32)]
+
+
+EXPORTS = ["gv_verify_batch", "gv_verify_ragged", "gv_hash", "gv_verify_batch_host", "gv_host_staging_bytes",
+           "gv_workspace_bytes", "gv_check", "gv_status_string", "gv_last_cuda_error", "gv_version"]
+
+
+def _load() -> ctypes.CDLL:
+    path = _build.LIB_PATH
+    if not os.path.exists(path):
+        raise ImportError(
+            f"{path} is missing: build it with `python -m paper_2507_23194_b200.build` "
+            "(or __graft_entry__.build()). There is no fallback implementation.")
+    L = ctypes.CDLL(path)
+    vp, i32, i64, u64, sz = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_uint64, ctypes.c_size_t
+    L.gv_verify_batch.restype = ctypes.c_int
+    L.gv_verify_batch.argtypes = [vp, vp, i32, u64, ctypes.c_int, ctypes.POINTER(gv_tol), vp, vp, vp, sz, vp]
+    L.gv_verify_ragged.restype = ctypes.c_int
+    L.gv_verify_ragged.argtypes = [vp, vp, vp, vp, vp, vp, i64, i32, ctypes.POINTER(gv_tol), vp, vp, sz, vp]
+    L.gv_hash.restype = ctypes.c_int
+    L.gv_hash.argtypes = [vp, u64, vp, vp]
+    L.gv_verify_batch_host.restype = ctypes.c_int
+    L.gv_verify_batch_host.argtypes = [vp, vp, i32, u64, ctypes.c_int, ctypes.POINTER(gv_tol), vp, vp, vp, sz, vp]
+    L.gv_host_staging_bytes.restype = sz
+    L.gv_host_staging_bytes.argtypes = [u64, ctypes.c_int, i32]
+    L.gv_workspace_bytes.restype = sz
+    L.gv_workspace_bytes.argtypes = [i64, i32]
+    L.gv_check.restype = ctypes.c_int
+    L.gv_check.argtypes = [vp, vp]
+    L.gv_status_string.restype = ctypes.c_char_p
+    L.gv_status_string.argtypes = [ctypes.c_int]
+    L.gv_last_cuda_error.restype = ctypes.c_char_p
+    L.gv_last_cuda_error.argtypes = []
+    L.gv_version.restype = ctypes.c_uint32
+    L.gv_version.argtypes = []
+    return L
+
+
+lib = _load()
+
+
+class GvError(RuntimeError):
+    def __init__(self, status: int):
+        self.status = status
+        msg = lib.gv_status_string(status).decode()
+        if status == GV_ERR_CUDA:
+            msg += ": " + lib.gv_last_cuda_error().decode()
+        super().__init__(f"gv status {status}: {msg}")
+
+
+def _raise(status: int) -> None:
+    if status != GV_OK:
+        raise GvError(status)
+
+
+def _stream_ptr(stream: Optional[torch.cuda.Stream]) -> ctypes.c_void_p:
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+def _tol(atol: float, rtol: float, equal_nan: bool) -> gv_tol:
+    return gv_tol(float(atol), float(rtol), int(bool(equal_nan)), 0)
+
+
+def gv_workspace_bytes(T: int = 0, N: int = 0) -> int:
+    return int(lib.gv_workspace_bytes(T, N))
+
+
+def gv_version() -> int:
+    return int(lib.gv_version())
+
+
+def results_to_numpy(results: torch.Tensor) -> np.ndarray:
+    """Device (or host) uint8 record buffer -> structured numpy array of gv_result records."""
+    return results.cpu().numpy().view(RESULT_DTYPE).reshape(-1)
+
+
+def gv_verify_batch(ref: torch.Tensor, cands: Sequence[torch.Tensor], atol: float = 0.0, rtol: float = 0.0,
+                    equal_nan: bool = False, results: Optional[torch.Tensor] = None,
+                    ref_hash: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None,
+                    stream: Optional[torch.cuda.Stream] = None, cand_ptrs=None) -> torch.Tensor:
+    """Enqueue one dense verification; returns the device tensor of N 64-byte records (uint8 [N, 64]).
+
+    Buffers not supplied are allocated here with torch (the C library itself allocates nothing).
+    ``cand_ptrs`` may carry a prebuilt ``(ctypes.c_void_p * N)`` array to skip marshalling.
+    """
+    dt = DTYPE_OF[ref.dtype]
+    N = len(cands)
+    dev = ref.device
+    if results is None:
+        results = torch.empty((max(N, 1), 64), dtype=torch.uint8, device=dev)
+    if workspace is None:
+        workspace = torch.empty(gv_workspace_bytes(0, N), dtype=torch.uint8, device=dev)
+    if cand_ptrs is None:
+        cand_ptrs = (ctypes.c_void_p * max(N, 1))(*[c.data_ptr() for c in cands])
+    t = _tol(atol, rtol, equal_nan)
+    rc = lib.gv_verify_batch(ref.data_ptr(), ctypes.cast(cand_ptrs, ctypes.c_void_p), N, ref.numel(), dt,
+                             ctypes.byref(t), results.data_ptr(),
+                             ref_hash.data_ptr() if ref_hash is not None else None,
+                             workspace.data_ptr(), workspace.numel(), _stream_ptr(stream))
+    _raise(rc)
+    return results[:N]
+
+
+def gv_verify_ragged(ref_buf: torch.Tensor, ref_off: torch.Tensor, cand_buf: torch.Tensor, cand_off: torch.Tensor,
+                     dtypes: torch.Tensor, N: int, atol: float, rtol: float, equal_nan: bool = False,
+                     n_elems: Optional[torch.Tensor] = None, results: Optional[torch.Tensor] = None,
+                     workspace: Optional[torch.Tensor] = None,
+                     stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:
+    """Enqueue one ragged verification; returns the device tensor of T*N records (uint8 [T*N, 64])."""
+    T = dtypes.numel()
+    dev = ref_buf.device
+    if results is None:
+        results = torch.empty((max(T * N, 1), 64), dtype=torch.uint8, device=dev)
+    if workspace is None:
+        workspace = torch.empty(gv_workspace_bytes(T, N), dtype=torch.uint8, device=dev)
+    t = _tol(atol, rtol, equal_nan)
+    rc = lib.gv_verify_ragged(ref_buf.data_ptr(), ref_off.data_ptr(), cand_buf.data_ptr(), cand_off.data_ptr(),
+                              dtypes.data_ptr(), n_elems.data_ptr() if n_elems is not None else None, T, N,
+                              ctypes.byref(t), results.data_ptr(), workspace.data_ptr(), workspace.numel(),
+                              _stream_ptr(stream))
+    _raise(rc)
+    return results[:T * N]
+
+
+def gv_hash(buf: torch.Tensor, out: Optional[torch.Tensor] = None,
+            stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:
+    """Enqueue the content hash of ``buf``'s bytes; returns a device int64 tensor holding the u64 hash."""
+    if out is None:
+        out = torch.empty(1, dtype=torch.int64, device=buf.device)
+    rc = lib.gv_hash(buf.data_ptr(), buf.numel() * buf.element_size(), out.data_ptr(), _stream_ptr(stream))
+    _raise(rc)
+    return out
+
+
+def gv_check(workspace: torch.Tensor, stream: Optional[torch.cuda.Stream] = None) -> int:
+    return int(lib.gv_check(workspace.data_ptr(), _stream_ptr(stream)))
+
+
+def gv_host_staging_bytes(n_elems: int, dt: int, slab: int) -> int:
+    return int(lib.gv_host_staging_bytes(n_elems, dt, slab))
+
+
+def gv_verify_batch_host(ref: torch.Tensor, cands: Sequence[torch.Tensor], atol: float, rtol: float,
+                         equal_nan: bool, staging: torch.Tensor, results: Optional[np.ndarray] = None,
+                         want_ref_hash: bool = True, stream: Optional[torch.cuda.Stream] = None):
+    """Host tensors in, host records out (synchronous). ``staging`` is a device uint8 buffer."""
+    dt = DTYPE_OF[ref.dtype]
+    N = len(cands)
+    if results is None:
+        results = np.zeros(max(N, 1), dtype=RESULT_DTYPE)
+    ref_hash = np.zeros(1, dtype=np.uint64)
+    ptrs = (ctypes.c_void_p * max(N, 1))(*[c.data_ptr() for c in cands])
+    t = _tol(atol, rtol, equal_nan)
+    rc = lib.gv_verify_batch_host(ref.data_ptr(), ctypes.cast(ptrs, ctypes.c_void_p), N, ref.numel(), dt,
+                                  ctypes.byref(t), results.ctypes.data_as(ctypes.c_void_p),
+                                  ref_hash.ctypes.data_as(ctypes.c_void_p) if want_ref_hash else None,
+                                  staging.data_ptr(), staging.numel(), _stream_ptr(stream))
+    _raise(rc)
+    return results[:N], int(ref_hash[0])

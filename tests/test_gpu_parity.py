@@ -1,0 +1,342 @@
+"""GPU parity: the CUDA library, called through its C ABI, against the CPU oracle, record by record
+and byte by byte (tolerance 0: every field of every record must be identical). Sizes here are ones
+the oracle finishes in seconds; they span several tiles, ragged tails, unaligned bases, more than one
+candidate chunk and more than one launch. Full-size workloads are in test_gpu_full_size.py."""
+import ctypes
+
+import numpy as np
+import pytest
+import torch
+
+pytestmark = pytest.mark.gpu
+
+if not torch.cuda.is_available():          # collected everywhere, run only where a GPU exists
+    pytest.skip("no CUDA device", allow_module_level=True)
+
+from paper_2507_23194_b200 import gv, workloads as W  # noqa: E402
+
+DEV = "cuda:0"
+TDT = {0: torch.float32, 1: torch.bfloat16, 2: torch.float16, 3: torch.int32, 4: torch.int64}
+ESZ = {0: 4, 1: 2, 2: 2, 3: 4, 4: 8}
+
+
+def host_bytes(t: torch.Tensor) -> np.ndarray:
+    """Raw bytes of a tensor as a numpy uint8 array (what the oracle consumes)."""
+    return t.detach().contiguous().view(torch.uint8).cpu().numpy()
+
+
+def oracle_batch(oracle, wl_ref, cands, code, atol, rtol, equal_nan):
+    r = host_bytes(wl_ref)
+    return oracle.verify_batch(r, [host_bytes(c) for c in cands], code, atol, rtol, equal_nan)
+
+
+def assert_records_equal(got: np.ndarray, want: np.ndarray, tag=""):
+    assert got.shape == want.shape, tag
+    if got.tobytes() != want.tobytes():
+        for j in range(len(got)):
+            if got[j].tobytes() != want[j].tobytes():
+                raise AssertionError(f"{tag}: record {j} differs\n gpu    {got[j]}\n oracle {want[j]}")
+
+
+def run_dense(ref, cands, atol, rtol, equal_nan, want_ref_hash=True):
+    rh = torch.zeros(1, dtype=torch.int64, device=DEV) if want_ref_hash else None
+    ws = torch.empty(gv.gv_workspace_bytes(0, len(cands)), dtype=torch.uint8, device=DEV)
+    res = gv.gv_verify_batch(ref, cands, atol, rtol, equal_nan, ref_hash=rh, workspace=ws)
+    torch.cuda.synchronize()
+    assert gv.gv_check(ws) == gv.GV_OK
+    out = gv.results_to_numpy(res)
+    return out, (int(rh.cpu().numpy().view(np.uint64)[0]) if want_ref_hash else None)
+
+
+# ------------------------------------------------------------------------------------------------
+# gv_hash
+# ------------------------------------------------------------------------------------------------
+def test_hash_all_small_sizes_and_offsets(oracle):
+    g = torch.Generator(device="cpu").manual_seed(11)
+    data = torch.randint(0, 256, (5000,), generator=g, dtype=torch.uint8)
+    dev = data.to(DEV)
+    sizes = list(range(0, 80)) + [255, 256, 257, 1023, 1024, 4095, 4096, 4097, 4113, 4999]
+    for off in (0, 1, 3, 8, 16):
+        for nb in sizes:
+            if off + nb > 5000:
+                continue
+            got = int(gv.gv_hash(dev[off:off + nb]).cpu().numpy().view(np.uint64)[0])
+            assert got == oracle.hash_bytes(data[off:off + nb].numpy()), (off, nb)
+
+
+def test_hash_large_and_config1_tensors(oracle):
+    wl = W.config1(DEV)
+    for c in [wl.ref] + wl.cands:
+        got = int(gv.gv_hash(c).cpu().numpy().view(np.uint64)[0])
+        assert got == oracle.hash_bytes(host_bytes(c))
+    z = torch.zeros(1 << 20, dtype=torch.float32, device=DEV)
+    assert int(gv.gv_hash(z).cpu().numpy().view(np.uint64)[0]) == 0x8C6F9C0F16C4607B
+    big = torch.randint(-2 ** 31, 2 ** 31 - 1, (50_000_001,), dtype=torch.int32, device=DEV)
+    assert int(gv.gv_hash(big).cpu().numpy().view(np.uint64)[0]) == oracle.hash_bytes(host_bytes(big))
+
+
+# ------------------------------------------------------------------------------------------------
+# dense: config 1 in full (the tiny correctness case), by-construction facts and oracle parity
+# ------------------------------------------------------------------------------------------------
+def test_config1_full(oracle):
+    wl = W.config1(DEV)
+    got, rh = run_dense(wl.ref, wl.cands, wl.atol, wl.rtol, wl.equal_nan)
+    want = oracle_batch(oracle, wl.ref, wl.cands, oracle.F32, wl.atol, wl.rtol, wl.equal_nan)
+    assert_records_equal(got, want, "config1")
+    assert rh == oracle.hash_bytes(host_bytes(wl.ref))
+    # by construction (independent of either implementation)
+    for j, f in enumerate(wl.facts):
+        if "n_mismatch" in f:
+            assert int(got[j]["n_mismatch"]) == f["n_mismatch"]
+            assert int(got[j]["first_mismatch"]) == (gv.GV_NO_INDEX if f["first"] is None else f["first"])
+        assert int(got[j]["n_nan_disagree"]) == f["n_nan"] and int(got[j]["n_inf_disagree"]) == f["n_inf"]
+    assert got[4].tobytes() == got[2].tobytes()
+    assert got[5]["max_rel_err"] == np.float32(2.0) and got[6]["max_rel_err"] == np.float32(1.0)
+    assert int(got[0]["hash"]) == rh and int(got[6]["hash"]) == 0x8C6F9C0F16C4607B
+    # invariance to candidate order: permuting the pointer list permutes the records
+    perm = [3, 0, 7, 5, 1, 6, 2, 4]
+    got_p, _ = run_dense(wl.ref, [wl.cands[i] for i in perm], wl.atol, wl.rtol, wl.equal_nan)
+    for pos, src in enumerate(perm):
+        assert got_p[pos].tobytes() == got[src].tobytes()
+
+
+# ------------------------------------------------------------------------------------------------
+# dense: sizes x dtypes x alignments, random data with injected specials
+# ------------------------------------------------------------------------------------------------
+def make_pair(code, n, seed, n_cands, specials=True):
+    g = torch.Generator(device="cpu").manual_seed(seed)
+    if code in (3, 4):
+        lo, hi = (-(1 << 31), (1 << 31) - 1) if code == 3 else (-(1 << 62), (1 << 62))
+        r = torch.randint(lo, hi, (n,), generator=g, dtype=TDT[code])
+        cands = []
+        for j in range(n_cands):
+            c = r.clone()
+            if n and j % 3 != 0:
+                k = max(1, n // (50 * (j + 1)))
+                pos = torch.randint(0, n, (k,), generator=g)
+                c[pos] = torch.randint(lo, hi, (k,), generator=g, dtype=TDT[code])
+            cands.append(c)
+        if code == 4 and n >= 4 and n_cands >= 2:
+            r[0], cands[1][0] = -(1 << 63), (1 << 63) - 1      # extreme difference, exact in u64
+        return r, cands
+    r = torch.randn(n, generator=g, dtype=torch.float32)
+    if specials and n >= 64:
+        pos = torch.randint(0, n, (12,), generator=g)
+        r[pos[0:2]] = float("nan")
+        r[pos[2:4]] = float("inf")
+        r[pos[4:6]] = float("-inf")
+        r[pos[6:9]] = 0.0
+        r[pos[9:12]] = -0.0
+    r = r.to(TDT[code])
+    cands = []
+    for j in range(n_cands):
+        kind = j % 6
+        rf = r.float()
+        if kind == 0:
+            c = r.clone()
+        elif kind == 1:
+            c = (rf * (1 + 1e-3 * torch.randn(n, generator=g))).to(TDT[code])
+        elif kind == 2:
+            c = (rf + 0.05 * torch.randn(n, generator=g)).to(TDT[code])
+        elif kind == 3:
+            c = r.clone()
+            if n:
+                pos = torch.randint(0, n, (max(1, n // 100),), generator=g)
+                vals = torch.tensor([float("nan"), float("inf"), float("-inf"), 0.0, 1e30, -1e30])
+                c[pos] = vals[torch.randint(0, 6, (pos.numel(),), generator=g)].to(TDT[code])
+        elif kind == 4:
+            c = torch.zeros_like(r)
+        else:
+            c = (-rf).to(TDT[code])
+        cands.append(c)
+    return r, cands
+
+
+SIZES = [0, 1, 2, 3, 7, 8, 9, 15, 16, 17, 255, 1023, 1024, 1025, 2047, 2048, 2049, 4096, 4100, 8191, 8192, 8193,
+         12289, 20000, 65536 + 5]
+
+
+@pytest.mark.parametrize("code", [0, 1, 2, 3, 4])
+def test_dense_size_sweep(oracle, code):
+    for i, n in enumerate(SIZES):
+        r, cands = make_pair(code, n, 100 + i, n_cands=7)
+        rd, cd = r.to(DEV), [c.to(DEV) for c in cands]
+        for atol, rtol, en in [(1e-2, 1e-2, False), (0.0, 0.0, True)]:
+            got, rh = run_dense(rd, cd, atol, rtol, en)
+            want = oracle.verify_batch(host_bytes(r), [host_bytes(c) for c in cands], code, atol, rtol, en)
+            assert_records_equal(got, want, f"dtype {code} n {n} tol {atol}")
+            assert rh == oracle.hash_bytes(host_bytes(r))
+
+
+@pytest.mark.parametrize("code", [0, 1, 2, 3, 4])
+def test_dense_unaligned_bases(oracle, code):
+    # reference and candidates start at element offsets 0..3 inside larger buffers (not 16-byte aligned)
+    n = 9000
+    for shift_r, shift_c in [(1, 0), (0, 1), (1, 1), (3, 2), (2, 3)]:
+        r, cands = make_pair(code, n + 8, 7 + shift_r, n_cands=5)
+        rd = r.to(DEV)[shift_r:shift_r + n]
+        cd = [c.to(DEV)[(shift_c + j) % 4:(shift_c + j) % 4 + n] for j, c in enumerate(cands)]
+        got, rh = run_dense(rd, cd, 1e-2, 1e-2, True)
+        want = oracle.verify_batch(host_bytes(rd), [host_bytes(c) for c in cd], code, 1e-2, 1e-2, True)
+        assert_records_equal(got, want, f"dtype {code} shifts {shift_r},{shift_c}")
+        assert rh == oracle.hash_bytes(host_bytes(rd))
+
+
+@pytest.mark.parametrize("code,n_cands", [(1, 17), (0, 33), (3, 40), (2, 300)])
+def test_dense_many_candidates(oracle, code, n_cands):
+    # more than one chunk of candidates; 300 > the per-launch pointer limit
+    n = 30000 if n_cands < 100 else 5000
+    r, cands = make_pair(code, n, 42, n_cands)
+    got, _ = run_dense(r.to(DEV), [c.to(DEV) for c in cands], 1e-2, 1e-2, False)
+    want = oracle.verify_batch(host_bytes(r), [host_bytes(c) for c in cands], code, 1e-2, 1e-2, False)
+    assert_records_equal(got, want, f"dtype {code} N {n_cands}")
+
+
+@pytest.mark.parametrize("code", [1, 2])
+def test_all_16bit_patterns_against_interesting_references(oracle, code):
+    raw_c = torch.arange(1 << 16, dtype=torch.int32).to(torch.int16).view(TDT[code])
+    refs = ([0x0000, 0x8000, 0x0001, 0x0080, 0x3F80, 0xBF80, 0x7F7F, 0xFF7F, 0x7F80, 0xFF80, 0x7FC0, 0x3F7F, 0x4049]
+            if code == 1 else
+            [0x0000, 0x8000, 0x0001, 0x03FF, 0x0400, 0x3C00, 0xBC00, 0x7BFF, 0xFBFF, 0x7C00, 0xFC00, 0x7E00, 0x4248])
+    cd = raw_c.to(DEV)
+    for rb in refs:
+        r = torch.full((1 << 16,), rb, dtype=torch.int32).to(torch.int16).view(TDT[code])
+        for atol, rtol, en in [(1e-2, 1e-2, False), (0.0, 0.0, True), (1e30, 1e30, False)]:
+            got, _ = run_dense(r.to(DEV), [cd], atol, rtol, en)
+            want = oracle.verify_batch(host_bytes(r), [host_bytes(raw_c)], code, atol, rtol, en)
+            assert_records_equal(got, want, f"dtype {code} ref {rb:#x} tol {atol}")
+
+
+def test_fp32_canaries_and_extremes(oracle):
+    # the golden truth-table rows as one batch, each row its own 1-element call, plus a tensor of
+    # extreme values crossed with itself
+    bits = np.array([0x00000000, 0x80000000, 0x00000001, 0x80000001, 0x007FFFFF, 0x00800000, 0x00800001,
+                     0x3F800000, 0xBF800000, 0x7F7FFFFF, 0xFF7FFFFF, 0x7F800000, 0xFF800000, 0x7FC00000,
+                     0xFFC00001, 0x3F7FFFFF, 0x3F800001, 0x7F61B1E6, 0xFF61B1E6, 0xBF38FA9F, 0xBF38F97E,
+                     0x3F640C03, 0x3F68E32C, 0x3A78DE92, 0x3F8A0F08], dtype=np.uint32)
+    c = torch.from_numpy(np.repeat(bits, len(bits)).view(np.float32).copy())
+    r = torch.from_numpy(np.tile(bits, len(bits)).view(np.float32).copy())
+    for atol, rtol, en in [(0.0, 0.0, False), (1e-5, 1e-5, False), (1e-2, 1e-2, True), (0.0, 2.0, False),
+                           (1e30, 1e30, True)]:
+        got, _ = run_dense(r.to(DEV), [c.to(DEV)], atol, rtol, en)
+        want = oracle.verify_batch(host_bytes(r), [host_bytes(c)], oracle.F32, atol, rtol, en)
+        assert_records_equal(got, want, f"extremes tol {atol},{rtol}")
+        # element by element too, so compensating errors cannot hide in the aggregate
+        if (atol, rtol) in [(1e-5, 1e-5), (0.0, 2.0)]:
+            cd, rd = c.to(DEV), r.to(DEV)
+            singles = [cd[i:i + 1].clone() for i in range(0, len(c), 7)]
+            for i, s in zip(range(0, len(c), 7), singles):
+                g1, _ = run_dense(rd[i:i + 1].clone(), [s], atol, rtol, en, want_ref_hash=False)
+                w1 = oracle.verify(host_bytes(r[i:i + 1]), host_bytes(c[i:i + 1]), oracle.F32, atol, rtol, en)
+                assert g1[0].tobytes() == w1.tobytes(), (i, g1[0], w1)
+
+
+def test_dense_empty_inputs(oracle):
+    r = torch.zeros(0, dtype=torch.float32, device=DEV)
+    got, rh = run_dense(r, [r.clone(), r.clone()], 1e-3, 1e-3, False)
+    for rec in got:
+        assert int(rec["n_mismatch"]) == 0 and int(rec["first_mismatch"]) == gv.GV_NO_INDEX
+        assert int(rec["hash"]) == 0 and rec["max_abs_err"] == 0 and rec["max_rel_err"] == 0
+    assert rh == 0
+    r = torch.randn(1000, device=DEV)
+    got, rh = run_dense(r, [], 1e-3, 1e-3, False)
+    assert len(got) == 0 and rh == oracle.hash_bytes(host_bytes(r))
+
+
+def test_results_independent_of_schedule(oracle):
+    # the same data verified as one batch, as single-candidate calls and in another order
+    r, cands = make_pair(1, 70001, 5, 9)
+    rd, cd = r.to(DEV), [c.to(DEV) for c in cands]
+    a, _ = run_dense(rd, cd, 1e-2, 1e-2, True)
+    for j in range(9):
+        b, _ = run_dense(rd, [cd[j]], 1e-2, 1e-2, True)
+        assert a[j].tobytes() == b[0].tobytes()
+    c, _ = run_dense(rd, cd[::-1], 1e-2, 1e-2, True)
+    assert c[::-1].tobytes() == a.tobytes()
+
+
+# ------------------------------------------------------------------------------------------------
+# reduced versions of the dense workload recipes
+# ------------------------------------------------------------------------------------------------
+def test_reduced_configs_2_3_4(oracle):
+    for wl in (W.config2(DEV, n=(1 << 18) + 24, n_cands=40), W.config3(DEV, n=(1 << 18) + 8, n_cands=10),
+               W.config4(DEV, n=1 << 18, n_cands=12), W.config4(DEV, n=(1 << 17) + 2, n_cands=12, wide=True)):
+        got, rh = run_dense(wl.ref, wl.cands, wl.atol, wl.rtol, wl.equal_nan)
+        want = oracle_batch(oracle, wl.ref, wl.cands, wl.dtype, wl.atol, wl.rtol, wl.equal_nan)
+        assert_records_equal(got, want, wl.name)
+        for j, f in enumerate(wl.facts):
+            if "n_mismatch" in f:
+                assert int(got[j]["n_mismatch"]) == f["n_mismatch"], (wl.name, j)
+            if f.get("hash_equals_ref"):
+                assert int(got[j]["hash"]) == rh
+
+
+# ------------------------------------------------------------------------------------------------
+# ragged
+# ------------------------------------------------------------------------------------------------
+def run_ragged(wl, with_counts=True):
+    ws = torch.empty(gv.gv_workspace_bytes(wl.T, wl.N), dtype=torch.uint8, device=DEV)
+    res = gv.gv_verify_ragged(wl.ref_buf, wl.ref_off, wl.cand_buf, wl.cand_off, wl.dtypes, wl.N, wl.atol, wl.rtol,
+                              wl.equal_nan, n_elems=wl.n_elems_t if with_counts else None, workspace=ws)
+    torch.cuda.synchronize()
+    return gv.results_to_numpy(res), gv.gv_check(ws)
+
+
+def oracle_ragged(oracle, wl):
+    return oracle.verify_ragged(wl.ref_buf.cpu().numpy(), wl.ref_off.cpu().numpy(), wl.cand_buf.cpu().numpy(),
+                                wl.cand_off.cpu().numpy(), wl.dtypes.cpu().numpy(), wl.N, wl.atol, wl.rtol,
+                                wl.equal_nan, n_elems=wl.n_elems_t.cpu().numpy())
+
+
+@pytest.mark.parametrize("align", [16, 0])
+def test_ragged_reduced_config5(oracle, align):
+    wl = W.config5(DEV, T=300, max_log2=16.0, align=align)
+    got, status = run_ragged(wl)
+    assert status == gv.GV_OK
+    want = oracle_ragged(oracle, wl)
+    assert_records_equal(got, want, f"ragged align {align}")
+    for i, f in enumerate(wl.facts):
+        assert int(got[i]["n_mismatch"]) == f["n_mismatch"]
+        assert int(got[i]["first_mismatch"]) == (gv.GV_NO_INDEX if f["first"] is None else f["first"])
+
+
+def test_ragged_counts_from_offsets_and_bad_table(oracle):
+    # tightly packed int32 tensors: element counts read off consecutive offsets
+    g = torch.Generator(device="cpu").manual_seed(3)
+    sizes = [0, 1, 5, 4096, 4097, 10000, 3]
+    offs = np.concatenate([[0], np.cumsum([4 * s for s in sizes])]).astype(np.int64)
+    total = int(offs[-1])
+    ref = torch.randint(-100, 100, (total // 4,), generator=g, dtype=torch.int32)
+    N = 3
+    cand = torch.cat([ref.clone() for _ in range(N)])
+    cand[5] += 1
+    cand_off = np.array([[offs[t] + j * total for j in range(N)] for t in range(len(sizes))], dtype=np.int64).reshape(-1)
+    dtypes = torch.full((len(sizes),), 3, dtype=torch.uint8)
+    ws = torch.empty(gv.gv_workspace_bytes(len(sizes), N), dtype=torch.uint8, device=DEV)
+    args = (ref.view(torch.uint8).to(DEV), torch.from_numpy(offs).to(DEV), cand.view(torch.uint8).to(DEV),
+            torch.from_numpy(cand_off).to(DEV), dtypes.to(DEV), N, 0.0, 0.0, False)
+    res = gv.gv_verify_ragged(*args, workspace=ws)
+    torch.cuda.synchronize()
+    assert gv.gv_check(ws) == gv.GV_OK
+    want = oracle.verify_ragged(host_bytes(ref), offs, host_bytes(cand), cand_off, dtypes.numpy(), N, 0.0, 0.0, False)
+    assert_records_equal(gv.results_to_numpy(res), want, "ragged tight int32")
+    # a decreasing offset is flagged, not followed
+    bad = offs.copy()
+    bad[3] = bad[2] - 8
+    res = gv.gv_verify_ragged(args[0], torch.from_numpy(bad).to(DEV), *args[2:], workspace=ws)
+    torch.cuda.synchronize()
+    assert gv.gv_check(ws) == gv.GV_ERR_BAD_TABLE
+
+
+# ------------------------------------------------------------------------------------------------
+# host-buffer entry point
+# ------------------------------------------------------------------------------------------------
+def test_verify_batch_host(oracle):
+    r, cands = make_pair(1, 50003, 9, 11)
+    rp, cp = r.pin_memory(), [c.pin_memory() for c in cands]
+    for slab in (1, 4, 64):
+        staging = torch.empty(gv.gv_host_staging_bytes(r.numel(), 1, slab), dtype=torch.uint8, device=DEV)
+        got, rh = gv.gv_verify_batch_host(rp, cp, 1e-2, 1e-2, True, staging)
+        want = oracle.verify_batch(host_bytes(r), [host_bytes(c) for c in cands], 1, 1e-2, 1e-2, True)
+        assert_records_equal(got, want, f"host entry slab {slab}")
+        assert rh == oracle.hash_bytes(host_bytes(r))

@@ -1,0 +1,105 @@
+"""Host-side checks that need no GPU: the C-ABI library loads, exports every symbol the header
+declares, and rejects bad arguments before touching the device (nothing is launched here)."""
+import ctypes
+import os
+import re
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def gvlib():
+    from paper_2507_23194_b200 import build as B
+    B.build()
+    from paper_2507_23194_b200 import gv
+    return gv
+
+
+def test_header_symbols_are_exported(gvlib):
+    hdr = open(os.path.join(ROOT, "include", "gv.h")).read()
+    hdr = re.sub(r"/\*.*?\*/", "", hdr, flags=re.S)
+    declared = set(re.findall(r"\b(gv_[a-z_]+)\s*\(", hdr))
+    assert {"gv_verify_batch", "gv_verify_ragged", "gv_hash"} <= declared
+    for name in declared:
+        assert hasattr(gvlib.lib, name), f"{name} is declared in gv.h but not exported"
+    assert declared == set(gvlib.EXPORTS), "binding and header disagree on the entry points"
+
+
+def test_version_and_strings(gvlib):
+    assert gvlib.gv_version() >= 0x000100
+    assert gvlib.lib.gv_status_string(0) == b"ok"
+    for s in range(1, 8):
+        assert len(gvlib.lib.gv_status_string(s)) > 0
+    assert gvlib.gv_workspace_bytes(0, 8) >= 256
+    assert gvlib.gv_workspace_bytes(10000, 4) >= 256 + 8 * 10001
+    assert gvlib.lib.gv_host_staging_bytes(1000, 1, 0) == 0
+
+
+def test_result_layout(gvlib):
+    assert gvlib.RESULT_DTYPE.itemsize == 64
+    assert gvlib.RESULT_DTYPE.fields["hash"][1] == 32
+    assert gvlib.RESULT_DTYPE.fields["max_abs_err"][1] == 48
+    assert gvlib.RESULT_DTYPE.fields["max_rel_err"][1] == 52
+
+
+def _call_batch(gv, ref=0x1000, cands=(0x2000,), N=1, n=16, dt=0, atol=1e-3, rtol=1e-3, results=0x3000,
+                ref_hash=None, ws=0x4000, ws_bytes=4096, tol_null=False):
+    ptrs = (ctypes.c_void_p * max(1, len(cands)))(*cands)
+    t = gv.gv_tol(atol, rtol, 0, 0)
+    return gv.lib.gv_verify_batch(ref, ctypes.cast(ptrs, ctypes.c_void_p), N, n, dt,
+                                  None if tol_null else ctypes.byref(t), results, ref_hash, ws, ws_bytes, None)
+
+
+def test_dense_argument_errors_return_before_any_launch(gvlib):
+    gv = gvlib
+    assert _call_batch(gv, dt=5) == gv.GV_ERR_UNSUPPORTED
+    assert _call_batch(gv, dt=-1) == gv.GV_ERR_UNSUPPORTED
+    assert _call_batch(gv, N=-1) == gv.GV_ERR_INVALID_ARG
+    assert _call_batch(gv, ref=None) == gv.GV_ERR_INVALID_ARG
+    assert _call_batch(gv, results=None) == gv.GV_ERR_INVALID_ARG
+    assert _call_batch(gv, cands=(None,)) == gv.GV_ERR_INVALID_ARG
+    assert _call_batch(gv, atol=float("nan")) == gv.GV_ERR_INVALID_ARG
+    assert _call_batch(gv, rtol=-1.0) == gv.GV_ERR_INVALID_ARG
+    assert _call_batch(gv, atol=float("inf")) == gv.GV_ERR_INVALID_ARG
+    assert _call_batch(gv, tol_null=True) == gv.GV_ERR_INVALID_ARG
+    assert _call_batch(gv, ws=None) == gv.GV_ERR_WORKSPACE
+    assert _call_batch(gv, ws_bytes=8) == gv.GV_ERR_WORKSPACE
+    assert _call_batch(gv, ws=0x4004) == gv.GV_ERR_WORKSPACE
+    assert _call_batch(gv, ref=0x1002) == gv.GV_ERR_MISALIGNED            # fp32 needs 4-byte alignment
+    assert _call_batch(gv, cands=(0x2001,), dt=1) == gv.GV_ERR_MISALIGNED   # bf16 needs 2-byte alignment
+    assert _call_batch(gv, results=0x3004) == gv.GV_ERR_MISALIGNED
+    assert _call_batch(gv, n=1 << 62) == gv.GV_ERR_INVALID_ARG
+    # integer dtypes ignore tolerances, so a null tol is fine for them -- but then the call would
+    # launch, which needs a device; only check that validation does not reject it for the tolerance
+    assert _call_batch(gv, dt=3, tol_null=True, ws=None) == gv.GV_ERR_WORKSPACE
+
+
+def test_ragged_and_hash_argument_errors(gvlib):
+    gv = gvlib
+    t = gv.gv_tol(1e-3, 1e-3, 0, 0)
+    f = gv.lib.gv_verify_ragged
+    ok_args = [0x1000, 0x2000, 0x3000, 0x4000, 0x5000, None, 4, 2, ctypes.byref(t), 0x6000, 0x7000, 1 << 20, None]
+
+    def call(**kw):
+        a = list(ok_args)
+        names = ["ref_base", "ref_off", "cand_base", "cand_off", "dtypes", "n_elems", "T", "N", "tol", "results",
+                 "ws", "ws_bytes", "stream"]
+        for k, v in kw.items():
+            a[names.index(k)] = v
+        return f(*a)
+
+    assert call(T=-1) == gv.GV_ERR_INVALID_ARG
+    assert call(N=-1) == gv.GV_ERR_INVALID_ARG
+    assert call(ref_off=None) == gv.GV_ERR_INVALID_ARG
+    assert call(dtypes=None) == gv.GV_ERR_INVALID_ARG
+    assert call(cand_off=None) == gv.GV_ERR_INVALID_ARG
+    assert call(tol=None) == gv.GV_ERR_INVALID_ARG
+    assert call(ws_bytes=16) == gv.GV_ERR_WORKSPACE
+    assert call(ws=None) == gv.GV_ERR_WORKSPACE
+    assert call(ref_off=0x2004) == gv.GV_ERR_MISALIGNED
+    assert gv.lib.gv_hash(0x1000, 16, None, None) == gv.GV_ERR_INVALID_ARG
+    assert gv.lib.gv_hash(None, 16, 0x1000, None) == gv.GV_ERR_INVALID_ARG
+    assert gv.lib.gv_hash(0x1000, 16, 0x1004, None) == gv.GV_ERR_MISALIGNED
+    assert gv.lib.gv_check(None, None) == gv.GV_ERR_INVALID_ARG

@@ -99,20 +99,23 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
-def build_workload(name: str, device):
+def build_workload(name: str, device, cands: int = 0, tensors: int = 0):
+    """``cands`` / ``tensors`` shrink the batch (fewer candidates, fewer ragged tensors) for small
+    profiling captures; 0 keeps the full recipe."""
     from paper_2507_23194_b200 import workloads as W
+    kw = {"n_cands": cands} if cands else {}
     if name == "cfg1":
         return W.config1(device)
     if name == "cfg2":
-        return W.config2(device)
+        return W.config2(device, **kw)
     if name == "cfg3":
-        return W.config3(device)
+        return W.config3(device, **kw)
     if name == "cfg4":
-        return W.config4(device)
+        return W.config4(device, **kw)
     if name == "cfg4w":
-        return W.config4(device, wide=True)
+        return W.config4(device, wide=True, **kw)
     if name == "cfg5":
-        return W.config5(device)
+        return W.config5(device, **({"T": tensors} if tensors else {}))
     raise SystemExit(f"unknown workload {name}")
 
 
@@ -156,7 +159,7 @@ def run_reference(args):
     if rank != 0:
         return
     device = "cuda:0" if torch.cuda.is_available() else "cpu"
-    wl = build_workload(args.workload, device)
+    wl = build_workload(args.workload, device, args.cands, args.tensors)
     vals, sample = [], ""
     per_step_budget = max(2.0, min(15.0, 120.0 / max(1, args.steps + args.warmup)))
     for i in range(args.warmup + args.steps):
@@ -190,6 +193,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg2")
+    ap.add_argument("--cands", type=int, default=0, help="fewer candidates than the recipe (profiling captures)")
+    ap.add_argument("--tensors", type=int, default=0, help="fewer ragged tensors than the recipe (profiling captures)")
+    ap.add_argument("--only-class", default="", help="keep only candidates of this recipe class (dense workloads)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
@@ -214,8 +220,13 @@ def main():
         dist.init_process_group("nccl", device_id=torch.device(device))
 
     from paper_2507_23194_b200 import gv, workloads as W
-    wl = build_workload(args.workload, device)
+    wl = build_workload(args.workload, device, args.cands, args.tensors)
     ragged = isinstance(wl, W.RaggedWorkload)
+    if args.only_class and not ragged:
+        keep = [j for j, f in enumerate(wl.facts) if f["class"] == args.only_class]
+        wl.cands = [wl.cands[j] for j in keep]
+        wl.facts = [wl.facts[j] for j in keep]
+        wl.name += ":" + args.only_class
 
     stream = torch.cuda.current_stream()
     if ragged:

@@ -37,6 +37,71 @@ __host__ __device__ inline int elem_size(int dt) {
 // ------------------------------------------------------------------------------------------
 // content hash
 // ------------------------------------------------------------------------------------------
+// The mixing function as the hot loops evaluate it. Integer add/shift/logic instructions and
+// integer multiply-add instructions execute on two different half-rate pipes of the SM; written
+// the plain way, the 64-bit xor-shifts and additions all land on the first and make it the
+// bottleneck of the whole kernel. Here part of them is expressed through 32x32->64 multiply-adds
+// by a power of two (z >> s and z << (32 - s) are the two halves of z * 2^(32 - s)), which moves
+// that work to the multiplier pipe. `two_pow` operands come from an opaque register so the
+// assembler keeps them as multiplies. Same value as the plain definition for every input
+// (checked bit for bit against the oracle).
+#ifndef GV_HASH_MASK
+#define GV_HASH_MASK 0x0
+#endif
+__device__ __forceinline__ uint32_t opaque_u32(uint32_t v) {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %1;" : "=r"(r) : "r"(v));
+    return r;
+}
+// (hi:lo) ^= (hi:lo) >> S for 0 < S < 32, shifts done by the multiplier pipe
+template <int S>
+__device__ __forceinline__ void xorshift_mul(uint32_t& lo, uint32_t& hi, uint32_t two_pow /* 2^(32-S) */) {
+    uint32_t p_lo, p_hi, t;
+    asm("{\n\t.reg .u64 p;\n\t"
+        "mul.wide.u32 p, %3, %5;\n\t"          // hi * 2^(32-S): low half = hi << (32-S), high half = hi >> S
+        "mov.b64 {%0, %1}, p;\n\t"
+        "mad.hi.u32 %2, %4, %5, %0;\n\t}"      // (lo >> S) + (hi << (32-S)): disjoint bits, + is |
+        : "=r"(p_lo), "=r"(p_hi), "=r"(t)
+        : "r"(hi), "r"(lo), "r"(two_pow));
+    lo ^= t;
+    hi ^= p_hi;
+}
+template <int S>
+__device__ __forceinline__ void xorshift_alu(uint32_t& lo, uint32_t& hi) {
+    const uint32_t t = __funnelshift_r(lo, hi, S);
+    lo ^= t;
+    hi ^= hi >> S;
+}
+__device__ __forceinline__ void mul64_const(uint32_t& lo, uint32_t& hi, uint32_t c_lo, uint32_t c_hi) {
+    const uint64_t p = static_cast<uint64_t>(lo) * c_lo;
+    hi = static_cast<uint32_t>(p >> 32) + lo * c_hi + hi * c_lo;
+    lo = static_cast<uint32_t>(p);
+}
+// MASK bit 0/1/2: xor-shift 30/27/31 through the multiplier; bit 3: the "+ gamma" through a wide multiply-add
+template <int MASK>
+__device__ __forceinline__ uint64_t splitmix64_split(uint32_t lo, uint32_t hi, uint32_t one, uint32_t p2, uint32_t p5,
+                                                     uint32_t p1) {
+    if (MASK & 8) {
+        uint32_t t_hi;
+        asm("{\n\t.reg .u64 p;\n\t"
+            "mad.wide.u32 p, %2, %3, 0x9E3779B97F4A7C15;\n\t"
+            "mov.b64 {%0, %1}, p;\n\t}"
+            : "=r"(lo), "=r"(t_hi)
+            : "r"(lo), "r"(one));
+        hi += t_hi;
+    } else {
+        const uint64_t z = ((static_cast<uint64_t>(hi) << 32) | lo) + 0x9E3779B97F4A7C15ull;
+        lo = static_cast<uint32_t>(z);
+        hi = static_cast<uint32_t>(z >> 32);
+    }
+    if (MASK & 1) xorshift_mul<30>(lo, hi, p2); else xorshift_alu<30>(lo, hi);
+    mul64_const(lo, hi, 0x1CE4E5B9u, 0xBF58476Du);
+    if (MASK & 2) xorshift_mul<27>(lo, hi, p5); else xorshift_alu<27>(lo, hi);
+    mul64_const(lo, hi, 0x133111EBu, 0x94D049BBu);
+    if (MASK & 4) xorshift_mul<31>(lo, hi, p1); else xorshift_alu<31>(lo, hi);
+    return (static_cast<uint64_t>(hi) << 32) | lo;
+}
+
 __device__ __forceinline__ uint64_t splitmix64(uint64_t x) {
     uint64_t z = x + 0x9E3779B97F4A7C15ull;
     z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
@@ -60,6 +125,20 @@ __device__ __forceinline__ uint64_t hash_vec_full(const uint4& v, uint64_t k0) {
     return splitmix64(k0 ^ pack64(v.x, v.y)) + splitmix64((k0 + 1) ^ pack64(v.z, v.w));
 }
 
+// Full vector whose word indices fit 32 bits (tensors below 32 GiB): the high half of the index is
+// zero, so only the low halves are xored.
+// Powers of two (and 1) held in registers the assembler cannot see through; see splitmix64_split.
+struct HashConsts {
+    uint32_t one, p2, p5, p1;
+    __device__ __forceinline__ void init() {
+        one = opaque_u32(1u); p2 = opaque_u32(1u << 2); p5 = opaque_u32(1u << 5); p1 = opaque_u32(1u << 1);
+    }
+};
+__device__ __forceinline__ uint64_t hash_vec_full_k32(const uint4& v, uint32_t k0, const HashConsts& hc) {
+    return splitmix64_split<GV_HASH_MASK>(v.x ^ k0, v.y, hc.one, hc.p2, hc.p5, hc.p1) +
+           splitmix64_split<GV_HASH_MASK>(v.z ^ (k0 + 1u), v.w, hc.one, hc.p2, hc.p5, hc.p1);
+}
+
 // ------------------------------------------------------------------------------------------
 // loads
 // ------------------------------------------------------------------------------------------
@@ -69,6 +148,26 @@ __device__ __forceinline__ uint4 ldg_stream(const void* p) {
     asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
                  : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
                  : "l"(p));
+    return v;
+}
+
+// Per-thread asynchronous 16-byte copy global -> shared (L2 only, bypasses L1) and its group
+// bookkeeping: each thread later reads back only the bytes it copied itself, so completion needs no
+// barrier, only the thread's own wait.
+__device__ __forceinline__ void cp_async16(uint32_t smem_dst, const void* gsrc) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_dst), "l"(gsrc) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() {
+    asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
+}
+__device__ __forceinline__ uint4 lds128(uint32_t smem_addr) {
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "r"(smem_addr)
+                 : "memory");
     return v;
 }
 
@@ -164,6 +263,32 @@ struct Acc {
     }
 };
 
+// Per-candidate accumulators of one CTA (shared memory). Rare quantities are updated with
+// shared-memory atomics from the compare path; the common ones once per flush.
+struct CtaAcc {
+    unsigned long long hash, cnt, first, nan, inf, maxint;
+    unsigned int maxabs, maxrel;
+    unsigned int thr;      // relative-error filter threshold derived from maxrel (see rel_threshold_bits)
+    unsigned int pad;
+    // thresholds of the packed 16-bit filters, both halves equal (see PackedFilter): mh2 from maxabs, thr2 from maxrel
+    unsigned int mh2, thr2;
+    // The candidate's record in global memory. Raised maxima are also sent there at once (max is
+    // idempotent, the record is their destination anyway) so that other CTAs can pick them up and
+    // tighten their own filters long before the chunk ends.
+    gv_result* rec;
+    __device__ __forceinline__ void clear() {
+        hash = 0; cnt = 0; first = ~0ull; nan = 0; inf = 0; maxint = 0; maxabs = 0; maxrel = 0; thr = 0; pad = 0;
+        mh2 = 0; thr2 = 0; rec = nullptr;
+    }
+};
+
+#ifdef GV_DEBUG_COUNTERS
+__device__ unsigned long long g_dbg[8];
+#define GV_COUNT(i) atomicAdd(&g_dbg[i], 1ull)
+#else
+#define GV_COUNT(i) ((void)0)
+#endif
+
 struct TolF {
     float atol, rtol;
     int equal_nan;
@@ -175,7 +300,12 @@ __device__ __forceinline__ bool is_finite_bits(uint32_t b) { return (b & 0x7F800
 
 // The per-element rule, written out once, exactly as the header states it. Used for every
 // element on the general path and for the elements of vectors the fast path cannot settle.
-__device__ __forceinline__ void element_rule(float c, float r, const TolF& t, uint64_t idx, Acc& a) {
+// GUARDED: the exact quotient is only needed when it can exceed the running maximum. Callers that
+// hold the reciprocal estimate `inv` of hoist_ref and a threshold from rel_threshold_bits pass them,
+// and the division is skipped for elements whose estimate |d| * inv cannot beat the maximum.
+template <bool GUARDED>
+__device__ __forceinline__ void element_rule(float c, float r, const TolF& t, uint64_t idx, Acc& a,
+                                             float inv = 0.0f, uint32_t thr_bits = 0u) {
     const uint32_t cb = __float_as_uint(c), rb = __float_as_uint(r);
     const float d = __fsub_rn(c, r);
     const float ad = fabsf(d);
@@ -196,10 +326,310 @@ __device__ __forceinline__ void element_rule(float c, float r, const TolF& t, ui
         const uint32_t adb = __float_as_uint(ad);          // ad >= +0, possibly +Inf by overflow
         a.maxabs = adb > a.maxabs ? adb : a.maxabs;
         if ((rb & 0x7FFFFFFFu) != 0u) {
-            const uint32_t q = __float_as_uint(__fdiv_rn(ad, fabsf(r)));
-            a.maxrel = q > a.maxrel ? q : a.maxrel;
+            bool need = true;
+            if (GUARDED) {
+                const float q = __fmul_rn(ad, inv);
+                need = (q > __uint_as_float(thr_bits)) || (thr_bits == 0u && adb != 0u);
+            }
+            if (need) {
+                const uint32_t qe = __float_as_uint(__fdiv_rn(ad, fabsf(r)));
+                a.maxrel = qe > a.maxrel ? qe : a.maxrel;
+            }
         }
     }
+}
+
+// ------------------------------------------------------------------------------------------
+// fast path for full, aligned vectors of float dtypes
+// ------------------------------------------------------------------------------------------
+__device__ __forceinline__ float max3(float a, float b, float c) {
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+__device__ __forceinline__ float max3_nan(float a, float b, float c) {     // NaN if any input is NaN
+    float d;
+    asm("max.NaN.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+__device__ __forceinline__ float max2_nan(float a, float b) {
+    float d;
+    asm("max.NaN.f32 %0, %1, %2;" : "=f"(d) : "f"(a), "f"(b));
+    return d;
+}
+
+// Values derived from one reference vector, computed once per tile and reused for every
+// candidate of the chunk.
+//   rf    reference widened to binary32
+//   ntol  -min(tol, FLT_MAX) with tol = fl(atol + fl(rtol*|r|)); |d| <= tolc  <=>  |d| < Inf and |d| <= tol
+//   inv   estimate of 1/|r| for the relative-error filter (hardware reciprocal) when 2^-100 <= |r| <= 2^100,
+//         0 when r == 0 (such elements have no relative error), +Inf otherwise (forces the exact path)
+template <int EPV>
+struct RefVec {
+    float rf[EPV], ntol[EPV], inv[EPV];
+};
+
+__device__ __forceinline__ float rcp_approx(float a) {      // one MUFU; relative error below 2^-22
+    float r;
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(a));
+    return r;
+}
+
+template <int DT>
+__device__ __forceinline__ void hoist_ref(const uint4& raw, const TolF& t, RefVec<16 / Traits<DT>::ESZ>& o,
+                                          uint32_t& force) {
+    constexpr int EPV = 16 / Traits<DT>::ESZ;
+    Widen<DT>::run(raw, o.rf);
+    uint32_t umax = 0u;
+#pragma unroll
+    for (int e = 0; e < EPV; ++e) {
+        const float a = fabsf(o.rf[e]);
+        const uint32_t u = __float_as_uint(a);
+        const float tol = __fadd_rn(t.atol, __fmul_rn(t.rtol, a));
+        o.ntol[e] = -fminf(tol, __uint_as_float(0x7F7FFFFFu));      // NaN tol -> FLT_MAX; r NaN makes d NaN anyway
+        // 2^-100 <= |r| <= 2^100: reciprocal estimate; r == 0: 0; anything else (tiny, huge, Inf, NaN): +Inf
+        const bool in_range = (u - 0x0D800000u) <= (0x71800000u - 0x0D800000u);
+        o.inv[e] = in_range ? rcp_approx(a) : (u == 0u ? 0.0f : __uint_as_float(0x7F800000u));
+        umax = u > umax ? u : umax;
+    }
+    // an identical candidate vector is "all close, nothing to record" unless the reference holds a
+    // NaN that does not count as equal
+    force = (umax > 0x7F800000u && !t.equal_nan) ? 0xFFFFFFFFu : 0u;
+}
+
+// Relative-error filter state of one (CTA, candidate): thr = bits of M * (1 - 2^-20) rounded down,
+// where M is the largest exact quotient recorded so far, or 0 while M < 2^-100.
+// With inv = (1/|r|)(1 + e1), |e1| < 2^-22 (hardware reciprocal estimate) and q = fl(|d| * inv) in the
+// normal range, fl(|d| / |r|) <= q * (1 + 2^-22 + 2^-23) < q * (1 + 2^-21); hence a quotient above M
+// implies q > M * (1 - 2^-21) > thr. While thr == 0 any nonzero |d| goes to the exact path.
+__device__ __forceinline__ uint32_t rel_threshold_bits(uint32_t m_bits) {
+    if (m_bits < 0x0D800000u) return 0u;                                  // M < 2^-100 (or 0)
+    if (m_bits >= 0x7F800000u) return 0x7F800000u;                        // M = +Inf: nothing can exceed it
+    return __float_as_uint(__fmul_rd(__uint_as_float(m_bits), __uint_as_float(0x3F7FFFF0u)));   // 1 - 2^-20
+}
+
+// Raise the CTA's running maxima (bit patterns of non-negative floats) and forward them to the record.
+__device__ __forceinline__ void raise_maxabs(CtaAcc* s, uint32_t bits) {
+    if (bits > *reinterpret_cast<volatile unsigned int*>(&s->maxabs)) {
+        atomicMax(&s->maxabs, bits);
+        if (s->rec) atomicMax(reinterpret_cast<unsigned int*>(&s->rec->max_abs_err), bits);
+    }
+}
+__device__ __forceinline__ void raise_maxrel(CtaAcc* s, uint32_t bits) {
+    if (bits > *reinterpret_cast<volatile unsigned int*>(&s->maxrel)) {
+        atomicMax(&s->maxrel, bits);
+        atomicMax(&s->thr, rel_threshold_bits(bits));
+        if (s->rec) atomicMax(reinterpret_cast<unsigned int*>(&s->rec->max_rel_err), bits);
+    }
+}
+
+// IEEE quotient for the (rare) elements whose estimate beats the filter; out of line to keep the
+// hot loop small.
+__device__ __noinline__ uint32_t exact_quotient_bits(float ad, float abs_r) {
+    return __float_as_uint(__fdiv_rn(ad, abs_r));
+}
+
+// Compare one full vector on the fast path. Returns true when the vector is settled: every element
+// is close with finite |d| (so every pair is a finite pair). Then max |d| and, for the elements whose
+// estimate passes the filter, the exact relative error are merged into the CTA accumulators here.
+// Returns false when the caller must run the exact per-element rule on this vector (nothing has
+// been recorded in that case).
+template <int DT>
+__device__ __forceinline__ bool vec_fast_float(const uint4& c, const RefVec<16 / Traits<DT>::ESZ>& r, CtaAcc* s) {
+    constexpr int EPV = 16 / Traits<DT>::ESZ;
+    float cf[EPV], ad[EPV], m[EPV], q[EPV];
+    Widen<DT>::run(c, cf);
+#pragma unroll
+    for (int e = 0; e < EPV; ++e) {
+        ad[e] = fabsf(__fsub_rn(cf[e], r.rf[e]));
+        m[e] = __fadd_rn(ad[e], r.ntol[e]);          // > 0 or NaN  <=>  not (|d| <= tolc)
+        q[e] = __fmul_rn(ad[e], r.inv[e]);           // NaN only from 0 * Inf, ignored by max
+    }
+    float vm, va, vq;
+    if (EPV == 8) {
+        vm = max2_nan(max3_nan(m[0], m[1], m[2]), max3_nan(max3_nan(m[3], m[4], m[5]), m[6], m[7]));
+        va = fmaxf(max3(ad[0], ad[1], ad[2]), max3(max3(ad[3], ad[4], ad[5]), ad[6], ad[7]));
+        vq = fmaxf(max3(q[0], q[1], q[2]), max3(max3(q[3], q[4], q[5]), q[6], q[7]));
+    } else {
+        vm = max2_nan(max3_nan(m[0], m[1], m[2]), m[3]);
+        va = fmaxf(max3(ad[0], ad[1], ad[2]), ad[3]);
+        vq = fmaxf(max3(q[0], q[1], q[2]), q[3]);
+    }
+    if (!(vm <= 0.0f)) return false;                                  // some element not close, or NaN
+    const uint32_t vab = __float_as_uint(va);
+    raise_maxabs(s, vab);
+    const uint32_t thr_bits = *reinterpret_cast<volatile unsigned int*>(&s->thr);
+    if ((vq > __uint_as_float(thr_bits)) || (thr_bits == 0u && vab != 0u)) {
+        // some element may raise the relative maximum: exact quotients for those that pass the filter
+        GV_COUNT(2);
+        uint32_t best = 0u;
+#pragma unroll
+        for (int e = 0; e < EPV; ++e) {
+            const bool need = (q[e] > __uint_as_float(thr_bits)) || (thr_bits == 0u && ad[e] != 0.0f);
+            // r.inv == 0 marks r == 0 (no relative error); q is then 0 or NaN and ad may be nonzero
+            if (need && r.inv[e] != 0.0f) {
+                const uint32_t qe = exact_quotient_bits(ad[e], fabsf(r.rf[e]));
+                best = qe > best ? qe : best;
+            }
+        }
+        raise_maxrel(s, best);
+    }
+    return true;
+}
+
+// ------------------------------------------------------------------------------------------
+// packed 16-bit filter for bf16 / fp16 vectors
+// ------------------------------------------------------------------------------------------
+// For the two 16-bit float types the common case is settled without widening, two elements per
+// instruction, in the type's own arithmetic. This is exact, not approximate, because of Sterbenz's
+// lemma: when |c - r| <= |r| / 2 the difference c - r is representable in the operands' format, so
+// the packed subtraction returns the very number the binary32 rule computes. Per element a bound
+//     b = RZ16( r == 0 ? tolc : min(tolc, 0.48 |r|) )        (tolc = min(tol, FLT_MAX), RZ16 = toward zero)
+// is derived once per reference tile. If a = |c -_16 r| <= b then (rounding error of the packed
+// subtraction at most 2^-8 relative) |c - r| < |r| / 2, hence a = |c - r| exactly, and a <= tolc: the
+// element is close and a finite pair (r == 0: c - 0 is exact anyway). What remains is whether a
+// raises the running max |d| (compare with mh = RZ16 of it: a > max  <=>  a > mh for 16-bit a) and
+// whether a / |r| can raise the running max relative error M: with inv = the smallest 16-bit number
+// >= 1 / |r| the product a * inv >= a / |r|; a rounded quotient can exceed M only if the real one does,
+// so a * inv > thr16 with thr16 <= M is a safe test, evaluated by one fused multiply-add whose sign
+// is exact while M >= kMinRel16 (below that mh is kept at 0, so every nonzero a is sent on). The three conditions are evaluated as
+// relu(a - b) + relu(a - mh) + relu(a * inv - thr16) summed over the vector; a nonzero (or NaN) sum
+// sends the vector to the binary32 path, which then decides everything by itself. Nothing is
+// recorded here, so a needless detour costs time only.
+template <int DT> struct Half2;
+template <> struct Half2<GV_BF16> {
+    static constexpr uint32_t kNegOne2 = 0xBF80BF80u;
+    static constexpr uint32_t kInf = 0x7F80u;
+    static constexpr uint32_t kMinRelBits = 0x0D800000u;          // 2^-100 as binary32
+    static constexpr bool kExactThr = true;                        // a * inv - thr never rounds to zero above kMinRel
+    static __device__ __forceinline__ float widen(uint32_t h) { return __uint_as_float(h << 16); }
+    static __device__ __forceinline__ uint32_t sub(uint32_t a, uint32_t b) { uint32_t d; asm("sub.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b)); return d; }
+    static __device__ __forceinline__ uint32_t add(uint32_t a, uint32_t b) { uint32_t d; asm("add.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b)); return d; }
+    static __device__ __forceinline__ uint32_t abs(uint32_t a) { uint32_t d; asm("abs.bf16x2 %0, %1;" : "=r"(d) : "r"(a)); return d; }
+    static __device__ __forceinline__ uint32_t fma_relu(uint32_t a, uint32_t b, uint32_t c) { uint32_t d; asm("fma.rn.relu.bf16x2 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c)); return d; }
+    // binary32 x >= 0 (or NaN) -> 16-bit pattern rounded toward zero / toward +Inf
+    static __device__ __forceinline__ uint32_t rz(float x) { return __float_as_uint(x) >> 16; }
+    static __device__ __forceinline__ uint32_t ru(float x) {
+        const uint32_t b = __float_as_uint(x);
+        return (b >> 16) + (((b & 0xFFFFu) != 0u && b < 0x7F800000u) ? 1u : 0u);
+    }
+};
+template <> struct Half2<GV_F16> {
+    static constexpr uint32_t kNegOne2 = 0xBC00BC00u;
+    static constexpr uint32_t kInf = 0x7C00u;
+    static constexpr uint32_t kMinRelBits = 0x39000000u;          // 2^-13 as binary32
+    static constexpr bool kExactThr = false;                       // small differences can round to zero: keep a margin
+    static __device__ __forceinline__ float widen(uint32_t h) { return f16_to_f32(h); }
+    static __device__ __forceinline__ uint32_t sub(uint32_t a, uint32_t b) { uint32_t d; asm("sub.f16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b)); return d; }
+    static __device__ __forceinline__ uint32_t add(uint32_t a, uint32_t b) { uint32_t d; asm("add.f16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b)); return d; }
+    static __device__ __forceinline__ uint32_t abs(uint32_t a) { uint32_t d; asm("abs.f16x2 %0, %1;" : "=r"(d) : "r"(a)); return d; }
+    static __device__ __forceinline__ uint32_t fma_relu(uint32_t a, uint32_t b, uint32_t c) { uint32_t d; asm("fma.rn.relu.f16x2 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c)); return d; }
+    static __device__ __forceinline__ uint32_t rz(float x) { unsigned short h; asm("cvt.rz.f16.f32 %0, %1;" : "=h"(h) : "f"(x)); return h; }
+    static __device__ __forceinline__ uint32_t ru(float x) { unsigned short h; asm("cvt.rp.f16.f32 %0, %1;" : "=h"(h) : "f"(x)); return h; }
+};
+
+struct PackedRef {
+    uint32_t b[4];      // per-element bounds, two per word, positive
+    uint32_t inv[4];    // RU16(1/|r|); 0 where r == 0; +Inf where the reciprocal overflows or r is not finite
+};
+
+template <int DT>
+__device__ __forceinline__ void hoist_packed(const uint4& raw, const TolF& t, PackedRef& o, uint32_t& force) {
+    float rf[8];
+    Widen<DT>::run(raw, rf);
+    uint32_t b16[8], i16[8], umax = 0u;
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+        const float a = fabsf(rf[e]);
+        const uint32_t u = __float_as_uint(a);
+        const float tolc = fminf(__fadd_rn(t.atol, __fmul_rn(t.rtol, a)), __uint_as_float(0x7F7FFFFFu));
+        float bound = fminf(tolc, __fmul_rn(a, 0.48f));
+        if (u == 0u) bound = tolc;
+        if (u >= 0x7F800000u) bound = 0.0f;                      // Inf or NaN reference: never settled here
+        b16[e] = Half2<DT>::rz(bound);
+        // inv = the smallest 16-bit number h with h * |r| >= 1, found from the hardware estimate by
+        // testing neighbours; the products of two 16-bit numbers are exact in binary32
+        const float x = rcp_approx(a);
+        uint32_t h = Half2<DT>::rz(__fmul_rd(x, __uint_as_float(0x3F7FFFF0u)));       // a little below 1/|r|
+        if (!(__fmul_rn(Half2<DT>::widen(h), a) >= 1.0f)) h += 1u;
+        if (!(__fmul_rn(Half2<DT>::widen(h), a) >= 1.0f)) h += 1u;
+        if (u == 0u) h = 0u;
+        if (u > 0x7E000000u) h = Half2<DT>::ru(__uint_as_float(0x01000000u));      // |r| > 2^125: 2^-125 >= 1/|r| (estimate may flush)
+        if (u >= 0x7F800000u || (u < 0x00800000u && u != 0u)) h = Half2<DT>::kInf;  // not finite, or binary32-subnormal
+        i16[e] = h;
+        umax = u > umax ? u : umax;
+    }
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        o.b[j] = b16[2 * j] | (b16[2 * j + 1] << 16);
+        o.inv[j] = i16[2 * j] | (i16[2 * j + 1] << 16);
+    }
+    force = (umax > 0x7F800000u && !t.equal_nan) ? 0xFFFFFFFFu : 0u;
+}
+
+// Nonzero result: the vector must go to the binary32 path. mh2 / thr2 are the packed thresholds of
+// the candidate's CTA accumulator (both halves equal).
+template <int DT>
+__device__ __forceinline__ uint32_t packed_filter(const uint4& c, const uint4& r, const PackedRef& pr, uint32_t mh2,
+                                                  uint32_t thr2) {
+    using H = Half2<DT>;
+    const uint32_t cw[4] = {c.x, c.y, c.z, c.w}, rw[4] = {r.x, r.y, r.z, r.w};
+    const uint32_t nthr2 = thr2 ^ 0x80008000u;
+    uint32_t t[12];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        const uint32_t a = H::abs(H::sub(cw[j], rw[j]));
+        t[3 * j] = H::fma_relu(pr.b[j], H::kNegOne2, a);           // relu(a - b)
+        t[3 * j + 1] = H::fma_relu(mh2, H::kNegOne2, a);           // relu(a - mh)
+        t[3 * j + 2] = H::fma_relu(a, pr.inv[j], nthr2);           // relu(a * inv - thr)
+    }
+#ifdef GV_DEBUG_COUNTERS
+    {
+        const uint32_t d1 = H::add(H::add(t[0], t[3]), H::add(t[6], t[9]));
+        const uint32_t d2 = H::add(H::add(t[1], t[4]), H::add(t[7], t[10]));
+        const uint32_t d3 = H::add(H::add(t[2], t[5]), H::add(t[8], t[11]));
+        if (d1) GV_COUNT(3);
+        if (d2) GV_COUNT(4);
+        if (d3) GV_COUNT(5);
+        if (thr2 == 0u) GV_COUNT(6);
+    }
+#endif
+    // pairwise sum (any NaN or positive term makes the sum nonzero)
+    const uint32_t s0 = H::add(H::add(t[0], t[1]), H::add(t[2], t[3]));
+    const uint32_t s1 = H::add(H::add(t[4], t[5]), H::add(t[6], t[7]));
+    const uint32_t s2 = H::add(H::add(t[8], t[9]), H::add(t[10], t[11]));
+    return H::add(H::add(s0, s1), s2);
+}
+
+// Packed thresholds from the binary32 accumulators (monotone: both only ever grow).
+template <int DT>
+__device__ __forceinline__ void refresh_packed_thresholds(CtaAcc* s) {
+    using H = Half2<DT>;
+    const uint32_t mrel = *reinterpret_cast<volatile unsigned int*>(&s->maxrel);
+    const uint32_t mabs = *reinterpret_cast<volatile unsigned int*>(&s->maxabs);
+    if (mrel < H::kMinRelBits) return;                          // keep both at 0: every nonzero |d| is sent on
+    uint32_t thr16, mh16;
+    // A quotient can only raise M when the real a/|r| exceeds M (rounding is monotone), and a * inv >= a/|r|.
+    // bf16: the fused a * inv - thr keeps its sign exactly, so thr = RZ16(M) -- equal quotients (ties of
+    // quantised data) do not fire. fp16: differences below 2^-25 round to zero, so thr sits 2^-10 lower.
+    if (mrel >= 0x7F800000u) thr16 = H::kInf;
+    else if (H::kExactThr) thr16 = H::rz(__uint_as_float(mrel));
+    else thr16 = H::rz(__fmul_rd(__uint_as_float(mrel), 1.0f - 1.0f / 1024.0f));
+    mh16 = H::rz(__uint_as_float(mabs));
+    atomicMax(&s->thr2, thr16 | (thr16 << 16));
+    atomicMax(&s->mh2, mh16 | (mh16 << 16));
+}
+
+// Exact per-element rule over a full vector, using the hoisted reference values (the path taken
+// by vectors the fast path could not settle).
+template <int DT>
+__device__ __forceinline__ void vec_exact_float(const uint4& c, const RefVec<16 / Traits<DT>::ESZ>& r,
+                                                uint64_t elem0, const TolF& t, uint32_t thr_bits, Acc& a) {
+    constexpr int EPV = 16 / Traits<DT>::ESZ;
+    float cf[EPV];
+    Widen<DT>::run(c, cf);
+#pragma unroll
+    for (int e = 0; e < EPV; ++e) element_rule<true>(cf[e], r.rf[e], t, elem0 + e, a, r.inv[e], thr_bits);
 }
 
 // One 16-byte vector of a float dtype, general path: every element through the rule.
@@ -213,7 +643,7 @@ __device__ __forceinline__ void vec_general_float(const uint4& c, const uint4& r
     Widen<DT>::run(r, rf);
 #pragma unroll
     for (int e = 0; e < EPV; ++e) {
-        if (e < nvalid) element_rule(cf[e], rf[e], t, elem0 + e, a);
+        if (e < nvalid) element_rule<false>(cf[e], rf[e], t, elem0 + e, a);
     }
 }
 
@@ -324,23 +754,17 @@ __device__ __forceinline__ uint64_t warp_max_u64(uint64_t v) {
     return v;
 }
 
-// Per-candidate accumulators of one CTA (shared memory). Rare quantities are updated with
-// shared-memory atomics from the compare path; the common ones once per flush.
-struct CtaAcc {
-    unsigned long long hash, cnt, first, nan, inf, maxint;
-    unsigned int maxabs, maxrel;
-    __device__ __forceinline__ void clear() {
-        hash = 0; cnt = 0; first = ~0ull; nan = 0; inf = 0; maxint = 0; maxabs = 0; maxrel = 0;
-    }
-};
-
 // Rare-path partials of one thread's visit -> CTA accumulators.
+// (Reads before the atomics keep hot addresses quiet: a value that cannot change the
+// accumulator is dropped without an atomic.)
 __device__ __forceinline__ void push_rare(CtaAcc* s, const Acc& a) {
-    if (a.cnt) atomicMin(&s->first, static_cast<unsigned long long>(a.first));
+    if (a.cnt && a.first < *reinterpret_cast<volatile unsigned long long*>(&s->first))
+        atomicMin(&s->first, static_cast<unsigned long long>(a.first));
     if (a.nan) atomicAdd(&s->nan, static_cast<unsigned long long>(a.nan));
     if (a.inf) atomicAdd(&s->inf, static_cast<unsigned long long>(a.inf));
-    if (a.maxint) atomicMax(&s->maxint, static_cast<unsigned long long>(a.maxint));
-    if (a.maxrel) atomicMax(&s->maxrel, a.maxrel);
+    if (a.maxint > *reinterpret_cast<volatile unsigned long long*>(&s->maxint))
+        atomicMax(&s->maxint, static_cast<unsigned long long>(a.maxint));
+    raise_maxrel(s, a.maxrel);
 }
 
 // CTA accumulators -> result record in global memory (skips identities).

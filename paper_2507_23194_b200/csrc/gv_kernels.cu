@@ -81,220 +81,384 @@ struct DenseParams {
     float atol, rtol;
     int equal_nan;
     int N;                      // candidates in this launch (<= kMaxPtrs)
+    int all_aligned;            // reference and every candidate base are 16-byte aligned
     const unsigned char* cands[kMaxPtrs];
 };
 
-// Shared-memory layout of the dense kernel (dynamic):
-//   [0, 2*TILE)                     two reference tile buffers (bulk-copy destinations, 128-B aligned)
-//   then uint4 slots[kChunk][kThreads]   per (candidate, thread): hash lo, hash hi, count, max|d| bits
-//   then CtaAcc acc[kChunk], two mbarriers
-template <int V>
+// Dense kernel, organisation.
+//   * Every warp works on its own: warp-tiles of 512 bytes (one 16-byte vector per lane), tile t
+//     belongs to warp (t mod number of warps in the grid). No CTA-wide barrier in steady state.
+//   * Reference: the warp's tile is brought into shared memory by one 512-byte bulk async copy (TMA)
+//     completing on the warp's own mbarrier, double buffered (the next tile's copy is in flight
+//     while the current tile is compared against the chunk). Each lane then holds its vector and the
+//     values derived from it in registers for all candidates of the chunk.
+//   * Candidates: each lane streams its own 16 bytes of every candidate with asynchronous 16-byte
+//     copies into a private ring in shared memory, kRing copies in flight per lane, and reads them
+//     back itself -- no registers are spent on data in flight and no barrier on its arrival.
+//   * Accumulators: the 64-bit hash partial of every (candidate of the chunk, lane) lives in a
+//     shared-memory slot for the whole chunk; max |d|, max relative error, counts and the first
+//     index go to per-CTA shared accumulators only when they can change them. One block combine
+//     and one set of global integer atomics per (CTA, candidate).
+#ifndef GV_UNROLL
+#define GV_UNROLL 4
+#endif
+#ifndef GV_MINB_FLOAT
+#define GV_MINB_FLOAT 2
+#endif
+constexpr int kWarps = kThreads / 32;
+constexpr int kRing = 8;                  // asynchronous copies in flight per lane (power of two)
+constexpr int kWarpTile = 512;            // bytes of one warp-tile
+
 struct DenseSmem {
-    static constexpr int TILE = kThreads * 16 * V;
-    static constexpr size_t kSlots = 2 * TILE;
-    static constexpr size_t kAcc = kSlots + sizeof(uint4) * kChunk * kThreads;
-    static constexpr size_t kBar = kAcc + sizeof(CtaAcc) * kChunk;
-    static constexpr size_t kRefHash = kBar + 2 * sizeof(uint64_t);
-    static constexpr size_t kTotal = kRefHash + sizeof(unsigned long long);
+    static constexpr size_t kRingOff = 0;                                                 // [warp][kRing][32] uint4
+    static constexpr size_t kRefOff = kRingOff + size_t(kWarps) * kRing * kWarpTile;      // [warp][2][32] uint4
+    static constexpr size_t kSlotOff = kRefOff + size_t(kWarps) * 2 * kWarpTile;          // [warp][kChunk][32] u64
+    static constexpr size_t kAccOff = kSlotOff + size_t(kWarps) * kChunk * 32 * 8;        // CtaAcc[kChunk]
+    static constexpr size_t kBarOff = kAccOff + sizeof(CtaAcc) * kChunk;                  // [warp][2] mbarrier
+    static constexpr size_t kRefHashOff = kBarOff + size_t(kWarps) * 2 * 8;
+    static constexpr size_t kTotal = kRefHashOff + 8;
 };
 
-template <int DT, int V>
-__global__ void __launch_bounds__(kThreads) dense_kernel(const __grid_constant__ DenseParams p) {
+// The exact rule for one vector the fast path could not settle; kept out of line so the hot loop
+// stays small. Everything it finds goes straight to the CTA accumulators.
+template <int DT>
+__device__ __noinline__ void settle_vector_exact(uint4 c, RefVec<16 / Traits<DT>::ESZ> r, uint64_t elem0,
+                                                 TolF t, CtaAcc* s) {
+    Acc a;
+    a.clear();
+    const uint32_t thr = *reinterpret_cast<volatile unsigned int*>(&s->thr);
+    vec_exact_float<DT>(c, r, elem0, t, thr, a);
+    push_rare(s, a);
+    if (a.cnt) atomicAdd(&s->cnt, static_cast<unsigned long long>(a.cnt));
+    raise_maxabs(s, a.maxabs);
+}
+template <int DT>
+__device__ __noinline__ void settle_vector_int(uint4 c, uint4 r, uint64_t elem0, CtaAcc* s) {
+    Acc a;
+    a.clear();
+    vec_int<DT>(c, r, elem0, 16 / Traits<DT>::ESZ, a);
+    push_rare(s, a);
+    if (a.cnt) atomicAdd(&s->cnt, static_cast<unsigned long long>(a.cnt));
+}
+
+// A 16-bit float vector the packed filter could not settle: the binary32 fast path decides, and the
+// exact rule takes over where that one cannot either. Out of line; refreshes the packed thresholds.
+template <int DT>
+__device__ __noinline__ void resolve_vector_f32(uint4 c, uint4 r, uint64_t elem0, TolF t, CtaAcc* s) {
+    RefVec<8> rv;
+    uint32_t force;
+    GV_COUNT(0);
+    hoist_ref<DT>(r, t, rv, force);
+    if (!vec_fast_float<DT>(c, rv, s)) { GV_COUNT(1); settle_vector_exact<DT>(c, rv, elem0, t, s); }
+    refresh_packed_thresholds<DT>(s);
+}
+
+// BIGK: word indices of the hash need more than 32 bits (tensors of 32 GiB and more).
+template <int DT, bool BIGK>
+__global__ void __launch_bounds__(kThreads, Traits<DT>::IS_FLOAT ? GV_MINB_FLOAT : 3) dense_kernel(const __grid_constant__ DenseParams p) {
     constexpr int ESZ = Traits<DT>::ESZ;
     constexpr int EPV = 16 / ESZ;
-    constexpr int TILE = DenseSmem<V>::TILE;
+    constexpr bool IS_FLOAT = Traits<DT>::IS_FLOAT;
+    constexpr bool PACKED = (DT == GV_BF16 || DT == GV_F16);     // 16-bit floats: packed filter first
     extern __shared__ __align__(128) unsigned char smem[];
-    unsigned char* ref_buf = smem;
-    uint4* slots = reinterpret_cast<uint4*>(smem + DenseSmem<V>::kSlots);
-    CtaAcc* cacc = reinterpret_cast<CtaAcc*>(smem + DenseSmem<V>::kAcc);
-    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + DenseSmem<V>::kBar);
-    unsigned long long* s_refhash = reinterpret_cast<unsigned long long*>(smem + DenseSmem<V>::kRefHash);
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    CtaAcc* cacc = reinterpret_cast<CtaAcc*>(smem + DenseSmem::kAccOff);
+    unsigned long long* s_refhash = reinterpret_cast<unsigned long long*>(smem + DenseSmem::kRefHashOff);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + DenseSmem::kBarOff) + warp * 2;
+    unsigned char* ref_stage = smem + DenseSmem::kRefOff + size_t(warp) * 2 * kWarpTile;
+    uint2* slots = reinterpret_cast<uint2*>(smem + DenseSmem::kSlotOff) + size_t(warp) * kChunk * 32 + lane;
+    const uint32_t ring_base = smem_u32(smem + DenseSmem::kRingOff) + (warp * kRing * 32 + lane) * 16;
 
-    const int tid = threadIdx.x;
     const uint64_t nbytes = p.n * ESZ;
-    const uint64_t num_tiles = (nbytes + TILE - 1) / TILE;
-    const uint64_t my_tiles = blockIdx.x < num_tiles ? (num_tiles - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
+    const uint64_t full_tiles = p.all_aligned ? nbytes / kWarpTile : 0;      // tiles the fast loop takes
+    const uint64_t all_tiles = (nbytes + kWarpTile - 1) / kWarpTile;
+    const uint64_t gw = static_cast<uint64_t>(blockIdx.x) * kWarps + warp;   // this warp in the grid
+    const uint64_t GW = static_cast<uint64_t>(gridDim.x) * kWarps;
     const int num_groups = (p.N + kChunk - 1) / kChunk;
-    const uint64_t num_items = my_tiles * num_groups;
-    const bool ref_aligned = (reinterpret_cast<uintptr_t>(p.ref) & 15u) == 0;
     const TolF tol = {p.atol, p.rtol, p.equal_nan};
 
-    if (tid == 0) {
+    if (lane == 0) {
         mbar_init(&bars[0], 1);
         mbar_init(&bars[1], 1);
         mbar_fence_init();
-        *s_refhash = 0;
+    }
+    if (tid == 0) *s_refhash = 0;
+    if (tid < kChunk) {
+        cacc[tid].clear();
+        if (tid < p.N) cacc[tid].rec = &p.results[tid];
     }
     __syncthreads();
-    if (num_items == 0) return;
 
-    // item s of this CTA = (group s / my_tiles, tile blockIdx.x + (s % my_tiles) * gridDim.x)
-    auto tile_of = [&](uint64_t s) { return blockIdx.x + (s % my_tiles) * static_cast<uint64_t>(gridDim.x); };
-    auto tile_bytes = [&](uint64_t t) {
-        const uint64_t rem = nbytes - t * TILE;
-        return static_cast<uint32_t>(rem < TILE ? rem : TILE);
-    };
-    // a tile can be fetched by the bulk copy when source and size are multiples of 16 bytes
-    auto tma_ok = [&](uint64_t t) { return ref_aligned && (tile_bytes(t) & 15u) == 0; };
-    auto issue = [&](uint64_t s) {          // called by thread 0 only
-        const uint64_t t = tile_of(s);
-        if (tma_ok(t)) {
-            const uint32_t bytes = tile_bytes(t);
-            fence_proxy_async();
-            mbar_expect_tx(&bars[s & 1], bytes);
-            bulk_load(ref_buf + (s & 1) * TILE, p.ref + t * TILE, bytes, &bars[s & 1]);
-        }
-    };
-
-    if (tid == 0) issue(0);
     uint32_t phase[2] = {0u, 0u};
     uint64_t my_ref_hash = 0;
-    int aborted_buf = -1;      // >= 0: a wait expired on this buffer's barrier
+    bool timed_out = false;
+    HashConsts hc;
+    hc.init();
 
-    for (uint64_t s = 0; s < num_items; ++s) {
-        const int g = static_cast<int>(s / my_tiles);
+    for (int g = 0; g < num_groups; ++g) {
         const int kg = min(kChunk, p.N - g * kChunk);
-        const uint64_t t = tile_of(s);
-        const uint32_t tb = tile_bytes(t);
-        const int b = static_cast<int>(s & 1);
-        unsigned char* rbuf = ref_buf + b * TILE;
+        const unsigned char* const* cand = &p.cands[g * kChunk];
+        for (int k = 0; k < kg; ++k) slots[k * 32] = make_uint2(0u, 0u);
 
-        if (s % my_tiles == 0) {
-            // new chunk of candidates: start its accumulators from the identities
-            for (int k = 0; k < kg; ++k) slots[k * kThreads + tid] = make_uint4(0u, 0u, 0u, 0u);
-            if (tid < kChunk) cacc[tid].clear();
-            // (made visible by the barrier below, before any rare-path atomic can touch them)
-        }
+        // ================= fast loop: full warp-tiles, every base 16-byte aligned =================
+        if (gw < full_tiles && !timed_out) {
+            const uint32_t my_tiles = static_cast<uint32_t>(min((full_tiles - gw + GW - 1) / GW, uint64_t(0xFFFFFFFFu)));
+            const uint64_t tile_stride = GW * kWarpTile;
+            uint64_t voff = gw * kWarpTile + lane * 16;          // this lane's vector in the tensor (current tile)
 
-        // ---- reference tile: wait for the bulk copy, or fetch it with ordinary loads ----
-        bool ok = true;
-        if (tma_ok(t)) {
-            ok = mbar_wait_bounded(&bars[b], phase[b]);
-            if (ok) phase[b] ^= 1u;
-        } else {
-            // ragged tail / unaligned reference: element-sized loads, zero fill to the tile end
-            for (uint32_t o = tid * ESZ; o < static_cast<uint32_t>(TILE); o += kThreads * ESZ) {
-                if (ESZ == 2) {
-                    *reinterpret_cast<unsigned short*>(rbuf + o) =
-                        o < tb ? *reinterpret_cast<const unsigned short*>(p.ref + t * TILE + o) : static_cast<unsigned short>(0);
-                } else if (ESZ == 4) {
-                    *reinterpret_cast<uint32_t*>(rbuf + o) =
-                        o < tb ? *reinterpret_cast<const uint32_t*>(p.ref + t * TILE + o) : 0u;
+            // Values derived from the reference vector, computed lazily: only when a candidate
+            // vector differs from it (exact copies never pay for them).
+            RefVec<(IS_FLOAT && !PACKED) ? EPV : 1> rv;
+            PackedRef pr;
+            uint32_t force = 0u;
+            bool hoisted = false;
+            // maxima other CTAs have published for the chunk's candidates, fetched one tile ahead
+            uint32_t seen_abs = 0u, seen_rel = 0u;
+            auto new_tile = [&](const uint4& r) {
+                hoisted = false;
+                force = 0u;
+                if constexpr (IS_FLOAT) {
+                    if (lane < kg) {
+                        CtaAcc* s = &cacc[lane];
+                        if (seen_abs > *reinterpret_cast<volatile unsigned int*>(&s->maxabs)) atomicMax(&s->maxabs, seen_abs);
+                        if (seen_rel > *reinterpret_cast<volatile unsigned int*>(&s->maxrel)) {
+                            atomicMax(&s->maxrel, seen_rel);
+                            atomicMax(&s->thr, rel_threshold_bits(seen_rel));
+                        }
+                        if constexpr (PACKED) refresh_packed_thresholds<DT>(s);
+                        const gv_result* rec = &p.results[g * kChunk + lane];
+                        asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(seen_abs) : "l"(&rec->max_abs_err));
+                        asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(seen_rel) : "l"(&rec->max_rel_err));
+                    }
+                }
+                if constexpr (IS_FLOAT) {
+                    // only a NaN in the reference (without equal_nan) forces identical vectors onto the
+                    // compare path; that needs no arithmetic, just the exponent/mantissa test
+                    if (!tol.equal_nan) {
+                        bool any_nan = false;
+                        if constexpr (DT == GV_F32) {
+                            any_nan = is_nan_bits(r.x) || is_nan_bits(r.y) || is_nan_bits(r.z) || is_nan_bits(r.w);
+                        } else {
+                            const uint32_t w[4] = {r.x, r.y, r.z, r.w};
+                            constexpr uint32_t kAbs = 0x7FFF7FFFu;
+                            constexpr uint32_t kInf = (DT == GV_BF16) ? 0x7F80u : 0x7C00u;
+#pragma unroll
+                            for (int j = 0; j < 4; ++j) {
+                                const uint32_t a = w[j] & kAbs;
+                                any_nan = any_nan || (a & 0xFFFFu) > kInf || (a >> 16) > kInf;
+                            }
+                        }
+                        force = any_nan ? 0xFFFFFFFFu : 0u;
+                    }
+                }
+            };
+            // Derive the per-tile values when some lane of the warp first needs them. The decision is
+            // warp-uniform (a vote), so the derivation runs once per tile, not once per diverged lane.
+            auto ensure_hoisted = [&](const uint4& r) {
+                if (!hoisted) {
+                    uint32_t f2;
+                    if constexpr (PACKED) hoist_packed<DT>(r, tol, pr, f2);
+                    else if constexpr (IS_FLOAT) hoist_ref<DT>(r, tol, rv, f2);
+                    hoisted = true;
+                }
+            };
+            // a candidate vector that is not bit-identical to the reference vector (ensure_hoisted done)
+            auto differing = [&](const uint4& c, const uint4& r, int k) {
+                if constexpr (!IS_FLOAT) {
+                    settle_vector_int<DT>(c, r, voff / ESZ, &cacc[k]);
+                } else if constexpr (PACKED) {
+                    const uint32_t mh2 = *reinterpret_cast<volatile unsigned int*>(&cacc[k].mh2);
+                    const uint32_t thr2 = *reinterpret_cast<volatile unsigned int*>(&cacc[k].thr2);
+                    if (packed_filter<DT>(c, r, pr, mh2, thr2) != 0u)
+                        resolve_vector_f32<DT>(c, r, voff / ESZ, tol, &cacc[k]);
                 } else {
-                    *reinterpret_cast<unsigned long long*>(rbuf + o) =
-                        o < tb ? *reinterpret_cast<const unsigned long long*>(p.ref + t * TILE + o) : 0ull;
+                    if (!vec_fast_float<DT>(c, rv, &cacc[k])) settle_vector_exact<DT>(c, rv, voff / ESZ, tol, &cacc[k]);
+                }
+            };
+            // one visit: candidate vector c (already read from the ring) against the held reference
+            auto visit = [&](const uint4& c, const uint4& r, int k) {
+                uint64_t h;
+                if constexpr (BIGK) h = hash_vec_full(c, voff / 8);
+                else h = hash_vec_full_k32(c, static_cast<uint32_t>(voff / 8), hc);
+                const uint2 sl = slots[k * 32];
+                h += pack64(sl.x, sl.y);
+                slots[k * 32] = make_uint2(static_cast<uint32_t>(h), static_cast<uint32_t>(h >> 32));
+                const bool differs = (c.x != r.x) || (c.y != r.y) || (c.z != r.z) || (c.w != r.w) || (force != 0u);
+                if (__any_sync(0xFFFFFFFFu, differs)) {
+                    ensure_hoisted(r);
+                    if (differs) differing(c, r, k);
+                }
+            };
+            // reference of tile i: wait for its bulk copy, take this lane's vector, start the next copy
+            auto next_ref = [&](uint32_t i, uint4& r) -> bool {
+                const int b = static_cast<int>(i & 1u);
+                bool ok = mbar_wait_bounded(&bars[b], phase[b]);
+                ok = __all_sync(0xFFFFFFFFu, ok);
+                if (!ok) return false;
+                phase[b] ^= 1u;
+                r = *reinterpret_cast<const uint4*>(ref_stage + b * kWarpTile + lane * 16);
+                __syncwarp();      // every lane has read buffer b; buffer b^1 was drained one tile ago
+                if (lane == 0 && i + 1 < my_tiles) {
+                    fence_proxy_async();
+                    mbar_expect_tx(&bars[b ^ 1], kWarpTile);
+                    bulk_load(ref_stage + (b ^ 1) * kWarpTile, p.ref + (voff - lane * 16) + tile_stride, kWarpTile,
+                              &bars[b ^ 1]);
+                }
+                return true;
+            };
+            if (lane == 0) {
+                fence_proxy_async();
+                mbar_expect_tx(&bars[0], kWarpTile);
+                bulk_load(ref_stage, p.ref + gw * kWarpTile, kWarpTile, &bars[0]);
+            }
+
+            if (kg == kChunk) {
+                // ---- full chunk: ring depth 8 = half a chunk. While candidate k of a tile is consumed
+                // from stage k & 7, that stage is refilled with candidate k + 8 of the same tile
+                // (k < 8) or candidate k - 8 of the next tile (k >= 8).
+                constexpr int U = GV_UNROLL;               // visits per unrolled block (divides kRing)
+#pragma unroll 1
+                for (int k = 0; k < kRing; ++k) {
+                    cp_async16(ring_base + k * 512u, cand[k] + voff);
+                    if ((k % U) == U - 1) cp_async_commit();
+                }
+#pragma unroll 1
+                for (uint32_t i = 0; i < my_tiles; ++i) {
+                    uint4 r;
+                    if (!next_ref(i, r)) { timed_out = true; break; }
+                    if (g == 0 && p.ref_hash) my_ref_hash += hash_vec_full(r, voff / 8);
+                    new_tile(r);
+                    const bool has_next = i + 1 < my_tiles;
+#pragma unroll 1
+                    for (int k0 = 0; k0 < kChunk; k0 += U) {
+                        const uint32_t stage0 = ring_base + (k0 & (kRing - 1)) * 512u;
+                        const unsigned char* const* refill = cand + ((k0 + kRing) & (kChunk - 1));
+                        const uint64_t refill_off = k0 < kRing ? voff : voff + tile_stride;
+                        const bool live = k0 < kRing || has_next;
+                        cp_async_wait<kRing / U - 1>();     // the block of U stages issued kRing visits ago has landed
+                        uint4 c[U];
+#pragma unroll
+                        for (int u = 0; u < U; ++u) c[u] = lds128(stage0 + u * 512u);
+                        // straight-line part for all U visits: hash, slot update, identity test
+                        uint32_t diffmask = 0u;
+#pragma unroll
+                        for (int u = 0; u < U; ++u) {
+                            uint64_t h;
+                            if constexpr (BIGK) h = hash_vec_full(c[u], voff / 8);
+                            else h = hash_vec_full_k32(c[u], static_cast<uint32_t>(voff / 8), hc);
+                            const uint2 sl = slots[(k0 + u) * 32];
+                            h += pack64(sl.x, sl.y);
+                            slots[(k0 + u) * 32] = make_uint2(static_cast<uint32_t>(h), static_cast<uint32_t>(h >> 32));
+                            const bool differs = (c[u].x != r.x) || (c[u].y != r.y) || (c[u].z != r.z) || (c[u].w != r.w);
+                            diffmask |= differs ? (1u << u) : 0u;
+                        }
+                        diffmask |= force;      // force is 0 or all ones
+                        if (__any_sync(0xFFFFFFFFu, diffmask != 0u)) {
+                            ensure_hoisted(r);
+#pragma unroll
+                            for (int u = 0; u < U; ++u) {
+                                if (diffmask & (1u << u)) differing(c[u], r, k0 + u);
+                            }
+                        }
+#pragma unroll
+                        for (int u = 0; u < U; ++u) {
+                            if (live) cp_async16(stage0 + u * 512u, refill[u] + refill_off);
+                        }
+                        cp_async_commit();                  // one group per block of U refills
+                    }
+                    voff += tile_stride;
+                }
+            } else {
+                // ---- partial chunk (fewer than 16 candidates): same ring, generic bookkeeping
+                const uint64_t visits = static_cast<uint64_t>(my_tiles) * kg;
+                uint64_t issue_off = voff;
+                int issue_k = 0;
+                uint64_t issued = 0;
+                auto issue_one = [&]() {
+                    if (issued < visits) {
+                        cp_async16(ring_base + (static_cast<uint32_t>(issued) & (kRing - 1)) * 512u, cand[issue_k] + issue_off);
+                        ++issued;
+                        if (++issue_k == kg) { issue_k = 0; issue_off += tile_stride; }
+                    }
+                    cp_async_commit();          // one group per visit, possibly empty near the end
+                };
+#pragma unroll 1
+                for (int j = 0; j < kRing; ++j) issue_one();
+                uint32_t stage = 0;
+#pragma unroll 1
+                for (uint32_t i = 0; i < my_tiles; ++i) {
+                    uint4 r;
+                    if (!next_ref(i, r)) { timed_out = true; break; }
+                    if (g == 0 && p.ref_hash) my_ref_hash += hash_vec_full(r, voff / 8);
+                    new_tile(r);
+#pragma unroll 1
+                    for (int k = 0; k < kg; ++k) {
+                        cp_async_wait<kRing - 1>();
+                        const uint4 c = lds128(ring_base + stage * 512u);
+                        stage = (stage + 1) & (kRing - 1);
+                        issue_one();
+                        visit(c, r, k);
+                    }
+                    voff += tile_stride;
                 }
             }
-            __syncthreads();
-        }
-        uint4 r[V];
-        if (ok) {
-#pragma unroll
-            for (int v = 0; v < V; ++v) r[v] = *reinterpret_cast<const uint4*>(rbuf + (v * kThreads + tid) * 16);
-        }
-        ok = __syncthreads_and(ok ? 1 : 0) != 0;       // also: everyone has read its slice of rbuf
-        if (!ok) { aborted_buf = b; break; }
-        if (tid == 0 && s + 1 < num_items) issue(s + 1);   // next tile lands in the other buffer meanwhile
-
-        // per-vector geometry of this thread
-        uint64_t voff[V];      // byte offset of the vector in the tensor
-        int nvalid[V];         // elements of the vector that exist
-        bool full[V];
-#pragma unroll
-        for (int v = 0; v < V; ++v) {
-            voff[v] = t * TILE + static_cast<uint64_t>(v * kThreads + tid) * 16;
-            const uint64_t rem = voff[v] < nbytes ? nbytes - voff[v] : 0;
-            nvalid[v] = rem >= 16 ? EPV : static_cast<int>(rem / ESZ);
-            full[v] = rem >= 16;
-        }
-
-        if (g == 0 && p.ref_hash) {
-#pragma unroll
-            for (int v = 0; v < V; ++v) {
-                if (nvalid[v] > 0) my_ref_hash += hash_vec(r[v], voff[v] / 8, nvalid[v] * ESZ > 8 ? 2 : 1);
+            cp_async_wait<0>();
+            if (timed_out) {
+                // flag it; give the copy that may still be in flight a second bounded chance to land
+                if (lane == 0) {
+                    atomicOr(p.status, kStatusTimeout);
+                    (void)mbar_wait_bounded(&bars[0], phase[0]);
+                    (void)mbar_wait_bounded(&bars[1], phase[1]);
+                }
+                __syncwarp();
             }
         }
 
-        // ---- stream the candidates of the chunk ----
-        auto fetch = [&](int k, uint4 (&dst)[V]) {
-            const unsigned char* cp = p.cands[g * kChunk + k];
-            const bool cal = (reinterpret_cast<uintptr_t>(cp) & 15u) == 0;
-#pragma unroll
-            for (int v = 0; v < V; ++v) {
-                if (cal && full[v]) dst[v] = ldg_stream(cp + voff[v]);
-                else if (nvalid[v] > 0) dst[v] = load_vec_generic<ESZ>(cp, voff[v], nbytes);
-                else dst[v] = make_uint4(0u, 0u, 0u, 0u);
-            }
-        };
-        constexpr int PF = (V == 1) ? 4 : 2;        // candidates fetched ahead
-        uint4 pre[PF][V];
-#pragma unroll
-        for (int q = 0; q < PF; ++q) {
-            if (q < kg) fetch(q, pre[q]);
-        }
-        for (int k0 = 0; k0 < kg; k0 += PF) {
-#pragma unroll
-            for (int q = 0; q < PF; ++q) {
-                const int k = k0 + q;
-                if (k < kg) {
-                    uint4 cur[V];
-#pragma unroll
-                    for (int v = 0; v < V; ++v) cur[v] = pre[q][v];
-                    if (k + PF < kg) fetch(k + PF, pre[q]);
+        // ================= general loop: ragged tail, or some base not 16-byte aligned =================
+        // (synchronous element-sized loads; at most one warp-tile per tensor when bases are aligned)
+        for (uint64_t t = full_tiles + gw; t < all_tiles; t += GW) {
+            const uint64_t voff = t * kWarpTile + lane * 16;
+            const uint64_t rem = voff < nbytes ? nbytes - voff : 0;
+            const int nvalid = rem >= 16 ? EPV : static_cast<int>(rem / ESZ);
+            if (nvalid > 0) {
+                const uint4 r = load_vec_generic<ESZ>(p.ref, voff, nbytes);
+                const int nwords = nvalid * ESZ > 8 ? 2 : 1;
+                if (g == 0 && p.ref_hash) my_ref_hash += hash_vec(r, voff / 8, nwords);
+                for (int k = 0; k < kg; ++k) {
+                    const uint4 c = load_vec_generic<ESZ>(cand[k], voff, nbytes);
                     Acc a;
                     a.clear();
-#pragma unroll
-                    for (int v = 0; v < V; ++v) {
-                        if (nvalid[v] > 0) {
-                            a.hash += full[v] ? hash_vec_full(cur[v], voff[v] / 8)
-                                              : hash_vec(cur[v], voff[v] / 8, nvalid[v] * ESZ > 8 ? 2 : 1);
-                            vec_compare<DT>(cur[v], r[v], voff[v] / ESZ, nvalid[v], tol, a);
-                        }
-                    }
-                    uint4 sl = slots[k * kThreads + tid];
+                    a.hash = hash_vec(c, voff / 8, nwords);
+                    vec_compare<DT>(c, r, voff / ESZ, nvalid, tol, a);
+                    const uint2 sl = slots[k * 32];
                     const uint64_t h = pack64(sl.x, sl.y) + a.hash;
-                    sl.x = static_cast<uint32_t>(h);
-                    sl.y = static_cast<uint32_t>(h >> 32);
-                    sl.z += a.cnt;
-                    sl.w = a.maxabs > sl.w ? a.maxabs : sl.w;
-                    slots[k * kThreads + tid] = sl;
+                    slots[k * 32] = make_uint2(static_cast<uint32_t>(h), static_cast<uint32_t>(h >> 32));
                     push_rare(&cacc[k], a);
+                    if (a.cnt) atomicAdd(&cacc[k].cnt, static_cast<unsigned long long>(a.cnt));
+                    raise_maxabs(&cacc[k], a.maxabs);
                 }
             }
         }
 
-        // ---- end of a chunk: reduce the slots once and publish ----
-        if ((s + 1) % my_tiles == 0) {
-            for (int k = 0; k < kg; ++k) {
-                const uint4 sl = slots[k * kThreads + tid];
-                const uint64_t h = warp_sum_u64(pack64(sl.x, sl.y));
-                const uint64_t c = warp_sum_u64(static_cast<uint64_t>(sl.z));
-                const uint32_t m = __reduce_max_sync(0xFFFFFFFFu, sl.w);
-                if ((tid & 31) == 0) {
-                    if (h) atomicAdd(&cacc[k].hash, static_cast<unsigned long long>(h));
-                    if (c) atomicAdd(&cacc[k].cnt, static_cast<unsigned long long>(c));
-                    if (m) atomicMax(&cacc[k].maxabs, m);
-                }
-            }
-            __syncthreads();
-            if (tid < kg) push_global(&p.results[g * kChunk + tid], cacc[tid]);
-            __syncthreads();        // records pushed before the next chunk clears the accumulators
-        }
-    }
-
-    if (aborted_buf >= 0) {
-        // flag the timeout, give the one copy still in flight a second bounded chance to land
-        // (its destination is this CTA's shared memory), then leave
-        if (tid == 0) {
-            atomicOr(p.status, kStatusTimeout);
-            (void)mbar_wait_bounded(&bars[aborted_buf], phase[aborted_buf]);
+        // ---- end of a chunk: reduce the hash slots once and publish the chunk's records ----
+        for (int k = 0; k < kg; ++k) {
+            const uint2 sl = slots[k * 32];
+            const uint64_t h = warp_sum_u64(pack64(sl.x, sl.y));
+            if (lane == 0 && h) atomicAdd(&cacc[k].hash, static_cast<unsigned long long>(h));
         }
         __syncthreads();
-        return;
+        if (tid < kg) push_global(&p.results[g * kChunk + tid], cacc[tid]);
+        if (tid < kChunk) {
+            cacc[tid].clear();
+            const int next = (g + 1) * kChunk + tid;
+            if (next < p.N) cacc[tid].rec = &p.results[next];
+        }
+        __syncthreads();
     }
+
     if (p.ref_hash) {
         const uint64_t h = warp_sum_u64(my_ref_hash);
-        if ((tid & 31) == 0 && h) atomicAdd(s_refhash, static_cast<unsigned long long>(h));
+        if (lane == 0 && h) atomicAdd(s_refhash, static_cast<unsigned long long>(h));
         __syncthreads();
         if (tid == 0 && *s_refhash) atomicAdd(p.ref_hash, *s_refhash);
     }
@@ -566,13 +730,13 @@ bool tol_valid(const gv_tol* t) {
     return t && isfinite(t->atol) && isfinite(t->rtol) && t->atol >= 0.0 && t->rtol >= 0.0;
 }
 
-template <int DT, int V>
+template <int DT, bool BIGK>
 gv_status launch_dense_t(const gv::DenseParams& p, int sm_count, cudaStream_t st) {
-    using S = gv::DenseSmem<V>;
+    using S = gv::DenseSmem;
     static int blocks_per_sm[64] = {0};
     int dev = 0;
     GV_CUDA(cudaGetDevice(&dev));
-    auto kern = gv::dense_kernel<DT, V>;
+    auto kern = gv::dense_kernel<DT, BIGK>;
     if (blocks_per_sm[dev] == 0) {
         GV_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(S::kTotal)));
         int b = 0;
@@ -580,7 +744,8 @@ gv_status launch_dense_t(const gv::DenseParams& p, int sm_count, cudaStream_t st
         blocks_per_sm[dev] = b > 0 ? b : 1;
     }
     const uint64_t nbytes = p.n * gv::Traits<DT>::ESZ;
-    const uint64_t tiles = (nbytes + S::TILE - 1) / S::TILE;
+    const uint64_t cta_tile = static_cast<uint64_t>(gv::kWarps) * gv::kWarpTile;
+    const uint64_t tiles = (nbytes + cta_tile - 1) / cta_tile;
     uint64_t grid = static_cast<uint64_t>(sm_count) * blocks_per_sm[dev];
     if (grid > tiles) grid = tiles;
     if (grid == 0) return GV_OK;
@@ -590,17 +755,25 @@ gv_status launch_dense_t(const gv::DenseParams& p, int sm_count, cudaStream_t st
 }
 
 gv_status launch_dense(gv_dtype dt, const gv::DenseParams& p, int sm_count, cudaStream_t st) {
+    const bool bigk = p.n * static_cast<uint64_t>(gv::elem_size(dt)) >= (1ull << 35);
     switch (dt) {
-        case GV_F32: return launch_dense_t<GV_F32, 2>(p, sm_count, st);
-        case GV_BF16: return launch_dense_t<GV_BF16, 1>(p, sm_count, st);
-        case GV_F16: return launch_dense_t<GV_F16, 1>(p, sm_count, st);
-        case GV_I32: return launch_dense_t<GV_I32, 2>(p, sm_count, st);
-        case GV_I64: return launch_dense_t<GV_I64, 2>(p, sm_count, st);
+        case GV_F32: return bigk ? launch_dense_t<GV_F32, true>(p, sm_count, st) : launch_dense_t<GV_F32, false>(p, sm_count, st);
+        case GV_BF16: return bigk ? launch_dense_t<GV_BF16, true>(p, sm_count, st) : launch_dense_t<GV_BF16, false>(p, sm_count, st);
+        case GV_F16: return bigk ? launch_dense_t<GV_F16, true>(p, sm_count, st) : launch_dense_t<GV_F16, false>(p, sm_count, st);
+        case GV_I32: return bigk ? launch_dense_t<GV_I32, true>(p, sm_count, st) : launch_dense_t<GV_I32, false>(p, sm_count, st);
+        case GV_I64: return bigk ? launch_dense_t<GV_I64, true>(p, sm_count, st) : launch_dense_t<GV_I64, false>(p, sm_count, st);
     }
     return GV_ERR_UNSUPPORTED;
 }
 
 }  // namespace
+
+#ifdef GV_DEBUG_COUNTERS
+extern "C" void gv_debug_counters(unsigned long long* out, int reset) {
+    cudaMemcpyFromSymbol(out, gv::g_dbg, sizeof(unsigned long long) * 8);
+    if (reset) { unsigned long long z[8] = {0}; cudaMemcpyToSymbol(gv::g_dbg, z, sizeof(z)); }
+}
+#endif
 
 extern "C" {
 
@@ -663,8 +836,12 @@ gv_status gv_verify_batch(const void* ref, const void* const* cands, int32_t N, 
         p.rtol = is_float ? static_cast<float>(tol->rtol) : 0.0f;
         p.equal_nan = is_float ? (tol->equal_nan != 0) : 0;
         p.N = (N - j0) < gv::kMaxPtrs ? (N - j0) : gv::kMaxPtrs;
-        for (int k = 0; k < gv::kMaxPtrs; ++k)
+        uintptr_t all_bits = reinterpret_cast<uintptr_t>(ref);
+        for (int k = 0; k < gv::kMaxPtrs; ++k) {
             p.cands[k] = k < p.N ? static_cast<const unsigned char*>(cands[j0 + k]) : nullptr;
+            all_bits |= reinterpret_cast<uintptr_t>(p.cands[k]);
+        }
+        p.all_aligned = (all_bits & 15u) == 0;
         rc = launch_dense(dt, p, sm_count, st);
         if (rc != GV_OK) return rc;
     }

@@ -7,6 +7,7 @@
 #pragma once
 
 #include <cuda_runtime.h>
+#include <stddef.h>
 #include <stdint.h>
 
 #include "gv.h"
@@ -32,6 +33,10 @@ template <> struct Traits<GV_I64>  { static constexpr int ESZ = 8; static conste
 
 __host__ __device__ inline int elem_size(int dt) {
     return dt == GV_F32 ? 4 : dt == GV_BF16 ? 2 : dt == GV_F16 ? 2 : dt == GV_I32 ? 4 : dt == GV_I64 ? 8 : 0;
+}
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+    return static_cast<uint32_t>(__cvta_generic_to_shared(p));
 }
 
 // ------------------------------------------------------------------------------------------
@@ -265,20 +270,16 @@ struct Acc {
 
 // Per-candidate accumulators of one CTA (shared memory). Rare quantities are updated with
 // shared-memory atomics from the compare path; the common ones once per flush.
-struct CtaAcc {
+// (16-byte aligned: {maxabs, maxrel, thr, pad} is read with one 128-bit shared load)
+struct __align__(16) CtaAcc {
     unsigned long long hash, cnt, first, nan, inf, maxint;
     unsigned int maxabs, maxrel;
     unsigned int thr;      // relative-error filter threshold derived from maxrel (see rel_threshold_bits)
     unsigned int pad;
-    // thresholds of the packed 16-bit filters, both halves equal (see PackedFilter): mh2 from maxabs, thr2 from maxrel
-    unsigned int mh2, thr2;
-    // The candidate's record in global memory. Raised maxima are also sent there at once (max is
-    // idempotent, the record is their destination anyway) so that other CTAs can pick them up and
-    // tighten their own filters long before the chunk ends.
-    gv_result* rec;
+    unsigned int pad2[2];
     __device__ __forceinline__ void clear() {
         hash = 0; cnt = 0; first = ~0ull; nan = 0; inf = 0; maxint = 0; maxabs = 0; maxrel = 0; thr = 0; pad = 0;
-        mh2 = 0; thr2 = 0; rec = nullptr;
+        pad2[0] = 0; pad2[1] = 0;
     }
 };
 
@@ -408,18 +409,18 @@ __device__ __forceinline__ uint32_t rel_threshold_bits(uint32_t m_bits) {
     return __float_as_uint(__fmul_rd(__uint_as_float(m_bits), __uint_as_float(0x3F7FFFF0u)));   // 1 - 2^-20
 }
 
-// Raise the CTA's running maxima (bit patterns of non-negative floats) and forward them to the record.
+// Raise the CTA's running maxima (bit patterns of non-negative floats).
 __device__ __forceinline__ void raise_maxabs(CtaAcc* s, uint32_t bits) {
     if (bits > *reinterpret_cast<volatile unsigned int*>(&s->maxabs)) {
         atomicMax(&s->maxabs, bits);
-        if (s->rec) atomicMax(reinterpret_cast<unsigned int*>(&s->rec->max_abs_err), bits);
+
     }
 }
 __device__ __forceinline__ void raise_maxrel(CtaAcc* s, uint32_t bits) {
     if (bits > *reinterpret_cast<volatile unsigned int*>(&s->maxrel)) {
         atomicMax(&s->maxrel, bits);
         atomicMax(&s->thr, rel_threshold_bits(bits));
-        if (s->rec) atomicMax(reinterpret_cast<unsigned int*>(&s->rec->max_rel_err), bits);
+
     }
 }
 
@@ -429,13 +430,15 @@ __device__ __noinline__ uint32_t exact_quotient_bits(float ad, float abs_r) {
     return __float_as_uint(__fdiv_rn(ad, abs_r));
 }
 
-// Compare one full vector on the fast path. Returns true when the vector is settled: every element
-// is close with finite |d| (so every pair is a finite pair). Then max |d| and, for the elements whose
-// estimate passes the filter, the exact relative error are merged into the CTA accumulators here.
-// Returns false when the caller must run the exact per-element rule on this vector (nothing has
-// been recorded in that case).
+// Compare one full vector on the fast path. Returns true when the vector is settled here: every pair
+// is a finite pair (both values finite, |d| finite). Close elements only feed the maxima; elements
+// that are not close are counted (a finite pair is close exactly when |d| <= tolc) and the first
+// index is merged. Max |d| and, for the elements whose estimate passes the filter, the exact relative
+// error go to the CTA accumulators. Returns false when a NaN or an infinity is involved: the caller
+// then runs the exact per-element rule on this vector (nothing has been recorded in that case).
 template <int DT>
-__device__ __forceinline__ bool vec_fast_float(const uint4& c, const RefVec<16 / Traits<DT>::ESZ>& r, CtaAcc* s) {
+__device__ __forceinline__ bool vec_fast_float(const uint4& c, const RefVec<16 / Traits<DT>::ESZ>& r, CtaAcc* s,
+                                               uint64_t elem0) {
     constexpr int EPV = 16 / Traits<DT>::ESZ;
     float cf[EPV], ad[EPV], m[EPV], q[EPV];
     Widen<DT>::run(c, cf);
@@ -455,169 +458,60 @@ __device__ __forceinline__ bool vec_fast_float(const uint4& c, const RefVec<16 /
         va = fmaxf(max3(ad[0], ad[1], ad[2]), ad[3]);
         vq = fmaxf(max3(q[0], q[1], q[2]), q[3]);
     }
-    if (!(vm <= 0.0f)) return false;                                  // some element not close, or NaN
     const uint32_t vab = __float_as_uint(va);
-    raise_maxabs(s, vab);
-    const uint32_t thr_bits = *reinterpret_cast<volatile unsigned int*>(&s->thr);
+    if (!(vm <= 0.0f)) {
+        // some element is not close, or a NaN is present (vm propagates NaN)
+        if (vm != vm || vab >= 0x7F800000u) return false;
+        uint32_t cnt = 0u;
+        int first_e = EPV;
+#pragma unroll
+        for (int e = EPV - 1; e >= 0; --e) {
+            if (m[e] > 0.0f) { cnt += 1u; first_e = e; }
+        }
+        GV_COUNT(3);
+        // lanes of the warp that are here add their counts with one shared-memory atomic
+        const unsigned active = __activemask();
+        const uint32_t total = __reduce_add_sync(active, cnt);
+        if ((threadIdx.x & 31) == __ffs(active) - 1) atomicAdd(&s->cnt, static_cast<unsigned long long>(total));
+        const unsigned long long idx = elem0 + first_e;
+        if (idx < *reinterpret_cast<volatile unsigned long long*>(&s->first)) atomicMin(&s->first, idx);
+    }
+    // running maxima of this (CTA, candidate): max|d| bits, max relative error bits, filter threshold
+    const uint4 run = lds128(smem_u32(&s->maxabs));
+    if (vab > run.x) raise_maxabs(s, vab);
+    const uint32_t thr_bits = run.z;
     if ((vq > __uint_as_float(thr_bits)) || (thr_bits == 0u && vab != 0u)) {
-        // some element may raise the relative maximum: exact quotients for those that pass the filter
+        // Some element may raise the relative maximum M. For each element that passes the filter,
+        // first decide exactly whether the real quotient |d| / |r| exceeds M without dividing:
+        // |d| > M |r|  <=>  |d| - p > e  with p = fl(M |r|) and e = M |r| - p (the exact rounding error,
+        // delivered by one fused multiply-add). Elements that only tie with M -- common in quantised
+        // data -- stop here; rounding is monotone, so a real quotient <= M cannot round above M.
         GV_COUNT(2);
+        const float M = __uint_as_float(run.y);
         uint32_t best = 0u;
 #pragma unroll
         for (int e = 0; e < EPV; ++e) {
             const bool need = (q[e] > __uint_as_float(thr_bits)) || (thr_bits == 0u && ad[e] != 0.0f);
             // r.inv == 0 marks r == 0 (no relative error); q is then 0 or NaN and ad may be nonzero
             if (need && r.inv[e] != 0.0f) {
-                const uint32_t qe = exact_quotient_bits(ad[e], fabsf(r.rf[e]));
-                best = qe > best ? qe : best;
+                const float ar = fabsf(r.rf[e]);
+                bool beats = true;
+                if (thr_bits != 0u) {
+                    const float pm = __fmul_rn(M, ar);
+                    if (__float_as_uint(pm) >= 0x0D800000u && __float_as_uint(pm) < 0x7F800000u) {   // 2^-100 <= p < Inf: e is exact
+                        const float err = __fmaf_rn(M, ar, -pm);
+                        beats = __fsub_rn(ad[e], pm) > err;
+                    }
+                }
+                if (beats) {
+                    const uint32_t qe = exact_quotient_bits(ad[e], ar);
+                    best = qe > best ? qe : best;
+                }
             }
         }
-        raise_maxrel(s, best);
+        if (best > run.y) raise_maxrel(s, best);
     }
     return true;
-}
-
-// ------------------------------------------------------------------------------------------
-// packed 16-bit filter for bf16 / fp16 vectors
-// ------------------------------------------------------------------------------------------
-// For the two 16-bit float types the common case is settled without widening, two elements per
-// instruction, in the type's own arithmetic. This is exact, not approximate, because of Sterbenz's
-// lemma: when |c - r| <= |r| / 2 the difference c - r is representable in the operands' format, so
-// the packed subtraction returns the very number the binary32 rule computes. Per element a bound
-//     b = RZ16( r == 0 ? tolc : min(tolc, 0.48 |r|) )        (tolc = min(tol, FLT_MAX), RZ16 = toward zero)
-// is derived once per reference tile. If a = |c -_16 r| <= b then (rounding error of the packed
-// subtraction at most 2^-8 relative) |c - r| < |r| / 2, hence a = |c - r| exactly, and a <= tolc: the
-// element is close and a finite pair (r == 0: c - 0 is exact anyway). What remains is whether a
-// raises the running max |d| (compare with mh = RZ16 of it: a > max  <=>  a > mh for 16-bit a) and
-// whether a / |r| can raise the running max relative error M: with inv = the smallest 16-bit number
-// >= 1 / |r| the product a * inv >= a / |r|; a rounded quotient can exceed M only if the real one does,
-// so a * inv > thr16 with thr16 <= M is a safe test, evaluated by one fused multiply-add whose sign
-// is exact while M >= kMinRel16 (below that mh is kept at 0, so every nonzero a is sent on). The three conditions are evaluated as
-// relu(a - b) + relu(a - mh) + relu(a * inv - thr16) summed over the vector; a nonzero (or NaN) sum
-// sends the vector to the binary32 path, which then decides everything by itself. Nothing is
-// recorded here, so a needless detour costs time only.
-template <int DT> struct Half2;
-template <> struct Half2<GV_BF16> {
-    static constexpr uint32_t kNegOne2 = 0xBF80BF80u;
-    static constexpr uint32_t kInf = 0x7F80u;
-    static constexpr uint32_t kMinRelBits = 0x0D800000u;          // 2^-100 as binary32
-    static constexpr bool kExactThr = true;                        // a * inv - thr never rounds to zero above kMinRel
-    static __device__ __forceinline__ float widen(uint32_t h) { return __uint_as_float(h << 16); }
-    static __device__ __forceinline__ uint32_t sub(uint32_t a, uint32_t b) { uint32_t d; asm("sub.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b)); return d; }
-    static __device__ __forceinline__ uint32_t add(uint32_t a, uint32_t b) { uint32_t d; asm("add.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b)); return d; }
-    static __device__ __forceinline__ uint32_t abs(uint32_t a) { uint32_t d; asm("abs.bf16x2 %0, %1;" : "=r"(d) : "r"(a)); return d; }
-    static __device__ __forceinline__ uint32_t fma_relu(uint32_t a, uint32_t b, uint32_t c) { uint32_t d; asm("fma.rn.relu.bf16x2 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c)); return d; }
-    // binary32 x >= 0 (or NaN) -> 16-bit pattern rounded toward zero / toward +Inf
-    static __device__ __forceinline__ uint32_t rz(float x) { return __float_as_uint(x) >> 16; }
-    static __device__ __forceinline__ uint32_t ru(float x) {
-        const uint32_t b = __float_as_uint(x);
-        return (b >> 16) + (((b & 0xFFFFu) != 0u && b < 0x7F800000u) ? 1u : 0u);
-    }
-};
-template <> struct Half2<GV_F16> {
-    static constexpr uint32_t kNegOne2 = 0xBC00BC00u;
-    static constexpr uint32_t kInf = 0x7C00u;
-    static constexpr uint32_t kMinRelBits = 0x39000000u;          // 2^-13 as binary32
-    static constexpr bool kExactThr = false;                       // small differences can round to zero: keep a margin
-    static __device__ __forceinline__ float widen(uint32_t h) { return f16_to_f32(h); }
-    static __device__ __forceinline__ uint32_t sub(uint32_t a, uint32_t b) { uint32_t d; asm("sub.f16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b)); return d; }
-    static __device__ __forceinline__ uint32_t add(uint32_t a, uint32_t b) { uint32_t d; asm("add.f16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b)); return d; }
-    static __device__ __forceinline__ uint32_t abs(uint32_t a) { uint32_t d; asm("abs.f16x2 %0, %1;" : "=r"(d) : "r"(a)); return d; }
-    static __device__ __forceinline__ uint32_t fma_relu(uint32_t a, uint32_t b, uint32_t c) { uint32_t d; asm("fma.rn.relu.f16x2 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c)); return d; }
-    static __device__ __forceinline__ uint32_t rz(float x) { unsigned short h; asm("cvt.rz.f16.f32 %0, %1;" : "=h"(h) : "f"(x)); return h; }
-    static __device__ __forceinline__ uint32_t ru(float x) { unsigned short h; asm("cvt.rp.f16.f32 %0, %1;" : "=h"(h) : "f"(x)); return h; }
-};
-
-struct PackedRef {
-    uint32_t b[4];      // per-element bounds, two per word, positive
-    uint32_t inv[4];    // RU16(1/|r|); 0 where r == 0; +Inf where the reciprocal overflows or r is not finite
-};
-
-template <int DT>
-__device__ __forceinline__ void hoist_packed(const uint4& raw, const TolF& t, PackedRef& o, uint32_t& force) {
-    float rf[8];
-    Widen<DT>::run(raw, rf);
-    uint32_t b16[8], i16[8], umax = 0u;
-#pragma unroll
-    for (int e = 0; e < 8; ++e) {
-        const float a = fabsf(rf[e]);
-        const uint32_t u = __float_as_uint(a);
-        const float tolc = fminf(__fadd_rn(t.atol, __fmul_rn(t.rtol, a)), __uint_as_float(0x7F7FFFFFu));
-        float bound = fminf(tolc, __fmul_rn(a, 0.48f));
-        if (u == 0u) bound = tolc;
-        if (u >= 0x7F800000u) bound = 0.0f;                      // Inf or NaN reference: never settled here
-        b16[e] = Half2<DT>::rz(bound);
-        // inv = the smallest 16-bit number h with h * |r| >= 1, found from the hardware estimate by
-        // testing neighbours; the products of two 16-bit numbers are exact in binary32
-        const float x = rcp_approx(a);
-        uint32_t h = Half2<DT>::rz(__fmul_rd(x, __uint_as_float(0x3F7FFFF0u)));       // a little below 1/|r|
-        if (!(__fmul_rn(Half2<DT>::widen(h), a) >= 1.0f)) h += 1u;
-        if (!(__fmul_rn(Half2<DT>::widen(h), a) >= 1.0f)) h += 1u;
-        if (u == 0u) h = 0u;
-        if (u > 0x7E000000u) h = Half2<DT>::ru(__uint_as_float(0x01000000u));      // |r| > 2^125: 2^-125 >= 1/|r| (estimate may flush)
-        if (u >= 0x7F800000u || (u < 0x00800000u && u != 0u)) h = Half2<DT>::kInf;  // not finite, or binary32-subnormal
-        i16[e] = h;
-        umax = u > umax ? u : umax;
-    }
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-        o.b[j] = b16[2 * j] | (b16[2 * j + 1] << 16);
-        o.inv[j] = i16[2 * j] | (i16[2 * j + 1] << 16);
-    }
-    force = (umax > 0x7F800000u && !t.equal_nan) ? 0xFFFFFFFFu : 0u;
-}
-
-// Nonzero result: the vector must go to the binary32 path. mh2 / thr2 are the packed thresholds of
-// the candidate's CTA accumulator (both halves equal).
-template <int DT>
-__device__ __forceinline__ uint32_t packed_filter(const uint4& c, const uint4& r, const PackedRef& pr, uint32_t mh2,
-                                                  uint32_t thr2) {
-    using H = Half2<DT>;
-    const uint32_t cw[4] = {c.x, c.y, c.z, c.w}, rw[4] = {r.x, r.y, r.z, r.w};
-    const uint32_t nthr2 = thr2 ^ 0x80008000u;
-    uint32_t t[12];
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-        const uint32_t a = H::abs(H::sub(cw[j], rw[j]));
-        t[3 * j] = H::fma_relu(pr.b[j], H::kNegOne2, a);           // relu(a - b)
-        t[3 * j + 1] = H::fma_relu(mh2, H::kNegOne2, a);           // relu(a - mh)
-        t[3 * j + 2] = H::fma_relu(a, pr.inv[j], nthr2);           // relu(a * inv - thr)
-    }
-#ifdef GV_DEBUG_COUNTERS
-    {
-        const uint32_t d1 = H::add(H::add(t[0], t[3]), H::add(t[6], t[9]));
-        const uint32_t d2 = H::add(H::add(t[1], t[4]), H::add(t[7], t[10]));
-        const uint32_t d3 = H::add(H::add(t[2], t[5]), H::add(t[8], t[11]));
-        if (d1) GV_COUNT(3);
-        if (d2) GV_COUNT(4);
-        if (d3) GV_COUNT(5);
-        if (thr2 == 0u) GV_COUNT(6);
-    }
-#endif
-    // pairwise sum (any NaN or positive term makes the sum nonzero)
-    const uint32_t s0 = H::add(H::add(t[0], t[1]), H::add(t[2], t[3]));
-    const uint32_t s1 = H::add(H::add(t[4], t[5]), H::add(t[6], t[7]));
-    const uint32_t s2 = H::add(H::add(t[8], t[9]), H::add(t[10], t[11]));
-    return H::add(H::add(s0, s1), s2);
-}
-
-// Packed thresholds from the binary32 accumulators (monotone: both only ever grow).
-template <int DT>
-__device__ __forceinline__ void refresh_packed_thresholds(CtaAcc* s) {
-    using H = Half2<DT>;
-    const uint32_t mrel = *reinterpret_cast<volatile unsigned int*>(&s->maxrel);
-    const uint32_t mabs = *reinterpret_cast<volatile unsigned int*>(&s->maxabs);
-    if (mrel < H::kMinRelBits) return;                          // keep both at 0: every nonzero |d| is sent on
-    uint32_t thr16, mh16;
-    // A quotient can only raise M when the real a/|r| exceeds M (rounding is monotone), and a * inv >= a/|r|.
-    // bf16: the fused a * inv - thr keeps its sign exactly, so thr = RZ16(M) -- equal quotients (ties of
-    // quantised data) do not fire. fp16: differences below 2^-25 round to zero, so thr sits 2^-10 lower.
-    if (mrel >= 0x7F800000u) thr16 = H::kInf;
-    else if (H::kExactThr) thr16 = H::rz(__uint_as_float(mrel));
-    else thr16 = H::rz(__fmul_rd(__uint_as_float(mrel), 1.0f - 1.0f / 1024.0f));
-    mh16 = H::rz(__uint_as_float(mabs));
-    atomicMax(&s->thr2, thr16 | (thr16 << 16));
-    atomicMax(&s->mh2, mh16 | (mh16 << 16));
 }
 
 // Exact per-element rule over a full vector, using the hoisted reference values (the path taken
@@ -688,9 +582,6 @@ __device__ __forceinline__ void vec_compare(const uint4& c, const uint4& r, uint
 // ------------------------------------------------------------------------------------------
 // mbarrier + bulk async copy (TMA, 1-D, this CTA's shared memory only)
 // ------------------------------------------------------------------------------------------
-__device__ __forceinline__ uint32_t smem_u32(const void* p) {
-    return static_cast<uint32_t>(__cvta_generic_to_shared(p));
-}
 __device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
 }
@@ -778,5 +669,7 @@ __device__ __forceinline__ void push_global(gv_result* res, const CtaAcc& s) {
     if (s.maxabs) atomicMax(reinterpret_cast<unsigned int*>(&res->max_abs_err), s.maxabs);
     if (s.maxrel) atomicMax(reinterpret_cast<unsigned int*>(&res->max_rel_err), s.maxrel);
 }
+
+static_assert(sizeof(CtaAcc) % 16 == 0 && offsetof(CtaAcc, maxabs) % 16 == 0, "CtaAcc layout");
 
 }  // namespace gv

@@ -106,7 +106,10 @@ struct DenseParams {
 #define GV_MINB_FLOAT 2
 #endif
 constexpr int kWarps = kThreads / 32;
-constexpr int kRing = 8;                  // asynchronous copies in flight per lane (power of two)
+#ifndef GV_RING
+#define GV_RING 8
+#endif
+constexpr int kRing = GV_RING;            // asynchronous copies in flight per lane (power of two)
 constexpr int kWarpTile = 512;            // bytes of one warp-tile
 
 struct DenseSmem {
@@ -141,25 +144,12 @@ __device__ __noinline__ void settle_vector_int(uint4 c, uint4 r, uint64_t elem0,
     if (a.cnt) atomicAdd(&s->cnt, static_cast<unsigned long long>(a.cnt));
 }
 
-// A 16-bit float vector the packed filter could not settle: the binary32 fast path decides, and the
-// exact rule takes over where that one cannot either. Out of line; refreshes the packed thresholds.
-template <int DT>
-__device__ __noinline__ void resolve_vector_f32(uint4 c, uint4 r, uint64_t elem0, TolF t, CtaAcc* s) {
-    RefVec<8> rv;
-    uint32_t force;
-    GV_COUNT(0);
-    hoist_ref<DT>(r, t, rv, force);
-    if (!vec_fast_float<DT>(c, rv, s)) { GV_COUNT(1); settle_vector_exact<DT>(c, rv, elem0, t, s); }
-    refresh_packed_thresholds<DT>(s);
-}
-
 // BIGK: word indices of the hash need more than 32 bits (tensors of 32 GiB and more).
 template <int DT, bool BIGK>
 __global__ void __launch_bounds__(kThreads, Traits<DT>::IS_FLOAT ? GV_MINB_FLOAT : 3) dense_kernel(const __grid_constant__ DenseParams p) {
     constexpr int ESZ = Traits<DT>::ESZ;
     constexpr int EPV = 16 / ESZ;
     constexpr bool IS_FLOAT = Traits<DT>::IS_FLOAT;
-    constexpr bool PACKED = (DT == GV_BF16 || DT == GV_F16);     // 16-bit floats: packed filter first
     extern __shared__ __align__(128) unsigned char smem[];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     CtaAcc* cacc = reinterpret_cast<CtaAcc*>(smem + DenseSmem::kAccOff);
@@ -183,10 +173,7 @@ __global__ void __launch_bounds__(kThreads, Traits<DT>::IS_FLOAT ? GV_MINB_FLOAT
         mbar_fence_init();
     }
     if (tid == 0) *s_refhash = 0;
-    if (tid < kChunk) {
-        cacc[tid].clear();
-        if (tid < p.N) cacc[tid].rec = &p.results[tid];
-    }
+    if (tid < kChunk) cacc[tid].clear();
     __syncthreads();
 
     uint32_t phase[2] = {0u, 0u};
@@ -197,7 +184,7 @@ __global__ void __launch_bounds__(kThreads, Traits<DT>::IS_FLOAT ? GV_MINB_FLOAT
 
     for (int g = 0; g < num_groups; ++g) {
         const int kg = min(kChunk, p.N - g * kChunk);
-        const unsigned char* const* cand = &p.cands[g * kChunk];
+        const int cand0 = g * kChunk;          // first candidate of the chunk (pointers are read straight from the parameters)
         for (int k = 0; k < kg; ++k) slots[k * 32] = make_uint2(0u, 0u);
 
         // ================= fast loop: full warp-tiles, every base 16-byte aligned =================
@@ -208,29 +195,12 @@ __global__ void __launch_bounds__(kThreads, Traits<DT>::IS_FLOAT ? GV_MINB_FLOAT
 
             // Values derived from the reference vector, computed lazily: only when a candidate
             // vector differs from it (exact copies never pay for them).
-            RefVec<(IS_FLOAT && !PACKED) ? EPV : 1> rv;
-            PackedRef pr;
+            RefVec<IS_FLOAT ? EPV : 1> rv;
             uint32_t force = 0u;
             bool hoisted = false;
-            // maxima other CTAs have published for the chunk's candidates, fetched one tile ahead
-            uint32_t seen_abs = 0u, seen_rel = 0u;
             auto new_tile = [&](const uint4& r) {
                 hoisted = false;
                 force = 0u;
-                if constexpr (IS_FLOAT) {
-                    if (lane < kg) {
-                        CtaAcc* s = &cacc[lane];
-                        if (seen_abs > *reinterpret_cast<volatile unsigned int*>(&s->maxabs)) atomicMax(&s->maxabs, seen_abs);
-                        if (seen_rel > *reinterpret_cast<volatile unsigned int*>(&s->maxrel)) {
-                            atomicMax(&s->maxrel, seen_rel);
-                            atomicMax(&s->thr, rel_threshold_bits(seen_rel));
-                        }
-                        if constexpr (PACKED) refresh_packed_thresholds<DT>(s);
-                        const gv_result* rec = &p.results[g * kChunk + lane];
-                        asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(seen_abs) : "l"(&rec->max_abs_err));
-                        asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(seen_rel) : "l"(&rec->max_rel_err));
-                    }
-                }
                 if constexpr (IS_FLOAT) {
                     // only a NaN in the reference (without equal_nan) forces identical vectors onto the
                     // compare path; that needs no arithmetic, just the exponent/mantissa test
@@ -257,8 +227,7 @@ __global__ void __launch_bounds__(kThreads, Traits<DT>::IS_FLOAT ? GV_MINB_FLOAT
             auto ensure_hoisted = [&](const uint4& r) {
                 if (!hoisted) {
                     uint32_t f2;
-                    if constexpr (PACKED) hoist_packed<DT>(r, tol, pr, f2);
-                    else if constexpr (IS_FLOAT) hoist_ref<DT>(r, tol, rv, f2);
+                    if constexpr (IS_FLOAT) hoist_ref<DT>(r, tol, rv, f2);
                     hoisted = true;
                 }
             };
@@ -266,13 +235,8 @@ __global__ void __launch_bounds__(kThreads, Traits<DT>::IS_FLOAT ? GV_MINB_FLOAT
             auto differing = [&](const uint4& c, const uint4& r, int k) {
                 if constexpr (!IS_FLOAT) {
                     settle_vector_int<DT>(c, r, voff / ESZ, &cacc[k]);
-                } else if constexpr (PACKED) {
-                    const uint32_t mh2 = *reinterpret_cast<volatile unsigned int*>(&cacc[k].mh2);
-                    const uint32_t thr2 = *reinterpret_cast<volatile unsigned int*>(&cacc[k].thr2);
-                    if (packed_filter<DT>(c, r, pr, mh2, thr2) != 0u)
-                        resolve_vector_f32<DT>(c, r, voff / ESZ, tol, &cacc[k]);
                 } else {
-                    if (!vec_fast_float<DT>(c, rv, &cacc[k])) settle_vector_exact<DT>(c, rv, voff / ESZ, tol, &cacc[k]);
+                    if (!vec_fast_float<DT>(c, rv, &cacc[k], voff / ESZ)) settle_vector_exact<DT>(c, rv, voff / ESZ, tol, &cacc[k]);
                 }
             };
             // one visit: candidate vector c (already read from the ring) against the held reference
@@ -319,7 +283,7 @@ __global__ void __launch_bounds__(kThreads, Traits<DT>::IS_FLOAT ? GV_MINB_FLOAT
                 constexpr int U = GV_UNROLL;               // visits per unrolled block (divides kRing)
 #pragma unroll 1
                 for (int k = 0; k < kRing; ++k) {
-                    cp_async16(ring_base + k * 512u, cand[k] + voff);
+                    cp_async16(ring_base + k * 512u, p.cands[cand0 + k] + voff);
                     if ((k % U) == U - 1) cp_async_commit();
                 }
 #pragma unroll 1
@@ -332,7 +296,7 @@ __global__ void __launch_bounds__(kThreads, Traits<DT>::IS_FLOAT ? GV_MINB_FLOAT
 #pragma unroll 1
                     for (int k0 = 0; k0 < kChunk; k0 += U) {
                         const uint32_t stage0 = ring_base + (k0 & (kRing - 1)) * 512u;
-                        const unsigned char* const* refill = cand + ((k0 + kRing) & (kChunk - 1));
+                        const int refill = cand0 + ((k0 + kRing) & (kChunk - 1));
                         const uint64_t refill_off = k0 < kRing ? voff : voff + tile_stride;
                         const bool live = k0 < kRing || has_next;
                         cp_async_wait<kRing / U - 1>();     // the block of U stages issued kRing visits ago has landed
@@ -362,7 +326,7 @@ __global__ void __launch_bounds__(kThreads, Traits<DT>::IS_FLOAT ? GV_MINB_FLOAT
                         }
 #pragma unroll
                         for (int u = 0; u < U; ++u) {
-                            if (live) cp_async16(stage0 + u * 512u, refill[u] + refill_off);
+                            if (live) cp_async16(stage0 + u * 512u, p.cands[refill + u] + refill_off);
                         }
                         cp_async_commit();                  // one group per block of U refills
                     }
@@ -376,7 +340,7 @@ __global__ void __launch_bounds__(kThreads, Traits<DT>::IS_FLOAT ? GV_MINB_FLOAT
                 uint64_t issued = 0;
                 auto issue_one = [&]() {
                     if (issued < visits) {
-                        cp_async16(ring_base + (static_cast<uint32_t>(issued) & (kRing - 1)) * 512u, cand[issue_k] + issue_off);
+                        cp_async16(ring_base + (static_cast<uint32_t>(issued) & (kRing - 1)) * 512u, p.cands[cand0 + issue_k] + issue_off);
                         ++issued;
                         if (++issue_k == kg) { issue_k = 0; issue_off += tile_stride; }
                     }
@@ -425,7 +389,7 @@ __global__ void __launch_bounds__(kThreads, Traits<DT>::IS_FLOAT ? GV_MINB_FLOAT
                 const int nwords = nvalid * ESZ > 8 ? 2 : 1;
                 if (g == 0 && p.ref_hash) my_ref_hash += hash_vec(r, voff / 8, nwords);
                 for (int k = 0; k < kg; ++k) {
-                    const uint4 c = load_vec_generic<ESZ>(cand[k], voff, nbytes);
+                    const uint4 c = load_vec_generic<ESZ>(p.cands[cand0 + k], voff, nbytes);
                     Acc a;
                     a.clear();
                     a.hash = hash_vec(c, voff / 8, nwords);
@@ -448,11 +412,7 @@ __global__ void __launch_bounds__(kThreads, Traits<DT>::IS_FLOAT ? GV_MINB_FLOAT
         }
         __syncthreads();
         if (tid < kg) push_global(&p.results[g * kChunk + tid], cacc[tid]);
-        if (tid < kChunk) {
-            cacc[tid].clear();
-            const int next = (g + 1) * kChunk + tid;
-            if (next < p.N) cacc[tid].rec = &p.results[next];
-        }
+        if (tid < kChunk) cacc[tid].clear();
         __syncthreads();
     }
 
@@ -483,8 +443,7 @@ struct RaggedParams {
     int equal_nan;
 };
 
-constexpr int kRaggedV = 4;                                  // 16-byte vectors per thread per tile
-constexpr int kRaggedTile = kThreads * 16 * kRaggedV;        // 16 KiB
+constexpr int kRaggedTile = kWarpTile;      // ragged work is split into the same 512-byte warp-tiles
 
 // Pre-pass: validates the tables and turns sizes into an exclusive prefix of tile counts.
 // One CTA; T is at most a few million in practice (one pass of 1024-wide chunks).
@@ -546,144 +505,211 @@ __global__ void __launch_bounds__(1024) ragged_prepass_kernel(RaggedParams p) {
     }
 }
 
-// One tile of one tensor against its N candidates; block-wide reduction per candidate.
-template <int DT>
-__device__ __forceinline__ void ragged_tile(const RaggedParams& p, int64_t t, uint64_t tile, uint64_t n,
-                                            const unsigned char* ref, const unsigned char* rbuf,
-                                            CtaAcc* cacc) {
-    constexpr int ESZ = Traits<DT>::ESZ;
-    constexpr int EPV = 16 / ESZ;
-    constexpr int V = kRaggedV;
-    const int tid = threadIdx.x;
-    const uint64_t nbytes = n * ESZ;
-    const TolF tol = {p.atol, p.rtol, p.equal_nan};
-    (void)ref;
+// Ragged kernel, organisation. The warp-tiles of all tensors form one sequence (tile_prefix); every
+// warp of the grid takes one contiguous stretch of it, so it meets only a few tensor boundaries.
+// Inside a tensor it works like the dense kernel's general shape: the lane's reference vector is
+// held in registers and compared with the same vector of each of the tensor's candidates; the hash
+// partials of the current tensor live in per-(candidate, lane) shared-memory slots and the other
+// statistics in per-warp shared accumulators, all flushed with integer atomics when the warp leaves
+// the tensor. No barrier is used anywhere: warps never share a tensor's accumulators.
+struct RaggedSmem {
+    static constexpr size_t kSlotOff = 0;                                                  // [warp][kChunk][32] u64
+    static constexpr size_t kAccOff = kSlotOff + size_t(kWarps) * kChunk * 32 * 8;         // [warp][kChunk] CtaAcc
+    static constexpr size_t kPtrOff = kAccOff + size_t(kWarps) * kChunk * sizeof(CtaAcc);  // [warp][kChunk] candidate pointers
+    static constexpr size_t kTotal = kPtrOff + size_t(kWarps) * kChunk * 8;
+};
 
-    uint4 r[V];
-    uint64_t voff[V];
-    int nvalid[V];
-    bool full[V];
-#pragma unroll
-    for (int v = 0; v < V; ++v) {
-        r[v] = *reinterpret_cast<const uint4*>(rbuf + (v * kThreads + tid) * 16);
-        voff[v] = tile * kRaggedTile + static_cast<uint64_t>(v * kThreads + tid) * 16;
-        const uint64_t rem = voff[v] < nbytes ? nbytes - voff[v] : 0;
-        nvalid[v] = rem >= 16 ? EPV : static_cast<int>(rem / ESZ);
-        full[v] = rem >= 16;
-    }
-    for (int j = 0; j < p.N; ++j) {
-        const unsigned char* cp = p.cand_base + p.cand_off[t * p.N + j];
-        const bool cal = (reinterpret_cast<uintptr_t>(cp) & 15u) == 0;
-        uint4 c[V];
-#pragma unroll
-        for (int v = 0; v < V; ++v) {
-            if (cal && full[v]) c[v] = ldg_stream(cp + voff[v]);
-            else if (nvalid[v] > 0) c[v] = load_vec_generic<ESZ>(cp, voff[v], nbytes);
-            else c[v] = make_uint4(0u, 0u, 0u, 0u);
+// A full candidate vector that differs from its reference vector, any dtype. Out of line and
+// switched on the dtype at run time so that the ragged hot loop exists once, not once per dtype
+// (mixed-dtype batches would otherwise thrash the instruction cache). The derived reference values
+// are computed per call here: a ragged tile has only a handful of candidates to amortise them over.
+template <int DT>
+__device__ __forceinline__ void ragged_differing_t(const uint4& c, const uint4& r, uint64_t elem0, const TolF& tol,
+                                                   CtaAcc* s) {
+    if constexpr (Traits<DT>::IS_FLOAT) {
+        RefVec<16 / Traits<DT>::ESZ> rv;
+        uint32_t force;
+        hoist_ref<DT>(r, tol, rv, force);
+        if (!vec_fast_float<DT>(c, rv, s, elem0)) {
+            Acc a;
+            a.clear();
+            const uint32_t thr = *reinterpret_cast<volatile unsigned int*>(&s->thr);
+            vec_exact_float<DT>(c, rv, elem0, tol, thr, a);
+            push_rare(s, a);
+            if (a.cnt) atomicAdd(&s->cnt, static_cast<unsigned long long>(a.cnt));
+            raise_maxabs(s, a.maxabs);
         }
+    } else {
         Acc a;
         a.clear();
-#pragma unroll
-        for (int v = 0; v < V; ++v) {
-            if (nvalid[v] > 0) {
-                a.hash += full[v] ? hash_vec_full(c[v], voff[v] / 8)
-                                  : hash_vec(c[v], voff[v] / 8, nvalid[v] * ESZ > 8 ? 2 : 1);
-                vec_compare<DT>(c[v], r[v], voff[v] / ESZ, nvalid[v], tol, a);
-            }
-        }
-        // CTA-wide combine for candidate j (slot j % 2 so the next candidate need not wait)
-        CtaAcc* s = &cacc[j & 1];
-        const uint64_t h = warp_sum_u64(a.hash);
-        const uint32_t c32 = __reduce_add_sync(0xFFFFFFFFu, a.cnt);
-        const uint32_t m = __reduce_max_sync(0xFFFFFFFFu, a.maxabs);
-        if ((tid & 31) == 0) {
-            if (h) atomicAdd(&s->hash, static_cast<unsigned long long>(h));
-            if (c32) atomicAdd(&s->cnt, static_cast<unsigned long long>(c32));
-            if (m) atomicMax(&s->maxabs, m);
-        }
+        vec_int<DT>(c, r, elem0, 16 / Traits<DT>::ESZ, a);
         push_rare(s, a);
-        __syncthreads();
-        if (tid == 0) {
-            push_global(&p.results[t * p.N + j], *s);
-            s->clear();
-        }
-        // the slot is reused two candidates later; the barrier of the next iteration orders that
+        if (a.cnt) atomicAdd(&s->cnt, static_cast<unsigned long long>(a.cnt));
     }
-    __syncthreads();
+}
+__device__ __noinline__ void ragged_differing(int dt, uint4 c, uint4 r, uint64_t byte_off, TolF tol, CtaAcc* s) {
+    switch (dt) {
+        case GV_F32: ragged_differing_t<GV_F32>(c, r, byte_off / 4, tol, s); break;
+        case GV_BF16: ragged_differing_t<GV_BF16>(c, r, byte_off / 2, tol, s); break;
+        case GV_F16: ragged_differing_t<GV_F16>(c, r, byte_off / 2, tol, s); break;
+        case GV_I32: ragged_differing_t<GV_I32>(c, r, byte_off / 4, tol, s); break;
+        default: ragged_differing_t<GV_I64>(c, r, byte_off / 8, tol, s); break;
+    }
+}
+// The partial vector at the end of a tensor: element by element through the general rule.
+__device__ __noinline__ void ragged_partial(int dt, uint4 c, uint4 r, uint64_t byte_off, int nvalid, TolF tol,
+                                            CtaAcc* s, uint2* slot) {
+    Acc a;
+    a.clear();
+    const int esz = elem_size(dt);
+    a.hash = hash_vec(c, byte_off / 8, nvalid * esz > 8 ? 2 : 1);
+    switch (dt) {
+        case GV_F32: vec_compare<GV_F32>(c, r, byte_off / 4, nvalid, tol, a); break;
+        case GV_BF16: vec_compare<GV_BF16>(c, r, byte_off / 2, nvalid, tol, a); break;
+        case GV_F16: vec_compare<GV_F16>(c, r, byte_off / 2, nvalid, tol, a); break;
+        case GV_I32: vec_compare<GV_I32>(c, r, byte_off / 4, nvalid, tol, a); break;
+        default: vec_compare<GV_I64>(c, r, byte_off / 8, nvalid, tol, a); break;
+    }
+    const uint2 sl = *slot;
+    const uint64_t h = pack64(sl.x, sl.y) + a.hash;
+    *slot = make_uint2(static_cast<uint32_t>(h), static_cast<uint32_t>(h >> 32));
+    push_rare(s, a);
+    if (a.cnt) atomicAdd(&s->cnt, static_cast<unsigned long long>(a.cnt));
+    raise_maxabs(s, a.maxabs);
+}
+__device__ __forceinline__ uint4 load_vec_any(int esz, const unsigned char* base, uint64_t byte_off, uint64_t nbytes) {
+    if (esz == 2) return load_vec_generic<2>(base, byte_off, nbytes);
+    if (esz == 4) return load_vec_generic<4>(base, byte_off, nbytes);
+    return load_vec_generic<8>(base, byte_off, nbytes);
+}
+// NaN anywhere in a reference vector of a float dtype (bit tests only)
+__device__ __forceinline__ bool vec_has_nan(int dt, const uint4& r) {
+    const uint32_t w[4] = {r.x, r.y, r.z, r.w};
+    bool any = false;
+    if (dt == GV_F32) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) any = any || is_nan_bits(w[j]);
+    } else if (dt == GV_BF16 || dt == GV_F16) {
+        const uint32_t inf = dt == GV_BF16 ? 0x7F80u : 0x7C00u;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const uint32_t a = w[j] & 0x7FFF7FFFu;
+            any = any || (a & 0xFFFFu) > inf || (a >> 16) > inf;
+        }
+    }
+    return any;
 }
 
-__global__ void __launch_bounds__(kThreads) ragged_kernel(const __grid_constant__ RaggedParams p) {
-    __shared__ __align__(128) unsigned char rbuf[kRaggedTile];
-    __shared__ CtaAcc cacc[2];
-    __shared__ uint64_t bar;
-    const int tid = threadIdx.x;
-    if (tid == 0) {
-        mbar_init(&bar, 1);
-        mbar_fence_init();
-        cacc[0].clear();
-        cacc[1].clear();
-    }
-    __syncthreads();
-    const int64_t total = p.tile_prefix[p.T];
-    uint32_t phase = 0;
-    for (int64_t item = blockIdx.x; item < total; item += gridDim.x) {
-        // tensor of this item: last t with tile_prefix[t] <= item
-        int64_t lo = 0, hi = p.T;          // invariant: tile_prefix[lo] <= item < tile_prefix[hi]
-        while (hi - lo > 1) {
-            const int64_t mid = (lo + hi) >> 1;
-            if (p.tile_prefix[mid] <= item) lo = mid; else hi = mid;
+// Tiles [tile_begin, tile_end) of one tensor against kg of its candidates (pointers in wptr).
+__device__ __forceinline__ void ragged_stretch(const RaggedParams& p, int dt, const unsigned char* ref, uint64_t n,
+                                               uint64_t tile_begin, uint64_t tile_end, int kg, uint2* slots,
+                                               CtaAcc* wacc, const unsigned char* const* wptr, int lane) {
+    constexpr int KC = 4;                           // candidates loaded together
+    const int esz = elem_size(dt);
+    const uint64_t nbytes = n * esz;
+    const TolF tol = {p.atol, p.rtol, p.equal_nan};
+    const bool ref_al = (reinterpret_cast<uintptr_t>(ref) & 15u) == 0;
+    const bool nan_matters = (dt <= GV_F16) && !p.equal_nan;
+#pragma unroll 1
+    for (uint64_t tile = tile_begin; tile < tile_end; ++tile) {
+        const uint64_t voff = tile * kWarpTile + lane * 16;
+        const uint64_t rem = voff < nbytes ? nbytes - voff : 0;
+        const int nvalid = rem >= 16 ? 16 / esz : static_cast<int>(rem / esz);
+        const bool full = rem >= 16;
+        uint4 r = make_uint4(0u, 0u, 0u, 0u);
+        if (full && ref_al) r = ldg_stream(ref + voff);
+        else if (nvalid > 0) r = load_vec_any(esz, ref, voff, nbytes);
+        // an identical vector still needs the rule when the reference holds a NaN that is not "equal"
+        const bool force = nan_matters && full && vec_has_nan(dt, r);
+#pragma unroll 1
+        for (int k0 = 0; k0 < kg; k0 += KC) {
+            uint4 c[KC];
+#pragma unroll
+            for (int u = 0; u < KC; ++u) {
+                c[u] = make_uint4(0u, 0u, 0u, 0u);
+                if (k0 + u < kg) {
+                    const unsigned char* cp = wptr[k0 + u];
+                    if (full && (reinterpret_cast<uintptr_t>(cp) & 15u) == 0) c[u] = ldg_stream(cp + voff);
+                    else if (nvalid > 0) c[u] = load_vec_any(esz, cp, voff, nbytes);
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < KC; ++u) {
+                const int k = k0 + u;
+                if (k < kg) {
+                    if (full) {
+                        uint64_t h = hash_vec_full(c[u], voff / 8);
+                        const uint2 sl = slots[k * 32];
+                        h += pack64(sl.x, sl.y);
+                        slots[k * 32] = make_uint2(static_cast<uint32_t>(h), static_cast<uint32_t>(h >> 32));
+                        const bool differs = (c[u].x != r.x) || (c[u].y != r.y) || (c[u].z != r.z) || (c[u].w != r.w) || force;
+                        if (differs) ragged_differing(dt, c[u], r, voff, tol, &wacc[k]);
+                    } else if (nvalid > 0) {
+                        ragged_partial(dt, c[u], r, voff, nvalid, tol, &wacc[k], &slots[k * 32]);
+                    }
+                }
+            }
         }
-        const int64_t t = lo;
-        const uint64_t tile = static_cast<uint64_t>(item - p.tile_prefix[t]);
+    }
+}
+
+__global__ void __launch_bounds__(kThreads, 2) ragged_kernel(const __grid_constant__ RaggedParams p) {
+    extern __shared__ __align__(128) unsigned char smem[];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    uint2* slots = reinterpret_cast<uint2*>(smem + RaggedSmem::kSlotOff) + size_t(warp) * kChunk * 32 + lane;
+    CtaAcc* wacc = reinterpret_cast<CtaAcc*>(smem + RaggedSmem::kAccOff) + warp * kChunk;
+    const unsigned char** wptr = reinterpret_cast<const unsigned char**>(smem + RaggedSmem::kPtrOff) + warp * kChunk;
+
+    const uint64_t total = static_cast<uint64_t>(p.tile_prefix[p.T]);
+    const uint64_t gw = static_cast<uint64_t>(blockIdx.x) * kWarps + warp;
+    const uint64_t GW = static_cast<uint64_t>(gridDim.x) * kWarps;
+    // contiguous stretch [begin, end) of the global tile sequence for this warp
+    const uint64_t per = total / GW, extra = total % GW;
+    const uint64_t begin = gw * per + (gw < extra ? gw : extra);
+    const uint64_t end = begin + per + (gw < extra ? 1 : 0);
+    if (begin >= end) return;
+
+    // tensor holding tile `begin`: last t with tile_prefix[t] <= begin (tensors without tiles are skipped)
+    int64_t lo = 0, hi = p.T;
+    while (hi - lo > 1) {
+        const int64_t mid = (lo + hi) >> 1;
+        if (static_cast<uint64_t>(p.tile_prefix[mid]) <= begin) lo = mid; else hi = mid;
+    }
+    int64_t t = lo;
+    uint64_t item = begin;
+    while (item < end) {
+        const uint64_t t_first = static_cast<uint64_t>(p.tile_prefix[t]);
+        const uint64_t t_last = static_cast<uint64_t>(p.tile_prefix[t + 1]);
+        if (t_last <= item) { ++t; continue; }                  // empty or already finished tensor
         const int dt = p.dtypes[t];
         const int esz = elem_size(dt);
         const uint64_t n = p.n_elems ? static_cast<uint64_t>(p.n_elems[t])
                                      : static_cast<uint64_t>(p.ref_off[t + 1] - p.ref_off[t]) / esz;
         const unsigned char* ref = p.ref_base + p.ref_off[t];
-        const uint64_t nbytes = n * esz;
-        const uint64_t rem = nbytes - tile * kRaggedTile;
-        const uint32_t tb = static_cast<uint32_t>(rem < kRaggedTile ? rem : kRaggedTile);
-        const unsigned char* src = ref + tile * kRaggedTile;
-
-        bool ok = true;
-        if ((reinterpret_cast<uintptr_t>(src) & 15u) == 0 && (tb & 15u) == 0) {
-            if (tid == 0) {
-                fence_proxy_async();
-                mbar_expect_tx(&bar, tb);
-                bulk_load(rbuf, src, tb, &bar);
+        const uint64_t tile_begin = item - t_first;
+        const uint64_t tile_end = (t_last < end ? t_last : end) - t_first;
+        for (int c0 = 0; c0 < p.N; c0 += kChunk) {
+            const int kg = min(kChunk, p.N - c0);
+            __syncwarp();
+            if (lane < kg) {
+                wptr[lane] = p.cand_base + p.cand_off[t * p.N + c0 + lane];
+                wacc[lane].clear();
             }
-            // (bytes of rbuf beyond tb keep stale contents; vectors there have no valid element)
-            ok = mbar_wait_bounded(&bar, phase);
-            if (ok) phase ^= 1u;
-        } else {
-            for (uint32_t o = tid * esz; o < static_cast<uint32_t>(kRaggedTile); o += kThreads * esz) {
-                if (esz == 2)
-                    *reinterpret_cast<unsigned short*>(rbuf + o) =
-                        o < tb ? *reinterpret_cast<const unsigned short*>(src + o) : static_cast<unsigned short>(0);
-                else if (esz == 4)
-                    *reinterpret_cast<uint32_t*>(rbuf + o) = o < tb ? *reinterpret_cast<const uint32_t*>(src + o) : 0u;
-                else
-                    *reinterpret_cast<unsigned long long*>(rbuf + o) =
-                        o < tb ? *reinterpret_cast<const unsigned long long*>(src + o) : 0ull;
+            for (int k = 0; k < kg; ++k) slots[k * 32] = make_uint2(0u, 0u);
+            __syncwarp();
+            ragged_stretch(p, dt, ref, n, tile_begin, tile_end, kg, slots, wacc, wptr, lane);
+            __syncwarp();
+            // leave the tensor (or this group of its candidates): combine and publish
+            for (int k = 0; k < kg; ++k) {
+                const uint2 sl = slots[k * 32];
+                const uint64_t h = warp_sum_u64(pack64(sl.x, sl.y));
+                if (lane == 0 && h) wacc[k].hash += h;
             }
+            __syncwarp();
+            if (lane < kg) push_global(&p.results[t * p.N + c0 + lane], wacc[lane]);
         }
-        ok = __syncthreads_and(ok ? 1 : 0) != 0;
-        if (!ok) {
-            if (tid == 0) {
-                atomicOr(p.status, kStatusTimeout);
-                (void)mbar_wait_bounded(&bar, phase);
-            }
-            __syncthreads();
-            return;
-        }
-        switch (dt) {
-            case GV_F32: ragged_tile<GV_F32>(p, t, tile, n, ref, rbuf, cacc); break;
-            case GV_BF16: ragged_tile<GV_BF16>(p, t, tile, n, ref, rbuf, cacc); break;
-            case GV_F16: ragged_tile<GV_F16>(p, t, tile, n, ref, rbuf, cacc); break;
-            case GV_I32: ragged_tile<GV_I32>(p, t, tile, n, ref, rbuf, cacc); break;
-            default: ragged_tile<GV_I64>(p, t, tile, n, ref, rbuf, cacc); break;
-        }
-        // ragged_tile ends with a barrier: rbuf may be overwritten by the next item
+        item = t_first + tile_end;
+        ++t;
     }
 }
 
@@ -896,12 +922,14 @@ gv_status gv_verify_ragged(const void* ref_base, const int64_t* ref_off, const v
     int dev = 0;
     GV_CUDA(cudaGetDevice(&dev));
     if (blocks_per_sm[dev] == 0) {
+        GV_CUDA(cudaFuncSetAttribute(gv::ragged_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     static_cast<int>(gv::RaggedSmem::kTotal)));
         int b = 0;
-        GV_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b, gv::ragged_kernel, gv::kThreads, 0));
+        GV_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b, gv::ragged_kernel, gv::kThreads, gv::RaggedSmem::kTotal));
         blocks_per_sm[dev] = b > 0 ? b : 1;
     }
     const unsigned grid = static_cast<unsigned>(sm_count * blocks_per_sm[dev]);
-    gv::ragged_kernel<<<grid, gv::kThreads, 0, st>>>(p);
+    gv::ragged_kernel<<<grid, gv::kThreads, gv::RaggedSmem::kTotal, st>>>(p);
     GV_CUDA(cudaGetLastError());
     return GV_OK;
 }

@@ -124,6 +124,41 @@ gv_status gv_verify_ragged(const void* ref_base, const int64_t* ref_off, const v
                            int64_t T, int32_t N, const gv_tol* tol, gv_result* results,
                            void* workspace, size_t workspace_bytes, void* cuda_stream);
 
+/* Ragged verification without any caller-provided scratch. (The paper has no counterpart to this
+ * entry point; it exists for a class of callers, not for a passage of the text.)
+ *
+ * Who needs it: host programs that are not allowed to obtain device memory themselves -- for example a
+ * plug-in running inside a framework or server that has handed the whole device to its own pool and
+ * forbids foreign cudaMalloc/cudaFree calls, or a control loop that cannot accept the device-wide
+ * synchronisation an allocation may cause -- and that therefore cannot produce the `workspace` buffer
+ * gv_verify_ragged asks for. Here the scratch (a status word and the tile-prefix table the pre-pass
+ * builds) lives in a fixed array inside the library's device image: 256 + 8 * (GV_NOALLOC_MAX_TENSORS + 1)
+ * bytes (about 0.5 MiB), held on every GPU that loads the library until the process exits. The call
+ * itself allocates and frees nothing, on the host or on the device, and calls no allocating routine.
+ *
+ * Arguments are those of gv_verify_ragged minus the workspace, plus
+ *   status_out  device, one uint32, nullable: receives the status bits that gv_check() would report
+ *               for a workspace (0 = fine, bit 0 = device-side wait expired, bit 1 = inconsistent
+ *               tables); valid once the stream has passed the call. With NULL the bits are not
+ *               retrievable.
+ * Limits and rules:
+ *   - T <= GV_NOALLOC_MAX_TENSORS, otherwise GV_ERR_WORKSPACE is returned, nothing is enqueued and
+ *     gv_last_cuda_error() explains the limit. N is not limited.
+ *   - The first call on each device looks up the array's device address (cudaGetSymbolAddress, with
+ *     that device current) and sets kernel attributes. Make that first call outside any stream
+ *     capture.
+ *   - All calls on a device share the one array, and it keeps the previous call's contents. The call
+ *     rewrites everything it later reads, so calls that follow one another on a stream are
+ *     independent; calls whose kernels overlap on the GPU (different streams, no ordering between
+ *     them) race on the array and give undefined records. Order them, or use gv_verify_ragged with
+ *     separate workspaces.
+ * Results are byte-identical to gv_verify_ragged's. */
+#define GV_NOALLOC_MAX_TENSORS 65536
+gv_status gv_verify_ragged_noalloc(const void* ref_base, const int64_t* ref_off, const void* cand_base,
+                                   const int64_t* cand_off, const uint8_t* dtypes, const int64_t* n_elems,
+                                   int64_t T, int32_t N, const gv_tol* tol, gv_result* results,
+                                   uint32_t* status_out, void* cuda_stream);
+
 /* Content hash of nbytes bytes at buf (device) into *out (device). buf needs no alignment.
  * The same function the verifier applies to each candidate (used to de-duplicate candidates). */
 gv_status gv_hash(const void* buf, uint64_t nbytes, uint64_t* out, void* cuda_stream);

@@ -934,6 +934,95 @@ gv_status gv_verify_ragged(const void* ref_base, const int64_t* ref_off, const v
     return GV_OK;
 }
 
+// ---------------------------------------------------------------------------------------------
+// gv_verify_ragged_noalloc: the ragged verification for callers that have no device memory to lend.
+// Its scratch (status word + tile-prefix table) is this fixed array, resident on every GPU that loads
+// the library for as long as the process lives.
+// ---------------------------------------------------------------------------------------------
+#define GV_NOALLOC_SCRATCH_BYTES (256 + (GV_NOALLOC_MAX_TENSORS + 1) * 8)
+static __device__ __align__(256) unsigned char g_noalloc_scratch[GV_NOALLOC_SCRATCH_BYTES];
+
+// Device address of g_noalloc_scratch per device. In host code the array's name is only a handle for
+// the runtime, not an address a kernel can use; the address is asked for once per device, with that
+// device current, the first time the entry point runs there.
+static void* g_noalloc_ptr[64] = {nullptr};
+
+gv_status gv_verify_ragged_noalloc(const void* ref_base, const int64_t* ref_off, const void* cand_base,
+                                   const int64_t* cand_off, const uint8_t* dtypes, const int64_t* n_elems,
+                                   int64_t T, int32_t N, const gv_tol* tol, gv_result* results,
+                                   uint32_t* status_out, void* cuda_stream) {
+    if (T < 0 || N < 0) return GV_ERR_INVALID_ARG;
+    if (T > GV_NOALLOC_MAX_TENSORS) {
+        snprintf(g_last_error, sizeof(g_last_error),
+                 "gv_verify_ragged_noalloc: T = %lld exceeds GV_NOALLOC_MAX_TENSORS = %d; split the batch or use "
+                 "gv_verify_ragged with a caller-provided workspace", static_cast<long long>(T), GV_NOALLOC_MAX_TENSORS);
+        return GV_ERR_WORKSPACE;
+    }
+    if (T > 0 && (!ref_base || !ref_off || !dtypes)) return GV_ERR_INVALID_ARG;
+    if (T > 0 && N > 0 && (!cand_base || !cand_off || !results)) return GV_ERR_INVALID_ARG;
+    if (!tol_valid(tol)) return GV_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(ref_off) & 7u) || (reinterpret_cast<uintptr_t>(cand_off) & 7u) ||
+        (reinterpret_cast<uintptr_t>(n_elems) & 7u) || (reinterpret_cast<uintptr_t>(results) & 7u) ||
+        (reinterpret_cast<uintptr_t>(status_out) & 3u))
+        return GV_ERR_MISALIGNED;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    int sm_count = 0;
+    gv_status rc = device_info(&sm_count);
+    if (rc != GV_OK) return rc;
+    int dev = 0;
+    GV_CUDA(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) return GV_ERR_CUDA;
+    if (!g_noalloc_ptr[dev]) {
+        void* ptr = nullptr;
+        GV_CUDA(cudaGetSymbolAddress(&ptr, g_noalloc_scratch));
+        g_noalloc_ptr[dev] = ptr;
+    }
+    unsigned char* scratch = static_cast<unsigned char*>(g_noalloc_ptr[dev]);
+
+    // The array still holds the previous call's status word and table. The status word is cleared by
+    // the first kernel below; the table is rewritten in full (entries 0..T) by the pre-pass before the
+    // main kernel reads it, so nothing else needs to start from zero.
+    uint32_t* status = reinterpret_cast<uint32_t*>(scratch);
+    const uint64_t count = static_cast<uint64_t>(T) * static_cast<uint64_t>(N);
+    const uint64_t n_init = count > 0 ? count : 1;
+    gv::init_results_kernel<<<static_cast<unsigned>((n_init + 255) / 256), 256, 0, st>>>(results, count, status,
+                                                                                          nullptr);
+    GV_CUDA(cudaGetLastError());
+    if (status_out) GV_CUDA(cudaMemsetAsync(status_out, 0, sizeof(uint32_t), st));
+    if (count == 0) return GV_OK;
+
+    gv::RaggedParams p;
+    p.ref_base = static_cast<const unsigned char*>(ref_base);
+    p.ref_off = ref_off;
+    p.cand_base = static_cast<const unsigned char*>(cand_base);
+    p.cand_off = cand_off;
+    p.dtypes = dtypes;
+    p.n_elems = n_elems;
+    p.T = T;
+    p.N = N;
+    p.results = results;
+    p.status = status_out ? status_out : status;
+    p.tile_prefix = reinterpret_cast<int64_t*>(scratch + 256);
+    p.atol = static_cast<float>(tol->atol);
+    p.rtol = static_cast<float>(tol->rtol);
+    p.equal_nan = tol->equal_nan != 0;
+    gv::ragged_prepass_kernel<<<1, 1024, 0, st>>>(p);
+    GV_CUDA(cudaGetLastError());
+
+    static int blocks_per_sm[64] = {0};
+    if (blocks_per_sm[dev] == 0) {
+        GV_CUDA(cudaFuncSetAttribute(gv::ragged_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     static_cast<int>(gv::RaggedSmem::kTotal)));
+        int b = 0;
+        GV_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b, gv::ragged_kernel, gv::kThreads, gv::RaggedSmem::kTotal));
+        blocks_per_sm[dev] = b > 0 ? b : 1;
+    }
+    const unsigned grid = static_cast<unsigned>(sm_count * blocks_per_sm[dev]);
+    gv::ragged_kernel<<<grid, gv::kThreads, gv::RaggedSmem::kTotal, st>>>(p);
+    GV_CUDA(cudaGetLastError());
+    return GV_OK;
+}
+
 gv_status gv_hash(const void* buf, uint64_t nbytes, uint64_t* out, void* cuda_stream) {
     if (!out || (nbytes > 0 && !buf)) return GV_ERR_INVALID_ARG;
     if (reinterpret_cast<uintptr_t>(out) & 7u) return GV_ERR_MISALIGNED;

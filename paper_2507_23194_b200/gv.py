@@ -37,7 +37,7 @@ class gv_tol(ctypes.Structure):
                 ("equal_nan", ctypes.c_int32), ("reserved", ctypes.c_int32)]
 
 
-EXPORTS = ["gv_verify_batch", "gv_verify_ragged", "gv_hash", "gv_verify_batch_host", "gv_host_staging_bytes",
+EXPORTS = ["gv_verify_batch", "gv_verify_ragged", "gv_verify_ragged_noalloc", "gv_hash", "gv_verify_batch_host", "gv_host_staging_bytes",
            "gv_workspace_bytes", "gv_check", "gv_status_string", "gv_last_cuda_error", "gv_version"]
 
 
@@ -53,6 +53,8 @@ def _load() -> ctypes.CDLL:
     L.gv_verify_batch.argtypes = [vp, vp, i32, u64, ctypes.c_int, ctypes.POINTER(gv_tol), vp, vp, vp, sz, vp]
     L.gv_verify_ragged.restype = ctypes.c_int
     L.gv_verify_ragged.argtypes = [vp, vp, vp, vp, vp, vp, i64, i32, ctypes.POINTER(gv_tol), vp, vp, sz, vp]
+    L.gv_verify_ragged_noalloc.restype = ctypes.c_int
+    L.gv_verify_ragged_noalloc.argtypes = [vp, vp, vp, vp, vp, vp, i64, i32, ctypes.POINTER(gv_tol), vp, vp, vp]
     L.gv_hash.restype = ctypes.c_int
     L.gv_hash.argtypes = [vp, u64, vp, vp]
     L.gv_verify_batch_host.restype = ctypes.c_int
@@ -155,6 +157,30 @@ def gv_verify_ragged(ref_buf: torch.Tensor, ref_off: torch.Tensor, cand_buf: tor
                               dtypes.data_ptr(), n_elems.data_ptr() if n_elems is not None else None, T, N,
                               ctypes.byref(t), results.data_ptr(), workspace.data_ptr(), workspace.numel(),
                               _stream_ptr(stream))
+    _raise(rc)
+    return results[:T * N]
+
+
+GV_NOALLOC_MAX_TENSORS = 65536
+
+
+def gv_verify_ragged_noalloc(ref_buf: torch.Tensor, ref_off: torch.Tensor, cand_buf: torch.Tensor,
+                             cand_off: torch.Tensor, dtypes: torch.Tensor, N: int, atol: float, rtol: float,
+                             equal_nan: bool, results: torch.Tensor, n_elems: Optional[torch.Tensor] = None,
+                             status_out: Optional[torch.Tensor] = None,
+                             stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:
+    """Ragged verification for callers that cannot provide a workspace: the library's own fixed scratch
+    array is used and nothing is allocated, so ``results`` (uint8 [T*N, 64]) must be passed in, and
+    ``status_out`` (one int32 on the device) too if the status bits are wanted. At most
+    ``GV_NOALLOC_MAX_TENSORS`` tensors per call; calls that overlap on the GPU race on the shared
+    scratch. Returns ``results``."""
+    T = dtypes.numel()
+    t = _tol(atol, rtol, equal_nan)
+    rc = lib.gv_verify_ragged_noalloc(ref_buf.data_ptr(), ref_off.data_ptr(), cand_buf.data_ptr(),
+                                      cand_off.data_ptr(), dtypes.data_ptr(),
+                                      n_elems.data_ptr() if n_elems is not None else None, T, N, ctypes.byref(t),
+                                      results.data_ptr(), status_out.data_ptr() if status_out is not None else None,
+                                      _stream_ptr(stream))
     _raise(rc)
     return results[:T * N]
 

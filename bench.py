@@ -33,9 +33,25 @@ sys.path.insert(0, ROOT)
 METRIC = "GB/s of candidate outputs verified (fraction of B200 HBM peak)"
 FALLBACK_HBM_GBS = 6650.0
 
-# DRAM bytes per launch of the dominant kernel from the ncu capture summarised under profiles/
-# (dram__bytes_read.sum + dram__bytes_write.sum); None until a capture of that workload exists.
-NCU_TRAFFIC_BYTES = {}
+# DRAM bytes per launch of the dominant kernel (dram__bytes_read.sum + dram__bytes_write.sum) from the
+# ncu captures summarised under profiles/. The captures ran on a reduced number of candidates /
+# tensors of the same shapes; the figures here are scaled to the full launch in proportion to the
+# units processed (traffic is proportional to them: every candidate byte is read once, the reference
+# once per chunk of 16 candidates).
+def _scaled(measured, ref_bytes, cap_cands, full_cands):
+    """Capture on cap_cands candidates -> full launch: the candidate part scales with the number of
+    candidates, the reference part with the number of 16-candidate chunks."""
+    chunks = lambda n: (n + 15) // 16
+    per_cand = (measured - chunks(cap_cands) * ref_bytes) / cap_cands
+    return per_cand * full_cands + chunks(full_cands) * ref_bytes
+
+
+NCU_TRAFFIC_BYTES = {
+    "cfg2": _scaled(2.282e9 + 6.5e6, 33554432, 64, 256),      # profiles/dense_kernel_bf16_cfg2.md
+    "cfg3": _scaled(2.416e9 + 3.8e6, 268435456, 8, 32),       # profiles/dense_kernel_f16_cfg3.md
+    "cfg4": _scaled(2.416e9 + 8.3e6, 268435456, 8, 64),       # profiles/dense_kernel_i32_cfg4.md
+    "cfg5": (2.289e9 + 11.9e6) * 10000 / 2000,                # profiles/ragged_kernel_cfg5.md (2000 of 10000 tensors)
+}
 
 
 def measured_peak():
@@ -189,7 +205,7 @@ def dtype_name(wl) -> str:
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg2")
@@ -324,7 +340,8 @@ def main():
     algo_bytes = cand_bytes + ref_bytes + 64 * (wl.T * wl.N if ragged else n_cands)
     kernel_ms = statistics.median(step_ms)
     achieved = algo_bytes / (kernel_ms * 1e-3) / 1e9
-    roofline = {"bound": "hbm", "kernel": "ragged_kernel" if ragged else "dense_kernel",
+    roofline = {"bound": "hbm", "co_bound": "alu (integer pipes of the content hash: ceiling about 7.3 TB/s for the hash alone, see profiles/instruction_rates_b200.md)",
+                "kernel": "ragged_kernel" if ragged else "dense_kernel",
                 "achieved": achieved, "peak": peak, "peak_kind": peak_kind + " (STREAM-style copy)",
                 "unit": "GB/s", "frac": achieved / peak, "traffic": NCU_TRAFFIC_BYTES.get(args.workload),
                 "algorithmic_bytes_per_launch": algo_bytes,

@@ -50,6 +50,9 @@ __device__ __forceinline__ uint32_t smem_u32(const void* p) {
 // that work to the multiplier pipe. `two_pow` operands come from an opaque register so the
 // assembler keeps them as multiplies. Same value as the plain definition for every input
 // (checked bit for bit against the oracle).
+#ifndef GV_MAX2
+#define GV_MAX2 0
+#endif
 #ifndef GV_HASH_MASK
 #define GV_HASH_MASK 0x0
 #endif
@@ -301,12 +304,16 @@ __device__ __forceinline__ bool is_finite_bits(uint32_t b) { return (b & 0x7F800
 
 // The per-element rule, written out once, exactly as the header states it. Used for every
 // element on the general path and for the elements of vectors the fast path cannot settle.
-// GUARDED: the exact quotient is only needed when it can exceed the running maximum. Callers that
-// hold the reciprocal estimate `inv` of hoist_ref and a threshold from rel_threshold_bits pass them,
-// and the division is skipped for elements whose estimate |d| * inv cannot beat the maximum.
+// 2^-64 as binary32 bits: below this magnitude a reference element (or a running maximum) is "tiny"
+// and the cheap relative-error filter is not trusted (see rel_threshold_bits).
+constexpr uint32_t kTinyBits = 0x1F800000u;
+
+// GUARDED: the exact quotient is only needed when it can exceed the running maximum M. Callers that
+// hold a threshold from rel_threshold_bits (T <= M (1 - 2^-20), or 0 while M is tiny) pass it, and the
+// division is skipped for elements with |d| <= T |r| (sign of one fused multiply-add).
 template <bool GUARDED>
 __device__ __forceinline__ void element_rule(float c, float r, const TolF& t, uint64_t idx, Acc& a,
-                                             float inv = 0.0f, uint32_t thr_bits = 0u) {
+                                             uint32_t thr_bits = 0u) {
     const uint32_t cb = __float_as_uint(c), rb = __float_as_uint(r);
     const float d = __fsub_rn(c, r);
     const float ad = fabsf(d);
@@ -326,12 +333,11 @@ __device__ __forceinline__ void element_rule(float c, float r, const TolF& t, ui
     if (is_finite_bits(cb) && is_finite_bits(rb)) {
         const uint32_t adb = __float_as_uint(ad);          // ad >= +0, possibly +Inf by overflow
         a.maxabs = adb > a.maxabs ? adb : a.maxabs;
-        if ((rb & 0x7FFFFFFFu) != 0u) {
+        const uint32_t rab = rb & 0x7FFFFFFFu;
+        if (rab != 0u) {
             bool need = true;
-            if (GUARDED) {
-                const float q = __fmul_rn(ad, inv);
-                need = (q > __uint_as_float(thr_bits)) || (thr_bits == 0u && adb != 0u);
-            }
+            if (GUARDED && thr_bits != 0u && rab >= kTinyBits)
+                need = __fmaf_rn(-__uint_as_float(thr_bits), fabsf(r), ad) > 0.0f;
             if (need) {
                 const uint32_t qe = __float_as_uint(__fdiv_rn(ad, fabsf(r)));
                 a.maxrel = qe > a.maxrel ? qe : a.maxrel;
@@ -361,50 +367,51 @@ __device__ __forceinline__ float max2_nan(float a, float b) {
 
 // Values derived from one reference vector, computed once per tile and reused for every
 // candidate of the chunk.
-//   rf    reference widened to binary32
-//   ntol  -min(tol, FLT_MAX) with tol = fl(atol + fl(rtol*|r|)); |d| <= tolc  <=>  |d| < Inf and |d| <= tol
-//   inv   estimate of 1/|r| for the relative-error filter (hardware reciprocal) when 2^-100 <= |r| <= 2^100,
-//         0 when r == 0 (such elements have no relative error), +Inf otherwise (forces the exact path)
+//   rf      reference widened to binary32
+//   tolmin  the smallest tolc = min(tol, FLT_MAX) of the vector, tol = fl(atol + fl(rtol*|r|)):
+//           max |d| <= tolmin settles "every element is close" with one comparison
 template <int EPV>
 struct RefVec {
-    float rf[EPV], ntol[EPV], inv[EPV];
+    float rf[EPV];
+    float tolmin;
 };
 
-__device__ __forceinline__ float rcp_approx(float a) {      // one MUFU; relative error below 2^-22
-    float r;
-    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(a));
-    return r;
+// tolc of one element, as the rule defines it (two roundings, then the clamp that encodes |d| < Inf)
+__device__ __forceinline__ float tolc_of(float abs_r, const TolF& t) {
+    return fminf(__fadd_rn(t.atol, __fmul_rn(t.rtol, abs_r)), __uint_as_float(0x7F7FFFFFu));
 }
 
+// flags: bit 0 = the vector holds a NaN that does not count as equal (identical candidate vectors
+// still need the rule); bit 1 = it holds a nonzero element below 2^-64 (relative filter not trusted)
 template <int DT>
 __device__ __forceinline__ void hoist_ref(const uint4& raw, const TolF& t, RefVec<16 / Traits<DT>::ESZ>& o,
-                                          uint32_t& force) {
+                                          uint32_t& flags) {
     constexpr int EPV = 16 / Traits<DT>::ESZ;
     Widen<DT>::run(raw, o.rf);
-    uint32_t umax = 0u;
+    uint32_t umax = 0u, umin1 = 0xFFFFFFFFu;
+    float tolmin = __uint_as_float(0x7F7FFFFFu);
 #pragma unroll
     for (int e = 0; e < EPV; ++e) {
         const float a = fabsf(o.rf[e]);
         const uint32_t u = __float_as_uint(a);
-        const float tol = __fadd_rn(t.atol, __fmul_rn(t.rtol, a));
-        o.ntol[e] = -fminf(tol, __uint_as_float(0x7F7FFFFFu));      // NaN tol -> FLT_MAX; r NaN makes d NaN anyway
-        // 2^-100 <= |r| <= 2^100: reciprocal estimate; r == 0: 0; anything else (tiny, huge, Inf, NaN): +Inf
-        const bool in_range = (u - 0x0D800000u) <= (0x71800000u - 0x0D800000u);
-        o.inv[e] = in_range ? rcp_approx(a) : (u == 0u ? 0.0f : __uint_as_float(0x7F800000u));
+        tolmin = fminf(tolmin, tolc_of(a, t));                        // a NaN tol is skipped: r NaN makes d NaN anyway
         umax = u > umax ? u : umax;
+        umin1 = (u - 1u) < umin1 ? (u - 1u) : umin1;                  // u == 0 wraps to the top: ignored
     }
-    // an identical candidate vector is "all close, nothing to record" unless the reference holds a
-    // NaN that does not count as equal
-    force = (umax > 0x7F800000u && !t.equal_nan) ? 0xFFFFFFFFu : 0u;
+    o.tolmin = tolmin;
+    flags = ((umax > 0x7F800000u && !t.equal_nan) ? 1u : 0u) | ((umin1 < kTinyBits - 1u) ? 2u : 0u);
 }
 
-// Relative-error filter state of one (CTA, candidate): thr = bits of M * (1 - 2^-20) rounded down,
-// where M is the largest exact quotient recorded so far, or 0 while M < 2^-100.
-// With inv = (1/|r|)(1 + e1), |e1| < 2^-22 (hardware reciprocal estimate) and q = fl(|d| * inv) in the
-// normal range, fl(|d| / |r|) <= q * (1 + 2^-22 + 2^-23) < q * (1 + 2^-21); hence a quotient above M
-// implies q > M * (1 - 2^-21) > thr. While thr == 0 any nonzero |d| goes to the exact path.
+// Relative-error filter of one (CTA, candidate). M = largest exact quotient recorded so far;
+// T = M (1 - 2^-20) rounded down, or 0 while M < 2^-64. An element can raise M only if
+// fl(|d| / |r|) > M, which implies |d| / |r| > M (1 - 2^-24), hence |d| - T |r| > |r| M 2^-21 > 0; the
+// fused multiply-add w = fma(-T, |r|, |d|) delivers that difference correctly rounded, so w > 0
+// whenever |r| M 2^-21 is not below the subnormal range -- guaranteed for |r| >= 2^-64 and
+// M >= 2^-64. Vectors holding a nonzero |r| < 2^-64 skip the filter (flag from hoist_ref), and while
+// T == 0 every nonzero |d| passes (w = |d|). When T |r| overflows, |d| / |r| < M and nothing is missed.
+// Elements with r == 0 pass the filter whenever |d| != 0 and are dropped afterwards (no relative error).
 __device__ __forceinline__ uint32_t rel_threshold_bits(uint32_t m_bits) {
-    if (m_bits < 0x0D800000u) return 0u;                                  // M < 2^-100 (or 0)
+    if (m_bits < kTinyBits) return 0u;
     if (m_bits >= 0x7F800000u) return 0x7F800000u;                        // M = +Inf: nothing can exceed it
     return __float_as_uint(__fmul_rd(__uint_as_float(m_bits), __uint_as_float(0x3F7FFFF0u)));   // 1 - 2^-20
 }
@@ -424,10 +431,22 @@ __device__ __forceinline__ void raise_maxrel(CtaAcc* s, uint32_t bits) {
     }
 }
 
-// IEEE quotient for the (rare) elements whose estimate beats the filter; out of line to keep the
-// hot loop small.
-__device__ __noinline__ uint32_t exact_quotient_bits(float ad, float abs_r) {
-    return __float_as_uint(__fdiv_rn(ad, abs_r));
+// One element that passed the relative-error filter (out of line: the hot loop only tests and calls).
+// First decides exactly, without dividing, whether the real quotient |d| / |r| exceeds M:
+// |d| > M |r|  <=>  |d| - p > e  with p = fl(M |r|) and e = M |r| - p, the exact rounding error of the
+// product, delivered by one fused multiply-add. Elements that only tie with M -- the norm in
+// quantised data -- stop there: rounding is monotone, so a real quotient <= M cannot round above M.
+// Returns the bits of the IEEE quotient, or 0 when it cannot raise M. thr_bits == 0: M unknown/tiny.
+__device__ __noinline__ uint32_t rel_candidate_bits(float ad, float ar, float M, uint32_t thr_bits) {
+    if (ar == 0.0f) return 0u;                              // r == 0: no relative error
+    if (thr_bits != 0u) {
+        const float pm = __fmul_rn(M, ar);
+        if (__float_as_uint(pm) >= 0x0D800000u && __float_as_uint(pm) < 0x7F800000u) {   // 2^-100 <= p < Inf: e is exact
+            const float err = __fmaf_rn(M, ar, -pm);
+            if (!(__fsub_rn(ad, pm) > err)) return 0u;
+        }
+    }
+    return __float_as_uint(__fdiv_rn(ad, ar));
 }
 
 // Compare one full vector on the fast path. Returns true when the vector is settled here: every pair
@@ -437,76 +456,60 @@ __device__ __noinline__ uint32_t exact_quotient_bits(float ad, float abs_r) {
 // error go to the CTA accumulators. Returns false when a NaN or an infinity is involved: the caller
 // then runs the exact per-element rule on this vector (nothing has been recorded in that case).
 template <int DT>
-__device__ __forceinline__ bool vec_fast_float(const uint4& c, const RefVec<16 / Traits<DT>::ESZ>& r, CtaAcc* s,
-                                               uint64_t elem0) {
+__device__ __forceinline__ bool vec_fast_float(const uint4& c, const RefVec<16 / Traits<DT>::ESZ>& r, uint32_t flags,
+                                               const TolF& t, CtaAcc* s, uint64_t elem0) {
     constexpr int EPV = 16 / Traits<DT>::ESZ;
-    float cf[EPV], ad[EPV], m[EPV], q[EPV];
+    // running maxima of this (CTA, candidate): max|d| bits, max relative error bits, filter threshold
+    const uint4 run = lds128(smem_u32(&s->maxabs));
+    const float nT = -__uint_as_float(run.z);
+    float cf[EPV], ad[EPV], w[EPV];
     Widen<DT>::run(c, cf);
 #pragma unroll
     for (int e = 0; e < EPV; ++e) {
         ad[e] = fabsf(__fsub_rn(cf[e], r.rf[e]));
-        m[e] = __fadd_rn(ad[e], r.ntol[e]);          // > 0 or NaN  <=>  not (|d| <= tolc)
-        q[e] = __fmul_rn(ad[e], r.inv[e]);           // NaN only from 0 * Inf, ignored by max
+        w[e] = __fmaf_rn(nT, fabsf(r.rf[e]), ad[e]);         // > 0  <=  the quotient could exceed M
     }
-    float vm, va, vq;
+    float va, vw;       // va propagates NaN: a NaN anywhere (candidate or reference) must not be skipped
     if (EPV == 8) {
-        vm = max2_nan(max3_nan(m[0], m[1], m[2]), max3_nan(max3_nan(m[3], m[4], m[5]), m[6], m[7]));
-        va = fmaxf(max3(ad[0], ad[1], ad[2]), max3(max3(ad[3], ad[4], ad[5]), ad[6], ad[7]));
-        vq = fmaxf(max3(q[0], q[1], q[2]), max3(max3(q[3], q[4], q[5]), q[6], q[7]));
+        va = max2_nan(max3_nan(ad[0], ad[1], ad[2]), max3_nan(max3_nan(ad[3], ad[4], ad[5]), ad[6], ad[7]));
+        vw = fmaxf(max3(w[0], w[1], w[2]), max3(max3(w[3], w[4], w[5]), w[6], w[7]));
     } else {
-        vm = max2_nan(max3_nan(m[0], m[1], m[2]), m[3]);
-        va = fmaxf(max3(ad[0], ad[1], ad[2]), ad[3]);
-        vq = fmaxf(max3(q[0], q[1], q[2]), q[3]);
+        va = max2_nan(max3_nan(ad[0], ad[1], ad[2]), ad[3]);
+        vw = fmaxf(max3(w[0], w[1], w[2]), w[3]);
     }
     const uint32_t vab = __float_as_uint(va);
-    if (!(vm <= 0.0f)) {
-        // some element is not close, or a NaN is present (vm propagates NaN)
-        if (vm != vm || vab >= 0x7F800000u) return false;
+    if (!(va <= r.tolmin)) {
+        // Some |d| exceeds the smallest tolerance of the vector, or a NaN is present. NaN or Inf:
+        // the caller runs the exact rule. Otherwise every pair is finite and an element is close
+        // exactly when |d| <= its own tolc.
+        if (va != va || vab >= 0x7F800000u) return false;
         uint32_t cnt = 0u;
         int first_e = EPV;
 #pragma unroll
         for (int e = EPV - 1; e >= 0; --e) {
-            if (m[e] > 0.0f) { cnt += 1u; first_e = e; }
+            if (ad[e] > tolc_of(fabsf(r.rf[e]), t)) { cnt += 1u; first_e = e; }
         }
-        GV_COUNT(3);
-        // lanes of the warp that are here add their counts with one shared-memory atomic
-        const unsigned active = __activemask();
-        const uint32_t total = __reduce_add_sync(active, cnt);
-        if ((threadIdx.x & 31) == __ffs(active) - 1) atomicAdd(&s->cnt, static_cast<unsigned long long>(total));
-        const unsigned long long idx = elem0 + first_e;
-        if (idx < *reinterpret_cast<volatile unsigned long long*>(&s->first)) atomicMin(&s->first, idx);
+        if (cnt) {
+            GV_COUNT(3);
+            // lanes of the warp that are here add their counts with one shared-memory atomic
+            const unsigned active = __activemask();
+            const uint32_t total = __reduce_add_sync(active, cnt);
+            if ((threadIdx.x & 31) == __ffs(active) - 1) atomicAdd(&s->cnt, static_cast<unsigned long long>(total));
+            const unsigned long long idx = elem0 + first_e;
+            if (idx < *reinterpret_cast<volatile unsigned long long*>(&s->first)) atomicMin(&s->first, idx);
+        }
     }
-    // running maxima of this (CTA, candidate): max|d| bits, max relative error bits, filter threshold
-    const uint4 run = lds128(smem_u32(&s->maxabs));
     if (vab > run.x) raise_maxabs(s, vab);
-    const uint32_t thr_bits = run.z;
-    if ((vq > __uint_as_float(thr_bits)) || (thr_bits == 0u && vab != 0u)) {
-        // Some element may raise the relative maximum M. For each element that passes the filter,
-        // first decide exactly whether the real quotient |d| / |r| exceeds M without dividing:
-        // |d| > M |r|  <=>  |d| - p > e  with p = fl(M |r|) and e = M |r| - p (the exact rounding error,
-        // delivered by one fused multiply-add). Elements that only tie with M -- common in quantised
-        // data -- stop here; rounding is monotone, so a real quotient <= M cannot round above M.
+    if (vw > 0.0f || ((flags & 2u) && vab != 0u)) {
+        // some element may raise the relative maximum M: each one that passes the filter is examined
         GV_COUNT(2);
         const float M = __uint_as_float(run.y);
         uint32_t best = 0u;
 #pragma unroll
         for (int e = 0; e < EPV; ++e) {
-            const bool need = (q[e] > __uint_as_float(thr_bits)) || (thr_bits == 0u && ad[e] != 0.0f);
-            // r.inv == 0 marks r == 0 (no relative error); q is then 0 or NaN and ad may be nonzero
-            if (need && r.inv[e] != 0.0f) {
-                const float ar = fabsf(r.rf[e]);
-                bool beats = true;
-                if (thr_bits != 0u) {
-                    const float pm = __fmul_rn(M, ar);
-                    if (__float_as_uint(pm) >= 0x0D800000u && __float_as_uint(pm) < 0x7F800000u) {   // 2^-100 <= p < Inf: e is exact
-                        const float err = __fmaf_rn(M, ar, -pm);
-                        beats = __fsub_rn(ad[e], pm) > err;
-                    }
-                }
-                if (beats) {
-                    const uint32_t qe = exact_quotient_bits(ad[e], ar);
-                    best = qe > best ? qe : best;
-                }
+            if ((w[e] > 0.0f) || ((flags & 2u) && ad[e] != 0.0f)) {
+                const uint32_t qe = rel_candidate_bits(ad[e], fabsf(r.rf[e]), M, run.z);
+                best = qe > best ? qe : best;
             }
         }
         if (best > run.y) raise_maxrel(s, best);
@@ -523,7 +526,7 @@ __device__ __forceinline__ void vec_exact_float(const uint4& c, const RefVec<16 
     float cf[EPV];
     Widen<DT>::run(c, cf);
 #pragma unroll
-    for (int e = 0; e < EPV; ++e) element_rule<true>(cf[e], r.rf[e], t, elem0 + e, a, r.inv[e], thr_bits);
+    for (int e = 0; e < EPV; ++e) element_rule<true>(cf[e], r.rf[e], t, elem0 + e, a, thr_bits);
 }
 
 // One 16-byte vector of a float dtype, general path: every element through the rule.

@@ -112,14 +112,25 @@ constexpr int kWarps = kThreads / 32;
 constexpr int kRing = GV_RING;            // asynchronous copies in flight per lane (power of two)
 constexpr int kWarpTile = 512;            // bytes of one warp-tile
 
+template <int WARPS>
 struct DenseSmem {
     static constexpr size_t kRingOff = 0;                                                 // [warp][kRing][32] uint4
-    static constexpr size_t kRefOff = kRingOff + size_t(kWarps) * kRing * kWarpTile;      // [warp][2][32] uint4
-    static constexpr size_t kSlotOff = kRefOff + size_t(kWarps) * 2 * kWarpTile;          // [warp][kChunk][32] u64
-    static constexpr size_t kAccOff = kSlotOff + size_t(kWarps) * kChunk * 32 * 8;        // CtaAcc[kChunk]
+    static constexpr size_t kRefOff = kRingOff + size_t(WARPS) * kRing * kWarpTile;       // [warp][2][32] uint4
+    static constexpr size_t kSlotOff = kRefOff + size_t(WARPS) * 2 * kWarpTile;           // [warp][kChunk][32] u64
+    static constexpr size_t kAccOff = kSlotOff + size_t(WARPS) * kChunk * 32 * 8;         // CtaAcc[kChunk]
     static constexpr size_t kBarOff = kAccOff + sizeof(CtaAcc) * kChunk;                  // [warp][2] mbarrier
-    static constexpr size_t kRefHashOff = kBarOff + size_t(kWarps) * 2 * 8;
+    static constexpr size_t kRefHashOff = kBarOff + size_t(WARPS) * 2 * 8;
     static constexpr size_t kTotal = kRefHashOff + 8;
+};
+
+// CTA shapes: integer kernels need ~72 registers and run 3 CTAs of 8 warps per SM; float kernels hold
+// the derived reference values as well and run 2 CTAs of GV_FLOAT_WARPS warps within the register file.
+#ifndef GV_FLOAT_WARPS
+#define GV_FLOAT_WARPS 8
+#endif
+template <int DT> struct DenseShape {
+    static constexpr int kWarpsPerCta = Traits<DT>::IS_FLOAT ? GV_FLOAT_WARPS : 8;
+    static constexpr int kCtasPerSm = Traits<DT>::IS_FLOAT ? GV_MINB_FLOAT : 3;
 };
 
 // The exact rule for one vector the fast path could not settle; kept out of line so the hot loop
@@ -146,18 +157,21 @@ __device__ __noinline__ void settle_vector_int(uint4 c, uint4 r, uint64_t elem0,
 
 // BIGK: word indices of the hash need more than 32 bits (tensors of 32 GiB and more).
 template <int DT, bool BIGK>
-__global__ void __launch_bounds__(kThreads, Traits<DT>::IS_FLOAT ? GV_MINB_FLOAT : 3) dense_kernel(const __grid_constant__ DenseParams p) {
+__global__ void __launch_bounds__(DenseShape<DT>::kWarpsPerCta * 32, DenseShape<DT>::kCtasPerSm)
+dense_kernel(const __grid_constant__ DenseParams p) {
+    constexpr int kWarps = DenseShape<DT>::kWarpsPerCta;      // (shadows the 8-warp default of the other kernels)
+    using Smem = DenseSmem<kWarps>;
     constexpr int ESZ = Traits<DT>::ESZ;
     constexpr int EPV = 16 / ESZ;
     constexpr bool IS_FLOAT = Traits<DT>::IS_FLOAT;
     extern __shared__ __align__(128) unsigned char smem[];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    CtaAcc* cacc = reinterpret_cast<CtaAcc*>(smem + DenseSmem::kAccOff);
-    unsigned long long* s_refhash = reinterpret_cast<unsigned long long*>(smem + DenseSmem::kRefHashOff);
-    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + DenseSmem::kBarOff) + warp * 2;
-    unsigned char* ref_stage = smem + DenseSmem::kRefOff + size_t(warp) * 2 * kWarpTile;
-    uint2* slots = reinterpret_cast<uint2*>(smem + DenseSmem::kSlotOff) + size_t(warp) * kChunk * 32 + lane;
-    const uint32_t ring_base = smem_u32(smem + DenseSmem::kRingOff) + (warp * kRing * 32 + lane) * 16;
+    CtaAcc* cacc = reinterpret_cast<CtaAcc*>(smem + Smem::kAccOff);
+    unsigned long long* s_refhash = reinterpret_cast<unsigned long long*>(smem + Smem::kRefHashOff);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + Smem::kBarOff) + warp * 2;
+    unsigned char* ref_stage = smem + Smem::kRefOff + size_t(warp) * 2 * kWarpTile;
+    uint2* slots = reinterpret_cast<uint2*>(smem + Smem::kSlotOff) + size_t(warp) * kChunk * 32 + lane;
+    const uint32_t ring_base = smem_u32(smem + Smem::kRingOff) + (warp * kRing * 32 + lane) * 16;
 
     const uint64_t nbytes = p.n * ESZ;
     const uint64_t full_tiles = p.all_aligned ? nbytes / kWarpTile : 0;      // tiles the fast loop takes
@@ -196,8 +210,8 @@ __global__ void __launch_bounds__(kThreads, Traits<DT>::IS_FLOAT ? GV_MINB_FLOAT
             // Values derived from the reference vector, computed lazily: only when a candidate
             // vector differs from it (exact copies never pay for them).
             RefVec<IS_FLOAT ? EPV : 1> rv;
-            uint32_t force = 0u;
-            bool hoisted = false;
+            uint32_t force = 0u, rflags = 0u;
+            bool hoisted = false, tile_forced = false;
             auto new_tile = [&](const uint4& r) {
                 hoisted = false;
                 force = 0u;
@@ -221,13 +235,14 @@ __global__ void __launch_bounds__(kThreads, Traits<DT>::IS_FLOAT ? GV_MINB_FLOAT
                         force = any_nan ? 0xFFFFFFFFu : 0u;
                     }
                 }
+                // warp-uniform: does any lane hold such a vector? (keeps the per-lane flag out of the hot path)
+                tile_forced = __any_sync(0xFFFFFFFFu, force != 0u);
             };
             // Derive the per-tile values when some lane of the warp first needs them. The decision is
             // warp-uniform (a vote), so the derivation runs once per tile, not once per diverged lane.
             auto ensure_hoisted = [&](const uint4& r) {
                 if (!hoisted) {
-                    uint32_t f2;
-                    if constexpr (IS_FLOAT) hoist_ref<DT>(r, tol, rv, f2);
+                    if constexpr (IS_FLOAT) hoist_ref<DT>(r, tol, rv, rflags);
                     hoisted = true;
                 }
             };
@@ -236,7 +251,7 @@ __global__ void __launch_bounds__(kThreads, Traits<DT>::IS_FLOAT ? GV_MINB_FLOAT
                 if constexpr (!IS_FLOAT) {
                     settle_vector_int<DT>(c, r, voff / ESZ, &cacc[k]);
                 } else {
-                    if (!vec_fast_float<DT>(c, rv, &cacc[k], voff / ESZ)) settle_vector_exact<DT>(c, rv, voff / ESZ, tol, &cacc[k]);
+                    if (!vec_fast_float<DT>(c, rv, rflags, tol, &cacc[k], voff / ESZ)) settle_vector_exact<DT>(c, rv, voff / ESZ, tol, &cacc[k]);
                 }
             };
             // one visit: candidate vector c (already read from the ring) against the held reference
@@ -247,10 +262,10 @@ __global__ void __launch_bounds__(kThreads, Traits<DT>::IS_FLOAT ? GV_MINB_FLOAT
                 const uint2 sl = slots[k * 32];
                 h += pack64(sl.x, sl.y);
                 slots[k * 32] = make_uint2(static_cast<uint32_t>(h), static_cast<uint32_t>(h >> 32));
-                const bool differs = (c.x != r.x) || (c.y != r.y) || (c.z != r.z) || (c.w != r.w) || (force != 0u);
-                if (__any_sync(0xFFFFFFFFu, differs)) {
+                const bool differs = (c.x != r.x) || (c.y != r.y) || (c.z != r.z) || (c.w != r.w);
+                if (__any_sync(0xFFFFFFFFu, differs) || tile_forced) {
                     ensure_hoisted(r);
-                    if (differs) differing(c, r, k);
+                    if (differs || force != 0u) differing(c, r, k);
                 }
             };
             // reference of tile i: wait for its bulk copy, take this lane's vector, start the next copy
@@ -316,9 +331,9 @@ __global__ void __launch_bounds__(kThreads, Traits<DT>::IS_FLOAT ? GV_MINB_FLOAT
                             const bool differs = (c[u].x != r.x) || (c[u].y != r.y) || (c[u].z != r.z) || (c[u].w != r.w);
                             diffmask |= differs ? (1u << u) : 0u;
                         }
-                        diffmask |= force;      // force is 0 or all ones
-                        if (__any_sync(0xFFFFFFFFu, diffmask != 0u)) {
+                        if (__any_sync(0xFFFFFFFFu, diffmask != 0u) || tile_forced) {
                             ensure_hoisted(r);
+                            diffmask |= force;      // force is 0 or all ones
 #pragma unroll
                             for (int u = 0; u < U; ++u) {
                                 if (diffmask & (1u << u)) differing(c[u], r, k0 + u);
@@ -513,7 +528,8 @@ __global__ void __launch_bounds__(1024) ragged_prepass_kernel(RaggedParams p) {
 // statistics in per-warp shared accumulators, all flushed with integer atomics when the warp leaves
 // the tensor. No barrier is used anywhere: warps never share a tensor's accumulators.
 struct RaggedSmem {
-    static constexpr size_t kSlotOff = 0;                                                  // [warp][kChunk][32] u64
+    static constexpr size_t kRingOff = 0;                                                  // [warp][kRing][32] uint4
+    static constexpr size_t kSlotOff = kRingOff + size_t(kWarps) * kRing * kWarpTile;      // [warp][kChunk][32] u64
     static constexpr size_t kAccOff = kSlotOff + size_t(kWarps) * kChunk * 32 * 8;         // [warp][kChunk] CtaAcc
     static constexpr size_t kPtrOff = kAccOff + size_t(kWarps) * kChunk * sizeof(CtaAcc);  // [warp][kChunk] candidate pointers
     static constexpr size_t kTotal = kPtrOff + size_t(kWarps) * kChunk * 8;
@@ -530,7 +546,7 @@ __device__ __forceinline__ void ragged_differing_t(const uint4& c, const uint4& 
         RefVec<16 / Traits<DT>::ESZ> rv;
         uint32_t force;
         hoist_ref<DT>(r, tol, rv, force);
-        if (!vec_fast_float<DT>(c, rv, s, elem0)) {
+        if (!vec_fast_float<DT>(c, rv, force, tol, s, elem0)) {
             Acc a;
             a.clear();
             const uint32_t thr = *reinterpret_cast<volatile unsigned int*>(&s->thr);
@@ -601,54 +617,86 @@ __device__ __forceinline__ bool vec_has_nan(int dt, const uint4& r) {
 }
 
 // Tiles [tile_begin, tile_end) of one tensor against kg of its candidates (pointers in wptr).
+// Full tiles with 16-byte aligned bases are streamed through the lane's asynchronous-copy ring
+// (reference vector first, then the kg candidate vectors of the tile, kRing copies in flight), so
+// the loads of the next tile or two fly while the current one is compared. The ragged tail tile and
+// unaligned tensors use synchronous element-sized loads.
 __device__ __forceinline__ void ragged_stretch(const RaggedParams& p, int dt, const unsigned char* ref, uint64_t n,
                                                uint64_t tile_begin, uint64_t tile_end, int kg, uint2* slots,
-                                               CtaAcc* wacc, const unsigned char* const* wptr, int lane) {
-    constexpr int KC = 4;                           // candidates loaded together
+                                               CtaAcc* wacc, const unsigned char* const* wptr, int lane,
+                                               uint32_t ring_base) {
     const int esz = elem_size(dt);
     const uint64_t nbytes = n * esz;
     const TolF tol = {p.atol, p.rtol, p.equal_nan};
-    const bool ref_al = (reinterpret_cast<uintptr_t>(ref) & 15u) == 0;
     const bool nan_matters = (dt <= GV_F16) && !p.equal_nan;
+    bool aligned = (reinterpret_cast<uintptr_t>(ref) & 15u) == 0;
+    for (int k = 0; k < kg; ++k) aligned = aligned && (reinterpret_cast<uintptr_t>(wptr[k]) & 15u) == 0;
+    const uint64_t full_end_all = nbytes / kWarpTile;                  // tiles [0, full_end_all) are full
+    const uint64_t full_end = aligned ? (tile_end < full_end_all ? tile_end : full_end_all) : tile_begin;
+
+    auto one_visit = [&](const uint4& c, const uint4& r, bool force, uint64_t voff, int k) {
+        uint64_t h = hash_vec_full(c, voff / 8);
+        const uint2 sl = slots[k * 32];
+        h += pack64(sl.x, sl.y);
+        slots[k * 32] = make_uint2(static_cast<uint32_t>(h), static_cast<uint32_t>(h >> 32));
+        const bool differs = (c.x != r.x) || (c.y != r.y) || (c.z != r.z) || (c.w != r.w) || force;
+        if (differs) ragged_differing(dt, c, r, voff, tol, &wacc[k]);
+    };
+
+    if (full_end > tile_begin) {
+        // ---- streamed part ----
+        const uint32_t per_tile = static_cast<uint32_t>(kg) + 1u;       // reference + candidates
+        uint64_t issue_tile = tile_begin;
+        int issue_j = -1;                                               // -1: reference, else candidate index
+        uint32_t issue_stage = 0;
+        auto issue_one = [&]() {
+            if (issue_tile < full_end) {
+                const unsigned char* base = issue_j < 0 ? ref : wptr[issue_j];
+                cp_async16(ring_base + issue_stage * 512u, base + issue_tile * kWarpTile + lane * 16);
+                issue_stage = (issue_stage + 1u) & (kRing - 1);
+                if (++issue_j == kg) { issue_j = -1; ++issue_tile; }
+            }
+            cp_async_commit();
+        };
+        (void)per_tile;
 #pragma unroll 1
-    for (uint64_t tile = tile_begin; tile < tile_end; ++tile) {
+        for (int j = 0; j < kRing; ++j) issue_one();
+        uint32_t stage = 0;
+#pragma unroll 1
+        for (uint64_t tile = tile_begin; tile < full_end; ++tile) {
+            const uint64_t voff = tile * kWarpTile + lane * 16;
+            cp_async_wait<kRing - 1>();
+            const uint4 r = lds128(ring_base + stage * 512u);
+            stage = (stage + 1u) & (kRing - 1);
+            issue_one();
+            const bool force = nan_matters && vec_has_nan(dt, r);
+#pragma unroll 1
+            for (int k = 0; k < kg; ++k) {
+                cp_async_wait<kRing - 1>();
+                const uint4 c = lds128(ring_base + stage * 512u);
+                stage = (stage + 1u) & (kRing - 1);
+                issue_one();
+                one_visit(c, r, force, voff, k);
+            }
+        }
+        cp_async_wait<0>();
+    }
+
+    // ---- synchronous part: the tail tile, or every tile of an unaligned tensor ----
+#pragma unroll 1
+    for (uint64_t tile = full_end; tile < tile_end; ++tile) {
         const uint64_t voff = tile * kWarpTile + lane * 16;
         const uint64_t rem = voff < nbytes ? nbytes - voff : 0;
         const int nvalid = rem >= 16 ? 16 / esz : static_cast<int>(rem / esz);
+        if (nvalid <= 0) continue;
         const bool full = rem >= 16;
-        uint4 r = make_uint4(0u, 0u, 0u, 0u);
-        if (full && ref_al) r = ldg_stream(ref + voff);
-        else if (nvalid > 0) r = load_vec_any(esz, ref, voff, nbytes);
-        // an identical vector still needs the rule when the reference holds a NaN that is not "equal"
+        const uint4 r = load_vec_any(esz, ref, voff, nbytes);
         const bool force = nan_matters && full && vec_has_nan(dt, r);
 #pragma unroll 1
-        for (int k0 = 0; k0 < kg; k0 += KC) {
-            uint4 c[KC];
-#pragma unroll
-            for (int u = 0; u < KC; ++u) {
-                c[u] = make_uint4(0u, 0u, 0u, 0u);
-                if (k0 + u < kg) {
-                    const unsigned char* cp = wptr[k0 + u];
-                    if (full && (reinterpret_cast<uintptr_t>(cp) & 15u) == 0) c[u] = ldg_stream(cp + voff);
-                    else if (nvalid > 0) c[u] = load_vec_any(esz, cp, voff, nbytes);
-                }
-            }
-#pragma unroll
-            for (int u = 0; u < KC; ++u) {
-                const int k = k0 + u;
-                if (k < kg) {
-                    if (full) {
-                        uint64_t h = hash_vec_full(c[u], voff / 8);
-                        const uint2 sl = slots[k * 32];
-                        h += pack64(sl.x, sl.y);
-                        slots[k * 32] = make_uint2(static_cast<uint32_t>(h), static_cast<uint32_t>(h >> 32));
-                        const bool differs = (c[u].x != r.x) || (c[u].y != r.y) || (c[u].z != r.z) || (c[u].w != r.w) || force;
-                        if (differs) ragged_differing(dt, c[u], r, voff, tol, &wacc[k]);
-                    } else if (nvalid > 0) {
-                        ragged_partial(dt, c[u], r, voff, nvalid, tol, &wacc[k], &slots[k * 32]);
-                    }
-                }
-            }
+        for (int k = 0; k < kg; ++k) {
+            const uint4 c = load_vec_any(esz, wptr[k], voff, nbytes);
+            if (full) one_visit(c, r, force, voff, k);
+            else ragged_partial(dt, c, r, voff, nvalid, tol, &wacc[k], &slots[k * 32]);
         }
     }
 }
@@ -659,6 +707,7 @@ __global__ void __launch_bounds__(kThreads, 2) ragged_kernel(const __grid_consta
     uint2* slots = reinterpret_cast<uint2*>(smem + RaggedSmem::kSlotOff) + size_t(warp) * kChunk * 32 + lane;
     CtaAcc* wacc = reinterpret_cast<CtaAcc*>(smem + RaggedSmem::kAccOff) + warp * kChunk;
     const unsigned char** wptr = reinterpret_cast<const unsigned char**>(smem + RaggedSmem::kPtrOff) + warp * kChunk;
+    const uint32_t ring_base = smem_u32(smem + RaggedSmem::kRingOff) + (warp * kRing * 32 + lane) * 16;
 
     const uint64_t total = static_cast<uint64_t>(p.tile_prefix[p.T]);
     const uint64_t gw = static_cast<uint64_t>(blockIdx.x) * kWarps + warp;
@@ -697,7 +746,7 @@ __global__ void __launch_bounds__(kThreads, 2) ragged_kernel(const __grid_consta
             }
             for (int k = 0; k < kg; ++k) slots[k * 32] = make_uint2(0u, 0u);
             __syncwarp();
-            ragged_stretch(p, dt, ref, n, tile_begin, tile_end, kg, slots, wacc, wptr, lane);
+            ragged_stretch(p, dt, ref, n, tile_begin, tile_end, kg, slots, wacc, wptr, lane, ring_base);
             __syncwarp();
             // leave the tensor (or this group of its candidates): combine and publish
             for (int k = 0; k < kg; ++k) {
@@ -758,7 +807,8 @@ bool tol_valid(const gv_tol* t) {
 
 template <int DT, bool BIGK>
 gv_status launch_dense_t(const gv::DenseParams& p, int sm_count, cudaStream_t st) {
-    using S = gv::DenseSmem;
+    constexpr int kWarpsCta = gv::DenseShape<DT>::kWarpsPerCta;
+    using S = gv::DenseSmem<kWarpsCta>;
     static int blocks_per_sm[64] = {0};
     int dev = 0;
     GV_CUDA(cudaGetDevice(&dev));
@@ -766,16 +816,16 @@ gv_status launch_dense_t(const gv::DenseParams& p, int sm_count, cudaStream_t st
     if (blocks_per_sm[dev] == 0) {
         GV_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(S::kTotal)));
         int b = 0;
-        GV_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b, kern, gv::kThreads, S::kTotal));
+        GV_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b, kern, kWarpsCta * 32, S::kTotal));
         blocks_per_sm[dev] = b > 0 ? b : 1;
     }
     const uint64_t nbytes = p.n * gv::Traits<DT>::ESZ;
-    const uint64_t cta_tile = static_cast<uint64_t>(gv::kWarps) * gv::kWarpTile;
+    const uint64_t cta_tile = static_cast<uint64_t>(kWarpsCta) * gv::kWarpTile;
     const uint64_t tiles = (nbytes + cta_tile - 1) / cta_tile;
     uint64_t grid = static_cast<uint64_t>(sm_count) * blocks_per_sm[dev];
     if (grid > tiles) grid = tiles;
     if (grid == 0) return GV_OK;
-    kern<<<static_cast<unsigned>(grid), gv::kThreads, S::kTotal, st>>>(p);
+    kern<<<static_cast<unsigned>(grid), kWarpsCta * 32, S::kTotal, st>>>(p);
     GV_CUDA(cudaGetLastError());
     return GV_OK;
 }

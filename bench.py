@@ -212,6 +212,8 @@ def main():
     ap.add_argument("--cands", type=int, default=0, help="fewer candidates than the recipe (profiling captures)")
     ap.add_argument("--tensors", type=int, default=0, help="fewer ragged tensors than the recipe (profiling captures)")
     ap.add_argument("--only-class", default="", help="keep only candidates of this recipe class (dense workloads)")
+    ap.add_argument("--as-int32", action="store_true",
+                    help="verify the same bytes in exact integer mode (tensors viewed as int32)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
@@ -243,6 +245,11 @@ def main():
         wl.cands = [wl.cands[j] for j in keep]
         wl.facts = [wl.facts[j] for j in keep]
         wl.name += ":" + args.only_class
+    if args.as_int32 and not ragged:
+        wl.ref = wl.ref.view(torch.int32)
+        wl.cands = [c.view(torch.int32) for c in wl.cands]
+        wl.dtype = W.GV_I32
+        wl.name += ":as_int32"
 
     stream = torch.cuda.current_stream()
     if ragged:

@@ -491,10 +491,10 @@ __device__ __forceinline__ bool vec_fast_float(const uint4& c, const RefVec<16 /
         }
         if (cnt) {
             GV_COUNT(3);
-            // lanes of the warp that are here add their counts with one shared-memory atomic
-            const unsigned active = __activemask();
-            const uint32_t total = __reduce_add_sync(active, cnt);
-            if ((threadIdx.x & 31) == __ffs(active) - 1) atomicAdd(&s->cnt, static_cast<unsigned long long>(total));
+            // one shared-memory atomic per lane that found mismatches. (Aggregating over the lanes
+            // that happen to be here would need their exact set; the mask of active threads is not a
+            // reliable source for it once the compiler moves the query, and a wrong set drops counts.)
+            atomicAdd(&s->cnt, static_cast<unsigned long long>(cnt));
             const unsigned long long idx = elem0 + first_e;
             if (idx < *reinterpret_cast<volatile unsigned long long*>(&s->first)) atomicMin(&s->first, idx);
         }

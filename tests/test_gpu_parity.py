@@ -340,3 +340,142 @@ def test_verify_batch_host(oracle):
         want = oracle.verify_batch(host_bytes(r), [host_bytes(c) for c in cands], 1, 1e-2, 1e-2, True)
         assert_records_equal(got, want, f"host entry slab {slab}")
         assert rh == oracle.hash_bytes(host_bytes(r))
+
+
+# ------------------------------------------------------------------------------------------------
+# randomised sweep: dtype x size x alignment x candidate count x tolerances x value patterns
+# ------------------------------------------------------------------------------------------------
+def _rand_values(rng, code, n):
+    """Reference values with a seeded mixture of scales and special values."""
+    if code in (3, 4):
+        info = np.iinfo(np.int32 if code == 3 else np.int64)
+        kind = rng.integers(0, 3)
+        if kind == 0:
+            a = rng.integers(-100, 100, n)
+        elif kind == 1:
+            a = rng.integers(info.min, info.max, n, dtype=np.int64, endpoint=False)
+        else:
+            a = rng.choice(np.array([0, 1, -1, info.min, info.max]), n)
+        return torch.from_numpy(a.astype(np.int32 if code == 3 else np.int64))
+    scale = float(10.0 ** rng.integers(-8, 6))
+    a = (rng.standard_normal(n) * scale).astype(np.float32)
+    if n and rng.random() < 0.7:
+        k = max(1, n // 50)
+        pos = rng.integers(0, n, k)
+        a[pos] = rng.choice(np.array([0.0, -0.0, np.inf, -np.inf, np.nan, 1e-40, -1e-45, 3e38, 65504.0, 1.0],
+                                     dtype=np.float32), k)
+    return torch.from_numpy(a).to(TDT[code])
+
+
+def _rand_candidate(rng, code, r):
+    n = r.numel()
+    kind = rng.integers(0, 7)
+    if code in (3, 4):
+        c = r.clone()
+        if kind >= 2 and n:
+            k = max(1, int(n * float(rng.choice([1e-3, 0.05, 1.0]))))
+            pos = torch.from_numpy(rng.integers(0, n, k))
+            c[pos] = _rand_values(rng, code, k)
+        return c
+    rf = r.float()
+    if kind == 0 or n == 0:
+        return r.clone()
+    if kind == 1:
+        return (rf * (1 + float(10.0 ** rng.integers(-7, -1)) * torch.from_numpy(rng.standard_normal(n).astype(np.float32)))).to(TDT[code])
+    if kind == 2:
+        return (rf + float(10.0 ** rng.integers(-9, 2)) * torch.from_numpy(rng.standard_normal(n).astype(np.float32))).to(TDT[code])
+    if kind == 3:
+        return torch.zeros_like(r)
+    if kind == 4:
+        return _rand_values(rng, code, n)
+    c = r.clone()
+    k = max(1, n // int(rng.choice([3, 30, 300])))
+    pos = torch.from_numpy(rng.integers(0, n, k))
+    c[pos] = _rand_values(rng, code, k)
+    return c
+
+
+@pytest.mark.parametrize("seed", range(12))
+def test_randomised_sweep(oracle, seed):
+    rng = np.random.default_rng(1000 + seed)
+    for _ in range(30):
+        code = int(rng.integers(0, 5))
+        n = int(rng.choice([0, 1, 5, 33, 127, 128, 129, 1000, 4099, 8192 + 3, 40000, 100003]))
+        n_cands = int(rng.choice([1, 2, 5, 16, 17, 31]))
+        shift_r = int(rng.integers(0, 3)) if rng.random() < 0.3 else 0
+        r_full = _rand_values(rng, code, n + 4)
+        r = r_full[shift_r:shift_r + n]
+        cands = []
+        for j in range(n_cands):
+            c_full = torch.zeros(n + 4, dtype=TDT[code])
+            sh = int(rng.integers(0, 3)) if rng.random() < 0.2 else 0
+            c_full[sh:sh + n] = _rand_candidate(rng, code, r)
+            cands.append((c_full, sh))
+        atol = float(rng.choice([0.0, 1e-8, 1e-3, 1.0, 1e30]))
+        rtol = float(rng.choice([0.0, 1e-6, 1e-2, 0.5, 2.0]))
+        en = bool(rng.integers(0, 2))
+        rd_full = r_full.to(DEV)
+        rd = rd_full[shift_r:shift_r + n]
+        cd_full = [c.to(DEV) for c, _ in cands]
+        cd = [cf[sh:sh + n] for cf, (_, sh) in zip(cd_full, cands)]
+        got, rh = run_dense(rd, cd, atol, rtol, en)
+        want = oracle.verify_batch(host_bytes(r), [host_bytes(c[sh:sh + n]) for c, sh in cands], code, atol, rtol, en)
+        assert_records_equal(got, want, f"seed {seed} dtype {code} n {n} N {n_cands} tol {atol},{rtol},{en}")
+        assert rh == oracle.hash_bytes(host_bytes(r))
+
+
+@pytest.mark.parametrize("seed", range(16))
+def test_randomised_ragged(oracle, seed):
+    # random tensors of all five dtypes (including empty ones), random candidate counts, tight or
+    # padded packing, special values; element counts passed explicitly
+    rng = np.random.default_rng(2000 + seed)
+    T = int(rng.choice([1, 7, 60, 150]))
+    N = int(rng.choice([1, 3, 4, 17]))
+    align = int(rng.choice([0, 16]))
+    codes = rng.integers(0, 5, T)
+    sizes = [int(rng.choice([0, 1, 3, 31, 64, 65, 127, 128, 129, 1000, 5000, 20011])) for _ in range(T)]
+    ref_chunks, cand_chunks, ref_off, cand_off = [], [], [], []
+    rc = cc = 0
+
+    def place(cur, esz):
+        a = align if align else esz
+        return (cur + a - 1) // a * a
+
+    for t in range(T):
+        code, n = int(codes[t]), sizes[t]
+        esz = ESZ[code]
+        r = _rand_values(rng, code, n)
+        start = place(rc, esz)
+        ref_chunks.append((start, r))
+        ref_off.append(start)
+        rc = start + n * esz
+        for j in range(N):
+            c = _rand_candidate(rng, code, r)
+            start = place(cc, esz)
+            cand_chunks.append((start, c))
+            cand_off.append(start)
+            cc = start + n * esz
+    ref_off.append(rc)
+    ref_buf = torch.zeros(max(rc, 1), dtype=torch.uint8)
+    cand_buf = torch.zeros(max(cc, 1), dtype=torch.uint8)
+    for start, x in ref_chunks:
+        if x.numel():
+            ref_buf[start:start + x.numel() * x.element_size()] = x.contiguous().view(torch.uint8)
+    for start, x in cand_chunks:
+        if x.numel():
+            cand_buf[start:start + x.numel() * x.element_size()] = x.contiguous().view(torch.uint8)
+    ref_off_t = torch.tensor(ref_off, dtype=torch.int64)
+    cand_off_t = torch.tensor(cand_off, dtype=torch.int64)
+    dtypes_t = torch.tensor(codes, dtype=torch.uint8)
+    n_el = torch.tensor(sizes, dtype=torch.int64)
+    atol = float(rng.choice([0.0, 1e-3, 1.0]))
+    rtol = float(rng.choice([0.0, 1e-2, 0.5]))
+    en = bool(rng.integers(0, 2))
+    ws = torch.empty(gv.gv_workspace_bytes(T, N), dtype=torch.uint8, device=DEV)
+    res = gv.gv_verify_ragged(ref_buf.to(DEV), ref_off_t.to(DEV), cand_buf.to(DEV), cand_off_t.to(DEV),
+                              dtypes_t.to(DEV), N, atol, rtol, en, n_elems=n_el.to(DEV), workspace=ws)
+    torch.cuda.synchronize()
+    assert gv.gv_check(ws) == gv.GV_OK
+    want = oracle.verify_ragged(ref_buf.numpy(), ref_off_t.numpy(), cand_buf.numpy(), cand_off_t.numpy(),
+                                dtypes_t.numpy(), N, atol, rtol, en, n_elems=n_el.numpy())
+    assert_records_equal(gv.results_to_numpy(res), want, f"ragged seed {seed} T {T} N {N} align {align}")

@@ -147,3 +147,57 @@ def test_config5_full(oracle):
                 g = got[t * wl.N:(t + 1) * wl.N]
                 w = want[a * wl.N:(a + 1) * wl.N]
                 assert g.tobytes() == w.tobytes(), f"tensor {t} (n={wl.n_elems[t]}, dtype {dtypes[t]})\n{g}\n{w}"
+
+
+def test_tensor_beyond_32_gib_uses_64_bit_word_indices(oracle):
+    """Maximum sizes: a 40 GiB int32 tensor (word indices of the hash pass 2^32, element indices pass
+    2^33). The oracle would need minutes for it, so the checks are properties that hold at any size:
+    an exact copy gives the zero record with the reference's hash; the reference hash equals what the
+    separate gv_hash kernel computes; a candidate changed in three known places differs from the copy
+    by exactly those three terms of the hash (recomputed here with Python integers), with the counts,
+    first index and exact maximum difference known by construction."""
+    free, _ = torch.cuda.mem_get_info()
+    n = 10 * (1 << 30)
+    need = 3 * n * 4 + (4 << 30)
+    if free < need:
+        pytest.skip(f"needs {need >> 30} GiB of free device memory")
+    g = torch.Generator(device=DEV).manual_seed(99)
+    ref = torch.empty(n, dtype=torch.int32, device=DEV)
+    step = 1 << 28
+    for s in range(0, n, step):                               # fill in slices (bounded temporaries)
+        ref[s:s + step] = torch.randint(-(1 << 30), 1 << 30, (min(step, n - s),), generator=g, device=DEV,
+                                        dtype=torch.int32)
+    copy = ref.clone()
+    mod = ref.clone()
+    places = [5, (1 << 33) + 11, n - 1]
+    deltas = [7, -3, 1 << 20]
+    old = [int(ref[p]) for p in places]
+    for p, d in zip(places, deltas):
+        mod[p] += d
+    res = torch.empty((2, 64), dtype=torch.uint8, device=DEV)
+    ws = torch.empty(gv.gv_workspace_bytes(0, 2), dtype=torch.uint8, device=DEV)
+    rh = torch.zeros(1, dtype=torch.int64, device=DEV)
+    gv.gv_verify_batch(ref, [copy, mod], results=res, ref_hash=rh, workspace=ws)
+    torch.cuda.synchronize()
+    assert gv.gv_check(ws) == gv.GV_OK
+    got = gv.results_to_numpy(res)
+    ref_hash = int(rh.cpu().numpy().view(np.uint64)[0])
+    assert ref_hash == int(gv.gv_hash(ref).cpu().numpy().view(np.uint64)[0])
+    zero = np.zeros((), dtype=gv.RESULT_DTYPE)
+    zero["first_mismatch"] = gv.GV_NO_INDEX
+    zero["hash"] = ref_hash
+    assert got[0].tobytes() == zero.tobytes()
+    assert int(got[1]["n_mismatch"]) == 3 and int(got[1]["first_mismatch"]) == 5
+    assert int(got[1]["max_abs_diff_int"]) == 1 << 20
+    # hash delta in closed form: only the three touched 64-bit words change
+    M64 = (1 << 64) - 1
+    want = ref_hash
+    for p in places:
+        k = p // 2
+        w_old = int.from_bytes(host_bytes(ref[2 * k:2 * k + 2]).tobytes(), "little")
+        w_new = int.from_bytes(host_bytes(mod[2 * k:2 * k + 2]).tobytes(), "little")
+        want = (want - oracle.splitmix64(k ^ w_old) + oracle.splitmix64(k ^ w_new)) & M64
+    assert int(got[1]["hash"]) == want
+    assert old == [int(ref[p]) for p in places]
+    del ref, copy, mod
+    torch.cuda.empty_cache()

@@ -254,17 +254,29 @@ dense_kernel(const __grid_constant__ DenseParams p) {
                     if (!vec_fast_float<DT>(c, rv, rflags, tol, &cacc[k], voff / ESZ)) settle_vector_exact<DT>(c, rv, voff / ESZ, tol, &cacc[k]);
                 }
             };
+            // Hash of a candidate vector. A vector that is bit-identical to the reference vector has the
+            // very hash terms of the reference vector (same words at the same word indices), so the
+            // lane only accumulates the reference's terms once per tile (ref_sum) and, per candidate,
+            // the *correction* hash(c) - hash(r) of the vectors that differ (slot). At the end of the
+            // chunk the candidate's partial is ref_sum + slot. Identical vectors cost no hash at all.
+            uint64_t h_ref = 0;        // hash terms of this lane's reference vector (current tile)
+            uint64_t ref_sum = 0;      // sum of h_ref over the tiles of this chunk
+            auto hash_of = [&](const uint4& v) -> uint64_t {
+                if constexpr (BIGK) return hash_vec_full(v, voff / 8);
+                else return hash_vec_full_k32(v, static_cast<uint32_t>(voff / 8), hc);
+            };
+            auto correct_slot = [&](const uint4& c, int k) {
+                const uint64_t d = hash_of(c) - h_ref;
+                const uint2 sl = slots[k * 32];
+                const uint64_t h = pack64(sl.x, sl.y) + d;
+                slots[k * 32] = make_uint2(static_cast<uint32_t>(h), static_cast<uint32_t>(h >> 32));
+            };
             // one visit: candidate vector c (already read from the ring) against the held reference
             auto visit = [&](const uint4& c, const uint4& r, int k) {
-                uint64_t h;
-                if constexpr (BIGK) h = hash_vec_full(c, voff / 8);
-                else h = hash_vec_full_k32(c, static_cast<uint32_t>(voff / 8), hc);
-                const uint2 sl = slots[k * 32];
-                h += pack64(sl.x, sl.y);
-                slots[k * 32] = make_uint2(static_cast<uint32_t>(h), static_cast<uint32_t>(h >> 32));
                 const bool differs = (c.x != r.x) || (c.y != r.y) || (c.z != r.z) || (c.w != r.w);
                 if (__any_sync(0xFFFFFFFFu, differs) || tile_forced) {
                     ensure_hoisted(r);
+                    if (differs) correct_slot(c, k);
                     if (differs || force != 0u) differing(c, r, k);
                 }
             };
@@ -305,7 +317,8 @@ dense_kernel(const __grid_constant__ DenseParams p) {
                 for (uint32_t i = 0; i < my_tiles; ++i) {
                     uint4 r;
                     if (!next_ref(i, r)) { timed_out = true; break; }
-                    if (g == 0 && p.ref_hash) my_ref_hash += hash_vec_full(r, voff / 8);
+                    h_ref = hash_of(r);
+                    ref_sum += h_ref;
                     new_tile(r);
                     const bool has_next = i + 1 < my_tiles;
 #pragma unroll 1
@@ -318,25 +331,23 @@ dense_kernel(const __grid_constant__ DenseParams p) {
                         uint4 c[U];
 #pragma unroll
                         for (int u = 0; u < U; ++u) c[u] = lds128(stage0 + u * 512u);
-                        // straight-line part for all U visits: hash, slot update, identity test
+                        // identity test for all U visits; identical vectors are done
                         uint32_t diffmask = 0u;
 #pragma unroll
                         for (int u = 0; u < U; ++u) {
-                            uint64_t h;
-                            if constexpr (BIGK) h = hash_vec_full(c[u], voff / 8);
-                            else h = hash_vec_full_k32(c[u], static_cast<uint32_t>(voff / 8), hc);
-                            const uint2 sl = slots[(k0 + u) * 32];
-                            h += pack64(sl.x, sl.y);
-                            slots[(k0 + u) * 32] = make_uint2(static_cast<uint32_t>(h), static_cast<uint32_t>(h >> 32));
                             const bool differs = (c[u].x != r.x) || (c[u].y != r.y) || (c[u].z != r.z) || (c[u].w != r.w);
                             diffmask |= differs ? (1u << u) : 0u;
                         }
                         if (__any_sync(0xFFFFFFFFu, diffmask != 0u) || tile_forced) {
                             ensure_hoisted(r);
-                            diffmask |= force;      // force is 0 or all ones
 #pragma unroll
                             for (int u = 0; u < U; ++u) {
-                                if (diffmask & (1u << u)) differing(c[u], r, k0 + u);
+                                if (diffmask & (1u << u)) {
+                                    correct_slot(c[u], k0 + u);        // hash chain and compare share one block
+                                    differing(c[u], r, k0 + u);
+                                } else if (force != 0u) {
+                                    differing(c[u], r, k0 + u);        // identical, but the reference holds a NaN
+                                }
                             }
                         }
 #pragma unroll
@@ -368,7 +379,8 @@ dense_kernel(const __grid_constant__ DenseParams p) {
                 for (uint32_t i = 0; i < my_tiles; ++i) {
                     uint4 r;
                     if (!next_ref(i, r)) { timed_out = true; break; }
-                    if (g == 0 && p.ref_hash) my_ref_hash += hash_vec_full(r, voff / 8);
+                    h_ref = hash_of(r);
+                    ref_sum += h_ref;
                     new_tile(r);
 #pragma unroll 1
                     for (int k = 0; k < kg; ++k) {
@@ -382,6 +394,13 @@ dense_kernel(const __grid_constant__ DenseParams p) {
                 }
             }
             cp_async_wait<0>();
+            // every candidate's partial = the reference's terms over this lane's tiles + its corrections
+            for (int k = 0; k < kg; ++k) {
+                const uint2 sl = slots[k * 32];
+                const uint64_t h = pack64(sl.x, sl.y) + ref_sum;
+                slots[k * 32] = make_uint2(static_cast<uint32_t>(h), static_cast<uint32_t>(h >> 32));
+            }
+            if (g == 0 && p.ref_hash) my_ref_hash += ref_sum;
             if (timed_out) {
                 // flag it; give the copy that may still be in flight a second bounded chance to land
                 if (lane == 0) {

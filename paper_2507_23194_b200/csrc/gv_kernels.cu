@@ -653,13 +653,19 @@ __device__ __forceinline__ void ragged_stretch(const RaggedParams& p, int dt, co
     const uint64_t full_end_all = nbytes / kWarpTile;                  // tiles [0, full_end_all) are full
     const uint64_t full_end = aligned ? (tile_end < full_end_all ? tile_end : full_end_all) : tile_begin;
 
-    auto one_visit = [&](const uint4& c, const uint4& r, bool force, uint64_t voff, int k) {
-        uint64_t h = hash_vec_full(c, voff / 8);
-        const uint2 sl = slots[k * 32];
-        h += pack64(sl.x, sl.y);
-        slots[k * 32] = make_uint2(static_cast<uint32_t>(h), static_cast<uint32_t>(h >> 32));
-        const bool differs = (c.x != r.x) || (c.y != r.y) || (c.z != r.z) || (c.w != r.w) || force;
-        if (differs) ragged_differing(dt, c, r, voff, tol, &wacc[k]);
+    // As in the dense kernel, a vector identical to the reference vector contributes the reference
+    // vector's own hash terms: those are summed once per tile (ref_sum), the slots only collect the
+    // corrections hash(c) - hash(r) of differing vectors, and ref_sum is added to every slot at the end.
+    uint64_t ref_sum = 0;
+    auto one_visit = [&](const uint4& c, const uint4& r, uint64_t h_ref, bool force, uint64_t voff, int k) {
+        const bool differs = (c.x != r.x) || (c.y != r.y) || (c.z != r.z) || (c.w != r.w);
+        if (differs) {
+            const uint64_t d = hash_vec_full(c, voff / 8) - h_ref;
+            const uint2 sl = slots[k * 32];
+            const uint64_t h = pack64(sl.x, sl.y) + d;
+            slots[k * 32] = make_uint2(static_cast<uint32_t>(h), static_cast<uint32_t>(h >> 32));
+        }
+        if (differs || force) ragged_differing(dt, c, r, voff, tol, &wacc[k]);
     };
 
     if (full_end > tile_begin) {
@@ -689,13 +695,15 @@ __device__ __forceinline__ void ragged_stretch(const RaggedParams& p, int dt, co
             stage = (stage + 1u) & (kRing - 1);
             issue_one();
             const bool force = nan_matters && vec_has_nan(dt, r);
+            const uint64_t h_ref = hash_vec_full(r, voff / 8);
+            ref_sum += h_ref;
 #pragma unroll 1
             for (int k = 0; k < kg; ++k) {
                 cp_async_wait<kRing - 1>();
                 const uint4 c = lds128(ring_base + stage * 512u);
                 stage = (stage + 1u) & (kRing - 1);
                 issue_one();
-                one_visit(c, r, force, voff, k);
+                one_visit(c, r, h_ref, force, voff, k);
             }
         }
         cp_async_wait<0>();
@@ -711,12 +719,22 @@ __device__ __forceinline__ void ragged_stretch(const RaggedParams& p, int dt, co
         const bool full = rem >= 16;
         const uint4 r = load_vec_any(esz, ref, voff, nbytes);
         const bool force = nan_matters && full && vec_has_nan(dt, r);
+        uint64_t h_ref = 0;
+        if (full) {
+            h_ref = hash_vec_full(r, voff / 8);
+            ref_sum += h_ref;
+        }
 #pragma unroll 1
         for (int k = 0; k < kg; ++k) {
             const uint4 c = load_vec_any(esz, wptr[k], voff, nbytes);
-            if (full) one_visit(c, r, force, voff, k);
+            if (full) one_visit(c, r, h_ref, force, voff, k);
             else ragged_partial(dt, c, r, voff, nvalid, tol, &wacc[k], &slots[k * 32]);
         }
+    }
+    for (int k = 0; k < kg; ++k) {
+        const uint2 sl = slots[k * 32];
+        const uint64_t h = pack64(sl.x, sl.y) + ref_sum;
+        slots[k * 32] = make_uint2(static_cast<uint32_t>(h), static_cast<uint32_t>(h >> 32));
     }
 }
 

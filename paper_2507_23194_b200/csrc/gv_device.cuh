@@ -455,9 +455,12 @@ __device__ __noinline__ uint32_t rel_candidate_bits(float ad, float ar, float M,
 // index is merged. Max |d| and, for the elements whose estimate passes the filter, the exact relative
 // error go to the CTA accumulators. Returns false when a NaN or an infinity is involved: the caller
 // then runs the exact per-element rule on this vector (nothing has been recorded in that case).
+// n_not_close: the number of elements found not close is ADDED to this per-lane counter; the caller
+// merges it into the accumulator at a point where the whole warp is converged (one reduction and one
+// atomic per warp) -- inside this function the set of lanes present is not known reliably.
 template <int DT>
 __device__ __forceinline__ bool vec_fast_float(const uint4& c, const RefVec<16 / Traits<DT>::ESZ>& r, uint32_t flags,
-                                               const TolF& t, CtaAcc* s, uint64_t elem0) {
+                                               const TolF& t, CtaAcc* s, uint64_t elem0, uint32_t& n_not_close) {
     constexpr int EPV = 16 / Traits<DT>::ESZ;
     // running maxima of this (CTA, candidate): max|d| bits, max relative error bits, filter threshold
     const uint4 run = lds128(smem_u32(&s->maxabs));
@@ -491,10 +494,7 @@ __device__ __forceinline__ bool vec_fast_float(const uint4& c, const RefVec<16 /
         }
         if (cnt) {
             GV_COUNT(3);
-            // one shared-memory atomic per lane that found mismatches. (Aggregating over the lanes
-            // that happen to be here would need their exact set; the mask of active threads is not a
-            // reliable source for it once the compiler moves the query, and a wrong set drops counts.)
-            atomicAdd(&s->cnt, static_cast<unsigned long long>(cnt));
+            n_not_close += cnt;
             const unsigned long long idx = elem0 + first_e;
             if (idx < *reinterpret_cast<volatile unsigned long long*>(&s->first)) atomicMin(&s->first, idx);
         }
@@ -646,6 +646,12 @@ __device__ __forceinline__ uint64_t warp_max_u64(uint64_t v) {
         v = x > v ? x : v;
     }
     return v;
+}
+
+// Merge per-lane mismatch counts at a point where all 32 lanes of the warp are converged.
+__device__ __forceinline__ void merge_counts_converged(CtaAcc* s, uint32_t lane_cnt) {
+    const uint32_t total = __reduce_add_sync(0xFFFFFFFFu, lane_cnt);
+    if (total && (threadIdx.x & 31) == 0) atomicAdd(&s->cnt, static_cast<unsigned long long>(total));
 }
 
 // Rare-path partials of one thread's visit -> CTA accumulators.

@@ -247,11 +247,14 @@ dense_kernel(const __grid_constant__ DenseParams p) {
                 }
             };
             // a candidate vector that is not bit-identical to the reference vector (ensure_hoisted done)
-            auto differing = [&](const uint4& c, const uint4& r, int k) {
+            // (mismatches of float vectors settled on the fast path are added to lane_cnt; the caller
+            // merges lane_cnt into the accumulator once the warp has reconverged)
+            auto differing = [&](const uint4& c, const uint4& r, int k, uint32_t& lane_cnt) {
                 if constexpr (!IS_FLOAT) {
                     settle_vector_int<DT>(c, r, voff / ESZ, &cacc[k]);
                 } else {
-                    if (!vec_fast_float<DT>(c, rv, rflags, tol, &cacc[k], voff / ESZ)) settle_vector_exact<DT>(c, rv, voff / ESZ, tol, &cacc[k]);
+                    if (!vec_fast_float<DT>(c, rv, rflags, tol, &cacc[k], voff / ESZ, lane_cnt))
+                        settle_vector_exact<DT>(c, rv, voff / ESZ, tol, &cacc[k]);
                 }
             };
             // Hash of a candidate vector. A vector that is bit-identical to the reference vector has the
@@ -276,8 +279,12 @@ dense_kernel(const __grid_constant__ DenseParams p) {
                 const bool differs = (c.x != r.x) || (c.y != r.y) || (c.z != r.z) || (c.w != r.w);
                 if (__any_sync(0xFFFFFFFFu, differs) || tile_forced) {
                     ensure_hoisted(r);
+                    uint32_t lane_cnt = 0u;
                     if (differs) correct_slot(c, k);
-                    if (differs || force != 0u) differing(c, r, k);
+                    if (differs || force != 0u) differing(c, r, k, lane_cnt);
+                    if constexpr (IS_FLOAT) {
+                        if (__any_sync(0xFFFFFFFFu, lane_cnt != 0u)) merge_counts_converged(&cacc[k], lane_cnt);
+                    }
                 }
             };
             // reference of tile i: wait for its bulk copy, take this lane's vector, start the next copy
@@ -340,13 +347,26 @@ dense_kernel(const __grid_constant__ DenseParams p) {
                         }
                         if (__any_sync(0xFFFFFFFFu, diffmask != 0u) || tile_forced) {
                             ensure_hoisted(r);
+                            uint32_t lane_cnt[U];
 #pragma unroll
                             for (int u = 0; u < U; ++u) {
+                                lane_cnt[u] = 0u;
                                 if (diffmask & (1u << u)) {
                                     correct_slot(c[u], k0 + u);        // hash chain and compare share one block
-                                    differing(c[u], r, k0 + u);
+                                    differing(c[u], r, k0 + u, lane_cnt[u]);
                                 } else if (force != 0u) {
-                                    differing(c[u], r, k0 + u);        // identical, but the reference holds a NaN
+                                    differing(c[u], r, k0 + u, lane_cnt[u]);   // identical, but the reference holds a NaN
+                                }
+                            }
+                            if constexpr (IS_FLOAT) {
+                                // the warp is converged again here; mismatches are rare, so one vote first,
+                                // then one reduction and at most one atomic per visit
+                                uint32_t any_cnt = 0u;
+#pragma unroll
+                                for (int u = 0; u < U; ++u) any_cnt |= lane_cnt[u];
+                                if (__any_sync(0xFFFFFFFFu, any_cnt != 0u)) {
+#pragma unroll
+                                    for (int u = 0; u < U; ++u) merge_counts_converged(&cacc[k0 + u], lane_cnt[u]);
                                 }
                             }
                         }
@@ -563,26 +583,25 @@ __device__ __forceinline__ void ragged_differing_t(const uint4& c, const uint4& 
                                                    CtaAcc* s) {
     if constexpr (Traits<DT>::IS_FLOAT) {
         RefVec<16 / Traits<DT>::ESZ> rv;
-        uint32_t force;
-        hoist_ref<DT>(r, tol, rv, force);
-        if (!vec_fast_float<DT>(c, rv, force, tol, s, elem0)) {
-            Acc a;
-            a.clear();
-            const uint32_t thr = *reinterpret_cast<volatile unsigned int*>(&s->thr);
-            vec_exact_float<DT>(c, rv, elem0, tol, thr, a);
-            push_rare(s, a);
-            if (a.cnt) atomicAdd(&s->cnt, static_cast<unsigned long long>(a.cnt));
-            raise_maxabs(s, a.maxabs);
-        }
+        uint32_t flags;
+        hoist_ref<DT>(r, tol, rv, flags);
+        uint32_t lane_cnt = 0u;
+        if (!vec_fast_float<DT>(c, rv, flags, tol, s, elem0, lane_cnt)) settle_vector_exact<DT>(c, rv, elem0, tol, s);
+        // (called from diverged code: one shared atomic per lane that found mismatches)
+        if (lane_cnt) atomicAdd(&s->cnt, static_cast<unsigned long long>(lane_cnt));
     } else {
-        Acc a;
-        a.clear();
-        vec_int<DT>(c, r, elem0, 16 / Traits<DT>::ESZ, a);
-        push_rare(s, a);
-        if (a.cnt) atomicAdd(&s->cnt, static_cast<unsigned long long>(a.cnt));
+        settle_vector_int<DT>(c, r, elem0, s);
     }
 }
-__device__ __noinline__ void ragged_differing(int dt, uint4 c, uint4 r, uint64_t byte_off, TolF tol, CtaAcc* s) {
+#ifndef GV_RAGGED_INLINE
+#define GV_RAGGED_INLINE 0
+#endif
+#if GV_RAGGED_INLINE
+__device__ __forceinline__
+#else
+__device__ __noinline__
+#endif
+void ragged_differing(int dt, const uint4& c, const uint4& r, uint64_t byte_off, const TolF& tol, CtaAcc* s) {
     switch (dt) {
         case GV_F32: ragged_differing_t<GV_F32>(c, r, byte_off / 4, tol, s); break;
         case GV_BF16: ragged_differing_t<GV_BF16>(c, r, byte_off / 2, tol, s); break;

@@ -586,22 +586,27 @@ __device__ __forceinline__ void ragged_differing_t(const uint4& c, const uint4& 
         uint32_t flags;
         hoist_ref<DT>(r, tol, rv, flags);
         uint32_t lane_cnt = 0u;
-        if (!vec_fast_float<DT>(c, rv, flags, tol, s, elem0, lane_cnt)) settle_vector_exact<DT>(c, rv, elem0, tol, s);
+        if (!vec_fast_float<DT>(c, rv, flags, tol, s, elem0, lane_cnt)) {
+            Acc a;
+            a.clear();
+            const uint32_t thr = *reinterpret_cast<volatile unsigned int*>(&s->thr);
+            vec_exact_float<DT>(c, rv, elem0, tol, thr, a);
+            push_rare(s, a);
+            lane_cnt += a.cnt;
+            raise_maxabs(s, a.maxabs);
+        }
         // (called from diverged code: one shared atomic per lane that found mismatches)
         if (lane_cnt) atomicAdd(&s->cnt, static_cast<unsigned long long>(lane_cnt));
     } else {
-        settle_vector_int<DT>(c, r, elem0, s);
+        Acc a;
+        a.clear();
+        vec_int<DT>(c, r, elem0, 16 / Traits<DT>::ESZ, a);
+        push_rare(s, a);
+        if (a.cnt) atomicAdd(&s->cnt, static_cast<unsigned long long>(a.cnt));
     }
 }
-#ifndef GV_RAGGED_INLINE
-#define GV_RAGGED_INLINE 0
-#endif
-#if GV_RAGGED_INLINE
-__device__ __forceinline__
-#else
-__device__ __noinline__
-#endif
-void ragged_differing(int dt, const uint4& c, const uint4& r, uint64_t byte_off, const TolF& tol, CtaAcc* s) {
+// (out of line, arguments by value: by-reference arguments would live in local memory)
+__device__ __noinline__ void ragged_differing(int dt, uint4 c, uint4 r, uint64_t byte_off, TolF tol, CtaAcc* s) {
     switch (dt) {
         case GV_F32: ragged_differing_t<GV_F32>(c, r, byte_off / 4, tol, s); break;
         case GV_BF16: ragged_differing_t<GV_BF16>(c, r, byte_off / 2, tol, s); break;

@@ -170,6 +170,10 @@ template <int N>
 __device__ __forceinline__ void cp_async_wait() {
     asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
 }
+__device__ __forceinline__ void sts128(uint32_t smem_addr, const uint4& v) {
+    asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(smem_addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w)
+                 : "memory");
+}
 __device__ __forceinline__ uint4 lds128(uint32_t smem_addr) {
     uint4 v;
     asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];"
@@ -388,16 +392,19 @@ __device__ __forceinline__ void hoist_ref(const uint4& raw, const TolF& t, RefVe
                                           uint32_t& flags) {
     constexpr int EPV = 16 / Traits<DT>::ESZ;
     Widen<DT>::run(raw, o.rf);
+    // tol is a monotone function of |r| (two correctly rounded monotone steps), so the smallest tol of
+    // the vector is the tol of its smallest |r|. fminf skips NaNs: a NaN element makes d NaN anyway.
     uint32_t umax = 0u, umin1 = 0xFFFFFFFFu;
-    float tolmin = __uint_as_float(0x7F7FFFFFu);
+    float amin = __uint_as_float(0x7F800000u);
 #pragma unroll
     for (int e = 0; e < EPV; ++e) {
         const float a = fabsf(o.rf[e]);
         const uint32_t u = __float_as_uint(a);
-        tolmin = fminf(tolmin, tolc_of(a, t));                        // a NaN tol is skipped: r NaN makes d NaN anyway
+        amin = fminf(amin, a);
         umax = u > umax ? u : umax;
         umin1 = (u - 1u) < umin1 ? (u - 1u) : umin1;                  // u == 0 wraps to the top: ignored
     }
+    const float tolmin = tolc_of(amin, t);
     o.tolmin = tolmin;
     flags = ((umax > 0x7F800000u && !t.equal_nan) ? 1u : 0u) | ((umin1 < kTinyBits - 1u) ? 2u : 0u);
 }

@@ -112,12 +112,26 @@ constexpr int kWarps = kThreads / 32;
 constexpr int kRing = GV_RING;            // asynchronous copies in flight per lane (power of two)
 constexpr int kWarpTile = 512;            // bytes of one warp-tile
 
+// Queue of differing vectors (one per warp). A candidate vector that differs from the reference
+// vector is not compared where it is found: the lane appends (candidate vector, reference vector,
+// byte offset | candidate slot, the reference vector's hash terms) to the warp's queue, and whenever
+// 32 entries have gathered the warp compares them at once, one entry per lane. Sparse differences
+// (a few lanes per visit) thus cost one full-width pass per 32 differing vectors instead of one
+// mostly idle pass per visit.
+constexpr int kQCap = 64;                           // entries (a power of two, >= 31 pending + 32 new)
+constexpr uint32_t kQPlane = kQCap * 16;            // bytes of one plane (candidate / reference / meta)
+constexpr size_t kQueueBytes = 3 * size_t(kQPlane);
+#ifndef GV_QDIRECT
+#define GV_QDIRECT 20                               // visits with at least this many differing lanes are compared in place
+#endif
+
 template <int WARPS>
 struct DenseSmem {
     static constexpr size_t kRingOff = 0;                                                 // [warp][kRing][32] uint4
     static constexpr size_t kRefOff = kRingOff + size_t(WARPS) * kRing * kWarpTile;       // [warp][2][32] uint4
     static constexpr size_t kSlotOff = kRefOff + size_t(WARPS) * 2 * kWarpTile;           // [warp][kChunk][32] u64
-    static constexpr size_t kAccOff = kSlotOff + size_t(WARPS) * kChunk * 32 * 8;         // CtaAcc[kChunk]
+    static constexpr size_t kQueueOff = kSlotOff + size_t(WARPS) * kChunk * 32 * 8;       // [warp][3][kQCap] uint4
+    static constexpr size_t kAccOff = kQueueOff + size_t(WARPS) * kQueueBytes;            // CtaAcc[kChunk]
     static constexpr size_t kBarOff = kAccOff + sizeof(CtaAcc) * kChunk;                  // [warp][2] mbarrier
     static constexpr size_t kRefHashOff = kBarOff + size_t(WARPS) * 2 * 8;
     static constexpr size_t kTotal = kRefHashOff + 8;
@@ -155,6 +169,55 @@ __device__ __noinline__ void settle_vector_int(uint4 c, uint4 r, uint64_t elem0,
     if (a.cnt) atomicAdd(&s->cnt, static_cast<unsigned long long>(a.cnt));
 }
 
+// Compare the n (<= 32) oldest entries of the warp's queue, one per lane; called with the warp
+// converged. qbase: shared address of the warp's queue; slots: this lane's column of hash slots;
+// acc: the accumulators the entries' slot numbers index.
+template <int DT, bool BIGK>
+__device__ __forceinline__ void batch_entries(uint32_t qbase, uint32_t head, uint32_t n, uint2* slots, CtaAcc* acc,
+                                              const TolF& tol) {
+    constexpr int ESZ = Traits<DT>::ESZ;
+    const uint32_t lane = threadIdx.x & 31u;
+    if (lane < n) {
+        const uint32_t at = qbase + ((head + lane) & (kQCap - 1)) * 16u;
+        const uint4 c = lds128(at);
+        const uint4 r = lds128(at + kQPlane);
+        const uint4 m = lds128(at + 2 * kQPlane);
+        const uint64_t meta = pack64(m.x, m.y), h_ref = pack64(m.z, m.w);
+        const int k = static_cast<int>(m.x & 15u);
+        const uint64_t voff = meta & ~uint64_t(15);
+        uint64_t h;
+        if constexpr (BIGK) {
+            h = hash_vec_full(c, voff / 8);
+        } else {
+            HashConsts hc;
+            hc.init();
+            h = hash_vec_full_k32(c, static_cast<uint32_t>(voff / 8), hc);
+        }
+        const uint2 sl = slots[k * 32];
+        const uint64_t hs = pack64(sl.x, sl.y) + (h - h_ref);
+        slots[k * 32] = make_uint2(static_cast<uint32_t>(hs), static_cast<uint32_t>(hs >> 32));
+        CtaAcc* s = &acc[k];
+        if constexpr (Traits<DT>::IS_FLOAT) {
+            RefVec<16 / ESZ> rv;
+            uint32_t rflags = 0u, cnt = 0u;
+            hoist_ref<DT>(r, tol, rv, rflags);
+            if (!vec_fast_float<DT>(c, rv, rflags, tol, s, voff / ESZ, cnt)) settle_vector_exact<DT>(c, rv, voff / ESZ, tol, s);
+            if (cnt) atomicAdd(&s->cnt, static_cast<unsigned long long>(cnt));
+        } else {
+            Acc a;
+            a.clear();
+            vec_int<DT>(c, r, voff / ESZ, 16 / ESZ, a);
+            push_rare(s, a);
+            if (a.cnt) atomicAdd(&s->cnt, static_cast<unsigned long long>(a.cnt));
+        }
+    }
+}
+template <int DT, bool BIGK>
+__device__ __noinline__ void process_batch(uint32_t qbase, uint32_t head, uint32_t n, uint2* slots, CtaAcc* cacc,
+                                           TolF tol) {
+    batch_entries<DT, BIGK>(qbase, head, n, slots, cacc, tol);
+}
+
 // BIGK: word indices of the hash need more than 32 bits (tensors of 32 GiB and more).
 template <int DT, bool BIGK>
 __global__ void __launch_bounds__(DenseShape<DT>::kWarpsPerCta * 32, DenseShape<DT>::kCtasPerSm)
@@ -172,6 +235,9 @@ dense_kernel(const __grid_constant__ DenseParams p) {
     unsigned char* ref_stage = smem + Smem::kRefOff + size_t(warp) * 2 * kWarpTile;
     uint2* slots = reinterpret_cast<uint2*>(smem + Smem::kSlotOff) + size_t(warp) * kChunk * 32 + lane;
     const uint32_t ring_base = smem_u32(smem + Smem::kRingOff) + (warp * kRing * 32 + lane) * 16;
+    const uint32_t qbase = smem_u32(smem + Smem::kQueueOff) + warp * static_cast<uint32_t>(kQueueBytes);
+    const uint32_t lanes_below = (1u << lane) - 1u;
+    uint32_t qhead = 0u, qcount = 0u;                       // the warp's queue of differing vectors (warp-uniform)
 
     const uint64_t nbytes = p.n * ESZ;
     const uint64_t full_tiles = p.all_aligned ? nbytes / kWarpTile : 0;      // tiles the fast loop takes
@@ -274,16 +340,45 @@ dense_kernel(const __grid_constant__ DenseParams p) {
                 const uint64_t h = pack64(sl.x, sl.y) + d;
                 slots[k * 32] = make_uint2(static_cast<uint32_t>(h), static_cast<uint32_t>(h >> 32));
             };
-            // one visit: candidate vector c (already read from the ring) against the held reference
+            // Append this lane's vector (if it wants a compare) to the warp's queue; bal = ballot of the
+            // lanes that do. Compares the 32 oldest entries as soon as 32 have gathered.
+            auto enqueue = [&](const uint4& c, const uint4& r, int k, bool want, uint32_t bal) {
+                if (want) {
+                    const uint32_t at = qbase + ((qhead + qcount + __popc(bal & lanes_below)) & (kQCap - 1)) * 16u;
+                    const uint64_t meta = voff | static_cast<uint64_t>(k);
+                    sts128(at, c);
+                    sts128(at + kQPlane, r);
+                    sts128(at + 2 * kQPlane, make_uint4(static_cast<uint32_t>(meta), static_cast<uint32_t>(meta >> 32),
+                                                        static_cast<uint32_t>(h_ref), static_cast<uint32_t>(h_ref >> 32)));
+                }
+                qcount += __popc(bal);
+                if (qcount >= 32u) {
+                    __syncwarp();
+                    process_batch<DT, BIGK>(qbase, qhead, 32u, slots, cacc, tol);
+                    __syncwarp();
+                    qhead = (qhead + 32u) & (kQCap - 1);
+                    qcount -= 32u;
+                }
+            };
+            // one visit: candidate vector c (already read from the ring) against the held reference.
+            // A lane wants a compare when its vector differs, or when the reference holds a NaN that
+            // equal_nan does not excuse. Dense differences (GV_QDIRECT lanes or more) are compared in
+            // place against the values hoisted for the tile; sparse ones are queued.
             auto visit = [&](const uint4& c, const uint4& r, int k) {
                 const bool differs = (c.x != r.x) || (c.y != r.y) || (c.z != r.z) || (c.w != r.w);
                 if (__any_sync(0xFFFFFFFFu, differs) || tile_forced) {
-                    ensure_hoisted(r);
-                    uint32_t lane_cnt = 0u;
-                    if (differs) correct_slot(c, k);
-                    if (differs || force != 0u) differing(c, r, k, lane_cnt);
-                    if constexpr (IS_FLOAT) {
-                        if (__any_sync(0xFFFFFFFFu, lane_cnt != 0u)) merge_counts_converged(&cacc[k], lane_cnt);
+                    const bool want = differs || force != 0u;
+                    const uint32_t bal = __ballot_sync(0xFFFFFFFFu, want);
+                    if (__popc(bal) >= GV_QDIRECT) {
+                        ensure_hoisted(r);
+                        uint32_t lane_cnt = 0u;
+                        if (differs) correct_slot(c, k);
+                        if (want) differing(c, r, k, lane_cnt);
+                        if constexpr (IS_FLOAT) {
+                            if (__any_sync(0xFFFFFFFFu, lane_cnt != 0u)) merge_counts_converged(&cacc[k], lane_cnt);
+                        }
+                    } else if (bal) {
+                        enqueue(c, r, k, want, bal);
                     }
                 }
             };
@@ -346,27 +441,40 @@ dense_kernel(const __grid_constant__ DenseParams p) {
                             diffmask |= differs ? (1u << u) : 0u;
                         }
                         if (__any_sync(0xFFFFFFFFu, diffmask != 0u) || tile_forced) {
-                            ensure_hoisted(r);
-                            uint32_t lane_cnt[U];
+                            // sparse visits go to the queue; dense ones are collected in directmask
+                            uint32_t directmask = 0u;
 #pragma unroll
                             for (int u = 0; u < U; ++u) {
-                                lane_cnt[u] = 0u;
-                                if (diffmask & (1u << u)) {
-                                    correct_slot(c[u], k0 + u);        // hash chain and compare share one block
-                                    differing(c[u], r, k0 + u, lane_cnt[u]);
-                                } else if (force != 0u) {
-                                    differing(c[u], r, k0 + u, lane_cnt[u]);   // identical, but the reference holds a NaN
-                                }
+                                const bool want = ((diffmask >> u) & 1u) || force != 0u;
+                                const uint32_t bal = __ballot_sync(0xFFFFFFFFu, want);
+                                if (__popc(bal) >= GV_QDIRECT) directmask |= 1u << u;
+                                else if (bal) enqueue(c[u], r, k0 + u, want, bal);
                             }
-                            if constexpr (IS_FLOAT) {
-                                // the warp is converged again here; mismatches are rare, so one vote first,
-                                // then one reduction and at most one atomic per visit
-                                uint32_t any_cnt = 0u;
+                            if (directmask) {
+                                ensure_hoisted(r);
+                                uint32_t lane_cnt[U];
 #pragma unroll
-                                for (int u = 0; u < U; ++u) any_cnt |= lane_cnt[u];
-                                if (__any_sync(0xFFFFFFFFu, any_cnt != 0u)) {
+                                for (int u = 0; u < U; ++u) {
+                                    lane_cnt[u] = 0u;
+                                    if (directmask & (1u << u)) {
+                                        if (diffmask & (1u << u)) {
+                                            correct_slot(c[u], k0 + u);        // hash chain and compare share one block
+                                            differing(c[u], r, k0 + u, lane_cnt[u]);
+                                        } else if (force != 0u) {
+                                            differing(c[u], r, k0 + u, lane_cnt[u]);   // identical, but the reference holds a NaN
+                                        }
+                                    }
+                                }
+                                if constexpr (IS_FLOAT) {
+                                    // the warp is converged again here; mismatches are rare, so one vote first,
+                                    // then one reduction and at most one atomic per visit
+                                    uint32_t any_cnt = 0u;
 #pragma unroll
-                                    for (int u = 0; u < U; ++u) merge_counts_converged(&cacc[k0 + u], lane_cnt[u]);
+                                    for (int u = 0; u < U; ++u) any_cnt |= lane_cnt[u];
+                                    if (__any_sync(0xFFFFFFFFu, any_cnt != 0u)) {
+#pragma unroll
+                                        for (int u = 0; u < U; ++u) merge_counts_converged(&cacc[k0 + u], lane_cnt[u]);
+                                    }
                                 }
                             }
                         }
@@ -414,6 +522,13 @@ dense_kernel(const __grid_constant__ DenseParams p) {
                 }
             }
             cp_async_wait<0>();
+            if (qcount) {                                  // the chunk's accumulators close: drain the queue
+                __syncwarp();
+                process_batch<DT, BIGK>(qbase, qhead, qcount, slots, cacc, tol);
+                __syncwarp();
+                qhead = 0u;
+                qcount = 0u;
+            }
             // every candidate's partial = the reference's terms over this lane's tiles + its corrections
             for (int k = 0; k < kg; ++k) {
                 const uint2 sl = slots[k * 32];
@@ -571,7 +686,8 @@ struct RaggedSmem {
     static constexpr size_t kSlotOff = kRingOff + size_t(kWarps) * kRing * kWarpTile;      // [warp][kChunk][32] u64
     static constexpr size_t kAccOff = kSlotOff + size_t(kWarps) * kChunk * 32 * 8;         // [warp][kChunk] CtaAcc
     static constexpr size_t kPtrOff = kAccOff + size_t(kWarps) * kChunk * sizeof(CtaAcc);  // [warp][kChunk] candidate pointers
-    static constexpr size_t kTotal = kPtrOff + size_t(kWarps) * kChunk * 8;
+    static constexpr size_t kQueueOff = kPtrOff + size_t(kWarps) * kChunk * 8;             // [warp][3][kQCap] uint4
+    static constexpr size_t kTotal = kQueueOff + size_t(kWarps) * kQueueBytes;
 };
 
 // A full candidate vector that differs from its reference vector, any dtype. Out of line and
@@ -613,6 +729,17 @@ __device__ __noinline__ void ragged_differing(int dt, uint4 c, uint4 r, uint64_t
         case GV_F16: ragged_differing_t<GV_F16>(c, r, byte_off / 2, tol, s); break;
         case GV_I32: ragged_differing_t<GV_I32>(c, r, byte_off / 4, tol, s); break;
         default: ragged_differing_t<GV_I64>(c, r, byte_off / 8, tol, s); break;
+    }
+}
+// The warp's queue of differing vectors (all of one tensor, hence of one dtype): the n oldest entries.
+__device__ __noinline__ void ragged_batch(int dt, uint32_t qbase, uint32_t head, uint32_t n, uint2* slots, CtaAcc* wacc,
+                                          TolF tol) {
+    switch (dt) {
+        case GV_F32: batch_entries<GV_F32, true>(qbase, head, n, slots, wacc, tol); break;
+        case GV_BF16: batch_entries<GV_BF16, true>(qbase, head, n, slots, wacc, tol); break;
+        case GV_F16: batch_entries<GV_F16, true>(qbase, head, n, slots, wacc, tol); break;
+        case GV_I32: batch_entries<GV_I32, true>(qbase, head, n, slots, wacc, tol); break;
+        default: batch_entries<GV_I64, true>(qbase, head, n, slots, wacc, tol); break;
     }
 }
 // The partial vector at the end of a tensor: element by element through the general rule.
@@ -667,7 +794,7 @@ __device__ __forceinline__ bool vec_has_nan(int dt, const uint4& r) {
 __device__ __forceinline__ void ragged_stretch(const RaggedParams& p, int dt, const unsigned char* ref, uint64_t n,
                                                uint64_t tile_begin, uint64_t tile_end, int kg, uint2* slots,
                                                CtaAcc* wacc, const unsigned char* const* wptr, int lane,
-                                               uint32_t ring_base) {
+                                               uint32_t ring_base, uint32_t qbase) {
     const int esz = elem_size(dt);
     const uint64_t nbytes = n * esz;
     const TolF tol = {p.atol, p.rtol, p.equal_nan};
@@ -690,6 +817,32 @@ __device__ __forceinline__ void ragged_stretch(const RaggedParams& p, int dt, co
             slots[k * 32] = make_uint2(static_cast<uint32_t>(h), static_cast<uint32_t>(h >> 32));
         }
         if (differs || force) ragged_differing(dt, c, r, voff, tol, &wacc[k]);
+    };
+
+    // Streamed tiles (the whole warp is present): differing vectors go to the warp's queue and are
+    // compared 32 at a time, one per lane, like the dense kernel's sparse visits.
+    const uint32_t lanes_below = (1u << lane) - 1u;
+    uint32_t qhead = 0u, qcount = 0u;
+    auto queued_visit = [&](const uint4& c, const uint4& r, uint64_t h_ref, bool force, uint64_t voff, int k) {
+        const bool want = (c.x != r.x) || (c.y != r.y) || (c.z != r.z) || (c.w != r.w) || force;
+        const uint32_t bal = __ballot_sync(0xFFFFFFFFu, want);
+        if (bal == 0u) return;
+        if (want) {
+            const uint32_t at = qbase + ((qhead + qcount + __popc(bal & lanes_below)) & (kQCap - 1)) * 16u;
+            const uint64_t meta = voff | static_cast<uint64_t>(k);
+            sts128(at, c);
+            sts128(at + kQPlane, r);
+            sts128(at + 2 * kQPlane, make_uint4(static_cast<uint32_t>(meta), static_cast<uint32_t>(meta >> 32),
+                                                static_cast<uint32_t>(h_ref), static_cast<uint32_t>(h_ref >> 32)));
+        }
+        qcount += __popc(bal);
+        if (qcount >= 32u) {
+            __syncwarp();
+            ragged_batch(dt, qbase, qhead, 32u, slots, wacc, tol);
+            __syncwarp();
+            qhead = (qhead + 32u) & (kQCap - 1);
+            qcount -= 32u;
+        }
     };
 
     if (full_end > tile_begin) {
@@ -727,10 +880,15 @@ __device__ __forceinline__ void ragged_stretch(const RaggedParams& p, int dt, co
                 const uint4 c = lds128(ring_base + stage * 512u);
                 stage = (stage + 1u) & (kRing - 1);
                 issue_one();
-                one_visit(c, r, h_ref, force, voff, k);
+                queued_visit(c, r, h_ref, force, voff, k);
             }
         }
         cp_async_wait<0>();
+        if (qcount) {                                   // the tensor's accumulators close: drain the queue
+            __syncwarp();
+            ragged_batch(dt, qbase, qhead, qcount, slots, wacc, tol);
+            __syncwarp();
+        }
     }
 
     // ---- synchronous part: the tail tile, or every tile of an unaligned tensor ----
@@ -769,6 +927,7 @@ __global__ void __launch_bounds__(kThreads, 2) ragged_kernel(const __grid_consta
     CtaAcc* wacc = reinterpret_cast<CtaAcc*>(smem + RaggedSmem::kAccOff) + warp * kChunk;
     const unsigned char** wptr = reinterpret_cast<const unsigned char**>(smem + RaggedSmem::kPtrOff) + warp * kChunk;
     const uint32_t ring_base = smem_u32(smem + RaggedSmem::kRingOff) + (warp * kRing * 32 + lane) * 16;
+    const uint32_t qbase = smem_u32(smem + RaggedSmem::kQueueOff) + warp * static_cast<uint32_t>(kQueueBytes);
 
     const uint64_t total = static_cast<uint64_t>(p.tile_prefix[p.T]);
     const uint64_t gw = static_cast<uint64_t>(blockIdx.x) * kWarps + warp;
@@ -807,7 +966,7 @@ __global__ void __launch_bounds__(kThreads, 2) ragged_kernel(const __grid_consta
             }
             for (int k = 0; k < kg; ++k) slots[k * 32] = make_uint2(0u, 0u);
             __syncwarp();
-            ragged_stretch(p, dt, ref, n, tile_begin, tile_end, kg, slots, wacc, wptr, lane, ring_base);
+            ragged_stretch(p, dt, ref, n, tile_begin, tile_end, kg, slots, wacc, wptr, lane, ring_base, qbase);
             __syncwarp();
             // leave the tensor (or this group of its candidates): combine and publish
             for (int k = 0; k < kg; ++k) {

@@ -441,22 +441,27 @@ dense_kernel(const __grid_constant__ DenseParams p) {
                             diffmask |= differs ? (1u << u) : 0u;
                         }
                         if (__any_sync(0xFFFFFFFFu, diffmask != 0u) || tile_forced) {
-                            // sparse visits go to the queue; dense ones are collected in directmask
-                            uint32_t directmask = 0u;
+                            // How many lanes want a compare, for all U visits at once: one byte per
+                            // visit, summed over the warp. Visits with GV_QDIRECT lanes or more are dense
+                            // (bit 7 of their byte in `dense`); the other non-empty ones go to the queue.
+                            static_assert(U == 4, "one byte per visit of the block");
+                            const uint32_t wantmask = force != 0u ? 0xFu : diffmask;
+                            const uint32_t counts = __reduce_add_sync(0xFFFFFFFFu, (wantmask * 0x00204081u) & 0x01010101u);
+                            const uint32_t dense = (counts + (0x80u - GV_QDIRECT) * 0x01010101u) & 0x80808080u;
 #pragma unroll
                             for (int u = 0; u < U; ++u) {
-                                const bool want = ((diffmask >> u) & 1u) || force != 0u;
-                                const uint32_t bal = __ballot_sync(0xFFFFFFFFu, want);
-                                if (__popc(bal) >= GV_QDIRECT) directmask |= 1u << u;
-                                else if (bal) enqueue(c[u], r, k0 + u, want, bal);
+                                if (!(dense & (0x80u << (8 * u))) && (counts & (0xFFu << (8 * u)))) {
+                                    const bool want = (wantmask >> u) & 1u;
+                                    enqueue(c[u], r, k0 + u, want, __ballot_sync(0xFFFFFFFFu, want));
+                                }
                             }
-                            if (directmask) {
+                            if (dense) {
                                 ensure_hoisted(r);
                                 uint32_t lane_cnt[U];
 #pragma unroll
                                 for (int u = 0; u < U; ++u) {
                                     lane_cnt[u] = 0u;
-                                    if (directmask & (1u << u)) {
+                                    if (dense & (0x80u << (8 * u))) {
                                         if (diffmask & (1u << u)) {
                                             correct_slot(c[u], k0 + u);        // hash chain and compare share one block
                                             differing(c[u], r, k0 + u, lane_cnt[u]);

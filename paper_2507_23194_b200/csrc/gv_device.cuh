@@ -385,8 +385,7 @@ __device__ __forceinline__ float tolc_of(float abs_r, const TolF& t) {
     return fminf(__fadd_rn(t.atol, __fmul_rn(t.rtol, abs_r)), __uint_as_float(0x7F7FFFFFu));
 }
 
-// flags: bit 0 = the vector holds a NaN that does not count as equal (identical candidate vectors
-// still need the rule); bit 1 = it holds a nonzero element below 2^-64 (relative filter not trusted)
+// flags: bit 1 = the vector holds a nonzero element below 2^-64 (relative filter not trusted)
 template <int DT>
 __device__ __forceinline__ void hoist_ref(const uint4& raw, const TolF& t, RefVec<16 / Traits<DT>::ESZ>& o,
                                           uint32_t& flags) {
@@ -394,19 +393,22 @@ __device__ __forceinline__ void hoist_ref(const uint4& raw, const TolF& t, RefVe
     Widen<DT>::run(raw, o.rf);
     // tol is a monotone function of |r| (two correctly rounded monotone steps), so the smallest tol of
     // the vector is the tol of its smallest |r|. fminf skips NaNs: a NaN element makes d NaN anyway.
-    uint32_t umax = 0u, umin1 = 0xFFFFFFFFu;
     float amin = __uint_as_float(0x7F800000u);
 #pragma unroll
-    for (int e = 0; e < EPV; ++e) {
-        const float a = fabsf(o.rf[e]);
-        const uint32_t u = __float_as_uint(a);
-        amin = fminf(amin, a);
-        umax = u > umax ? u : umax;
-        umin1 = (u - 1u) < umin1 ? (u - 1u) : umin1;                  // u == 0 wraps to the top: ignored
+    for (int e = 0; e < EPV; ++e) amin = fminf(amin, fabsf(o.rf[e]));
+    o.tolmin = tolc_of(amin, t);
+    // A nonzero element below 2^-64 can only exist when the smallest |r| is below 2^-64 (it may be a
+    // zero, so look at the elements then; f16 has no nonzero value that small).
+    flags = 0u;
+    if (DT != GV_F16 && __float_as_uint(amin) < kTinyBits) {
+        uint32_t umin1 = 0xFFFFFFFFu;
+#pragma unroll
+        for (int e = 0; e < EPV; ++e) {
+            const uint32_t u1 = (__float_as_uint(o.rf[e]) & 0x7FFFFFFFu) - 1u;   // zero wraps to the top: ignored
+            umin1 = u1 < umin1 ? u1 : umin1;
+        }
+        flags = (umin1 < kTinyBits - 1u) ? 2u : 0u;
     }
-    const float tolmin = tolc_of(amin, t);
-    o.tolmin = tolmin;
-    flags = ((umax > 0x7F800000u && !t.equal_nan) ? 1u : 0u) | ((umin1 < kTinyBits - 1u) ? 2u : 0u);
 }
 
 // Relative-error filter of one (CTA, candidate). M = largest exact quotient recorded so far;

@@ -256,6 +256,49 @@ def test_results_independent_of_schedule(oracle):
 
 
 # ------------------------------------------------------------------------------------------------
+# differing vectors at every density: from none to all 32 lanes of a warp-tile, several tiles per warp
+# ------------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("code,equal_nan", [(1, True), (0, False), (2, True), (3, False)])
+def test_differing_lane_densities(oracle, code, equal_nan):
+    """Candidate j differs from the reference in a fraction j/15 of its 16-byte vectors, so the
+    kernel meets visits with anything from 0 to 32 differing lanes (queued and in-place compares,
+    queue wrap-around, drains at chunk ends). The differing vectors mix noise inside the tolerance,
+    plain mismatches and, for float dtypes, NaN/Inf, and the reference itself holds a few NaNs."""
+    g = torch.Generator().manual_seed(4242 + code)
+    n = 6 * (1 << 20) + 1000 if ESZ[code] == 2 else 3 * (1 << 20) + 1000
+    epv = 16 // ESZ[code]
+    nv = n // epv
+    if code == 3:
+        r = torch.randint(-(1 << 20), 1 << 20, (n,), generator=g, dtype=torch.int32)
+    else:
+        r = torch.randn(n, generator=g).to(TDT[code])
+        r[torch.randint(0, n, (64,), generator=g)] = float("nan")
+    cands = []
+    for j in range(16):
+        pick = torch.rand(nv, generator=g) < (j / 15.0)
+        elem = pick.repeat_interleave(epv)
+        elem = torch.cat([elem, torch.zeros(n - nv * epv, dtype=torch.bool)])
+        elem &= torch.rand(n, generator=g) < 0.6                      # not every element of a picked vector
+        c = r.clone()
+        if code == 3:
+            c[elem] += torch.randint(1, 5, (int(elem.sum()),), generator=g, dtype=torch.int32)
+        else:
+            kind = torch.rand(n, generator=g)
+            rf = r.float()
+            small = (rf * (1 + 2e-3 * torch.randn(n, generator=g))).to(TDT[code])
+            big = (rf + 1.0).to(TDT[code])
+            c = torch.where(elem & (kind < 0.9), small, c)
+            c = torch.where(elem & (kind >= 0.9) & (kind < 0.995), big, c)
+            c = torch.where(elem & (kind >= 0.995) & (kind < 0.998), torch.full_like(c, float("inf")), c)
+            c = torch.where(elem & (kind >= 0.998), torch.full_like(c, float("nan")), c)
+        cands.append(c)
+    got, rh = run_dense(r.to(DEV), [c.to(DEV) for c in cands], 1e-2, 1e-2, equal_nan)
+    want = oracle_batch(oracle, r, cands, code, 1e-2, 1e-2, equal_nan)
+    assert_records_equal(got, want, f"densities dtype {code}")
+    assert rh == oracle.hash_bytes(host_bytes(r))
+
+
+# ------------------------------------------------------------------------------------------------
 # reduced versions of the dense workload recipes
 # ------------------------------------------------------------------------------------------------
 def test_reduced_configs_2_3_4(oracle):

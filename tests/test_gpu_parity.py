@@ -522,3 +522,65 @@ def test_randomised_ragged(oracle, seed):
     want = oracle.verify_ragged(ref_buf.numpy(), ref_off_t.numpy(), cand_buf.numpy(), cand_off_t.numpy(),
                                 dtypes_t.numpy(), N, atol, rtol, en, n_elems=n_el.numpy())
     assert_records_equal(gv.results_to_numpy(res), want, f"ragged seed {seed} T {T} N {N} align {align}")
+
+
+def test_ragged_differing_lane_densities(oracle):
+    """A few large tensors of every dtype, five candidates each with a differing-vector fraction of
+    0, 1/4, 1/2, 3/4 and 1: warps stream many tiles of one tensor, their queues of differing vectors
+    fill, wrap around and are drained when the warp leaves the tensor."""
+    g = torch.Generator().manual_seed(777)
+    N, T = 5, 10
+    sizes = [(1 << 20) + 77, (1 << 19) + 5, 3 * (1 << 18), (1 << 20) - 3, (1 << 18) + 1, 40000, (1 << 19), 999999,
+             (1 << 17) + 9, 1 << 20]
+    codes = [0, 1, 2, 3, 4, 1, 0, 2, 3, 1]
+    refs, cands = [], []
+    for t in range(T):
+        code, n = codes[t], sizes[t]
+        if code >= 3:
+            r = torch.randint(-(1 << 20), 1 << 20, (n,), generator=g, dtype=TDT[code])
+        else:
+            r = torch.randn(n, generator=g).to(TDT[code])
+            r[torch.randint(0, n, (16,), generator=g)] = float("nan")
+        refs.append(r)
+        epv = 16 // ESZ[code]
+        for j in range(N):
+            pick = (torch.rand(n // epv + 1, generator=g) < j / 4.0).repeat_interleave(epv)[:n]
+            pick &= torch.rand(n, generator=g) < 0.5
+            if code >= 3:
+                c = torch.where(pick, r + 3, r)
+            else:
+                kind = torch.rand(n, generator=g)
+                c = torch.where(pick & (kind < 0.9), (r.float() * (1 + 2e-3 * torch.randn(n, generator=g))).to(TDT[code]), r)
+                c = torch.where(pick & (kind >= 0.9) & (kind < 0.997), (r.float() - 2.0).to(TDT[code]), c)
+                c = torch.where(pick & (kind >= 0.997), torch.full_like(c, float("-inf")), c)
+            cands.append(c)
+    ref_off, cand_off, rc, cc = [], [], 0, 0
+    for t in range(T):
+        nb = sizes[t] * ESZ[codes[t]]
+        rc = (rc + 15) // 16 * 16
+        ref_off.append(rc)
+        rc += nb
+        for j in range(N):
+            cc = (cc + 15) // 16 * 16
+            cand_off.append(cc)
+            cc += nb
+    ref_off.append(rc)
+    ref_buf = torch.zeros(rc, dtype=torch.uint8)
+    cand_buf = torch.zeros(cc, dtype=torch.uint8)
+    for t in range(T):
+        nb = sizes[t] * ESZ[codes[t]]
+        ref_buf[ref_off[t]:ref_off[t] + nb] = refs[t].view(torch.uint8)
+        for j in range(N):
+            o = cand_off[t * N + j]
+            cand_buf[o:o + nb] = cands[t * N + j].view(torch.uint8)
+    ref_off_t, cand_off_t = torch.tensor(ref_off), torch.tensor(cand_off)
+    dtypes_t, n_el = torch.tensor(codes, dtype=torch.uint8), torch.tensor(sizes)
+    for en in (False, True):
+        ws = torch.empty(gv.gv_workspace_bytes(T, N), dtype=torch.uint8, device=DEV)
+        res = gv.gv_verify_ragged(ref_buf.to(DEV), ref_off_t.to(DEV), cand_buf.to(DEV), cand_off_t.to(DEV),
+                                  dtypes_t.to(DEV), N, 1e-2, 1e-2, en, n_elems=n_el.to(DEV), workspace=ws)
+        torch.cuda.synchronize()
+        assert gv.gv_check(ws) == gv.GV_OK
+        want = oracle.verify_ragged(ref_buf.numpy(), ref_off_t.numpy(), cand_buf.numpy(), cand_off_t.numpy(),
+                                    dtypes_t.numpy(), N, 1e-2, 1e-2, en, n_elems=n_el.numpy())
+        assert_records_equal(gv.results_to_numpy(res), want, f"ragged densities equal_nan {en}")

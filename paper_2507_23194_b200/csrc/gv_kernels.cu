@@ -690,8 +690,8 @@ struct RaggedSmem {
     static constexpr size_t kRingOff = 0;                                                  // [warp][kRing][32] uint4
     static constexpr size_t kSlotOff = kRingOff + size_t(kWarps) * kRing * kWarpTile;      // [warp][kChunk][32] u64
     static constexpr size_t kAccOff = kSlotOff + size_t(kWarps) * kChunk * 32 * 8;         // [warp][kChunk] CtaAcc
-    static constexpr size_t kPtrOff = kAccOff + size_t(kWarps) * kChunk * sizeof(CtaAcc);  // [warp][kChunk] candidate pointers
-    static constexpr size_t kQueueOff = kPtrOff + size_t(kWarps) * kChunk * 8;             // [warp][3][kQCap] uint4
+    static constexpr size_t kPtrOff = kAccOff + size_t(kWarps) * kChunk * sizeof(CtaAcc);  // [warp][kChunk + 2] reference + candidate pointers
+    static constexpr size_t kQueueOff = kPtrOff + size_t(kWarps) * (kChunk + 2) * 8;       // [warp][3][kQCap] uint4
     static constexpr size_t kTotal = kQueueOff + size_t(kWarps) * kQueueBytes;
 };
 
@@ -798,8 +798,9 @@ __device__ __forceinline__ bool vec_has_nan(int dt, const uint4& r) {
 // unaligned tensors use synchronous element-sized loads.
 __device__ __forceinline__ void ragged_stretch(const RaggedParams& p, int dt, const unsigned char* ref, uint64_t n,
                                                uint64_t tile_begin, uint64_t tile_end, int kg, uint2* slots,
-                                               CtaAcc* wacc, const unsigned char* const* wptr, int lane,
+                                               CtaAcc* wacc, const unsigned char* const* wsrc, int lane,
                                                uint32_t ring_base, uint32_t qbase) {
+    const unsigned char* const* wptr = wsrc + 1;        // wsrc[0] = the reference, wsrc[1 + k] = candidate k
     const int esz = elem_size(dt);
     const uint64_t nbytes = n * esz;
     const TolF tol = {p.atol, p.rtol, p.equal_nan};
@@ -852,39 +853,43 @@ __device__ __forceinline__ void ragged_stretch(const RaggedParams& p, int dt, co
 
     if (full_end > tile_begin) {
         // ---- streamed part ----
-        const uint32_t per_tile = static_cast<uint32_t>(kg) + 1u;       // reference + candidates
-        uint64_t issue_tile = tile_begin;
-        int issue_j = -1;                                               // -1: reference, else candidate index
-        uint32_t issue_stage = 0;
-        auto issue_one = [&]() {
-            if (issue_tile < full_end) {
-                const unsigned char* base = issue_j < 0 ? ref : wptr[issue_j];
-                cp_async16(ring_base + issue_stage * 512u, base + issue_tile * kWarpTile + lane * 16);
-                issue_stage = (issue_stage + 1u) & (kRing - 1);
-                if (++issue_j == kg) { issue_j = -1; ++issue_tile; }
+        // The copies form one sequence: per tile the reference vector, then the kg candidate vectors.
+        // The stage a visit has just consumed is refilled at once with the copy kRing places ahead,
+        // so consumer and producer share one stage counter. src[0] is the reference, src[1 + k]
+        // candidate k (wsrc, one table per warp in shared memory).
+        const uint64_t end_off = full_end * kWarpTile;
+        uint64_t issue_off = tile_begin * kWarpTile + lane * 16;        // this lane's byte offset of the next copy
+        int issue_j = 0;
+        auto issue_one = [&](uint32_t stage_addr) {
+            if (issue_off < end_off) {
+                cp_async16(stage_addr, wsrc[issue_j] + issue_off);
+                const bool wrap = issue_j == kg;
+                issue_j = wrap ? 0 : issue_j + 1;
+                issue_off += wrap ? kWarpTile : 0;
             }
             cp_async_commit();
         };
-        (void)per_tile;
 #pragma unroll 1
-        for (int j = 0; j < kRing; ++j) issue_one();
+        for (int j = 0; j < kRing; ++j) issue_one(ring_base + j * 512u);
         uint32_t stage = 0;
 #pragma unroll 1
         for (uint64_t tile = tile_begin; tile < full_end; ++tile) {
             const uint64_t voff = tile * kWarpTile + lane * 16;
             cp_async_wait<kRing - 1>();
-            const uint4 r = lds128(ring_base + stage * 512u);
+            uint32_t at = ring_base + stage * 512u;
+            const uint4 r = lds128(at);
             stage = (stage + 1u) & (kRing - 1);
-            issue_one();
+            issue_one(at);
             const bool force = nan_matters && vec_has_nan(dt, r);
             const uint64_t h_ref = hash_vec_full(r, voff / 8);
             ref_sum += h_ref;
 #pragma unroll 1
             for (int k = 0; k < kg; ++k) {
                 cp_async_wait<kRing - 1>();
-                const uint4 c = lds128(ring_base + stage * 512u);
+                at = ring_base + stage * 512u;
+                const uint4 c = lds128(at);
                 stage = (stage + 1u) & (kRing - 1);
-                issue_one();
+                issue_one(at);
                 queued_visit(c, r, h_ref, force, voff, k);
             }
         }
@@ -930,7 +935,7 @@ __global__ void __launch_bounds__(kThreads, 2) ragged_kernel(const __grid_consta
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     uint2* slots = reinterpret_cast<uint2*>(smem + RaggedSmem::kSlotOff) + size_t(warp) * kChunk * 32 + lane;
     CtaAcc* wacc = reinterpret_cast<CtaAcc*>(smem + RaggedSmem::kAccOff) + warp * kChunk;
-    const unsigned char** wptr = reinterpret_cast<const unsigned char**>(smem + RaggedSmem::kPtrOff) + warp * kChunk;
+    const unsigned char** wsrc = reinterpret_cast<const unsigned char**>(smem + RaggedSmem::kPtrOff) + warp * (kChunk + 2);
     const uint32_t ring_base = smem_u32(smem + RaggedSmem::kRingOff) + (warp * kRing * 32 + lane) * 16;
     const uint32_t qbase = smem_u32(smem + RaggedSmem::kQueueOff) + warp * static_cast<uint32_t>(kQueueBytes);
 
@@ -966,12 +971,13 @@ __global__ void __launch_bounds__(kThreads, 2) ragged_kernel(const __grid_consta
             const int kg = min(kChunk, p.N - c0);
             __syncwarp();
             if (lane < kg) {
-                wptr[lane] = p.cand_base + p.cand_off[t * p.N + c0 + lane];
+                wsrc[1 + lane] = p.cand_base + p.cand_off[t * p.N + c0 + lane];
                 wacc[lane].clear();
             }
+            if (lane == 0) wsrc[0] = ref;
             for (int k = 0; k < kg; ++k) slots[k * 32] = make_uint2(0u, 0u);
             __syncwarp();
-            ragged_stretch(p, dt, ref, n, tile_begin, tile_end, kg, slots, wacc, wptr, lane, ring_base, qbase);
+            ragged_stretch(p, dt, ref, n, tile_begin, tile_end, kg, slots, wacc, wsrc, lane, ring_base, qbase);
             __syncwarp();
             // leave the tensor (or this group of its candidates): combine and publish
             for (int k = 0; k < kg; ++k) {

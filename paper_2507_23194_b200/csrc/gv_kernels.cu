@@ -492,21 +492,20 @@ dense_kernel(const __grid_constant__ DenseParams p) {
                     voff += tile_stride;
                 }
             } else {
-                // ---- partial chunk (fewer than 16 candidates): same ring, generic bookkeeping
-                const uint64_t visits = static_cast<uint64_t>(my_tiles) * kg;
+                // ---- partial chunk (fewer than 16 candidates): same ring, one visit at a time. The stage a
+                // visit has just consumed is refilled at once with the copy kRing visits ahead.
                 uint64_t issue_off = voff;
                 int issue_k = 0;
-                uint64_t issued = 0;
-                auto issue_one = [&]() {
-                    if (issued < visits) {
-                        cp_async16(ring_base + (static_cast<uint32_t>(issued) & (kRing - 1)) * 512u, p.cands[cand0 + issue_k] + issue_off);
-                        ++issued;
-                        if (++issue_k == kg) { issue_k = 0; issue_off += tile_stride; }
+                uint32_t tiles_left = my_tiles;            // tiles whose copies have not all been issued
+                auto issue_one = [&](uint32_t stage_addr) {
+                    if (tiles_left) {
+                        cp_async16(stage_addr, p.cands[cand0 + issue_k] + issue_off);
+                        if (++issue_k == kg) { issue_k = 0; issue_off += tile_stride; --tiles_left; }
                     }
                     cp_async_commit();          // one group per visit, possibly empty near the end
                 };
 #pragma unroll 1
-                for (int j = 0; j < kRing; ++j) issue_one();
+                for (int j = 0; j < kRing; ++j) issue_one(ring_base + j * 512u);
                 uint32_t stage = 0;
 #pragma unroll 1
                 for (uint32_t i = 0; i < my_tiles; ++i) {
@@ -518,9 +517,10 @@ dense_kernel(const __grid_constant__ DenseParams p) {
 #pragma unroll 1
                     for (int k = 0; k < kg; ++k) {
                         cp_async_wait<kRing - 1>();
-                        const uint4 c = lds128(ring_base + stage * 512u);
+                        const uint32_t at = ring_base + stage * 512u;
+                        const uint4 c = lds128(at);
                         stage = (stage + 1) & (kRing - 1);
-                        issue_one();
+                        issue_one(at);
                         visit(c, r, k);
                     }
                     voff += tile_stride;

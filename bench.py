@@ -47,10 +47,10 @@ def _scaled(measured, ref_bytes, cap_cands, full_cands):
 
 
 NCU_TRAFFIC_BYTES = {
-    "cfg2": _scaled(2.282e9 + 6.5e6, 33554432, 64, 256),      # profiles/dense_kernel_bf16_cfg2.md
-    "cfg3": _scaled(2.416e9 + 3.8e6, 268435456, 8, 32),       # profiles/dense_kernel_f16_cfg3.md
-    "cfg4": _scaled(2.416e9 + 8.3e6, 268435456, 8, 64),       # profiles/dense_kernel_i32_cfg4.md
-    "cfg5": (2.289e9 + 11.9e6) * 10000 / 2000,                # profiles/ragged_kernel_cfg5.md (2000 of 10000 tensors)
+    "cfg2": _scaled(2.282e9 + 5.5e6, 33554432, 64, 256),      # profiles/dense_kernel_bf16_cfg2.md
+    "cfg3": _scaled(4.563e9 + 5.3e6, 268435456, 16, 32),      # profiles/dense_kernel_f16_cfg3.md
+    "cfg4": _scaled(4.564e9 + 6.7e6, 268435456, 16, 64),      # profiles/dense_kernel_i32_cfg4.md
+    "cfg5": (2.291e9 + 11.3e6) * 10000 / 2000,                # profiles/ragged_kernel_cfg5.md (2000 of 10000 tensors)
 }
 
 
@@ -347,7 +347,7 @@ def main():
     algo_bytes = cand_bytes + ref_bytes + 64 * (wl.T * wl.N if ragged else n_cands)
     kernel_ms = statistics.median(step_ms)
     achieved = algo_bytes / (kernel_ms * 1e-3) / 1e9
-    roofline = {"bound": "hbm", "co_bound": "alu (integer pipes of the content hash: ceiling about 7.3 TB/s for the hash alone, see profiles/instruction_rates_b200.md)",
+    roofline = {"bound": "hbm", "co_bound": "alu (vectors identical to the reference stream at HBM rate; vectors that differ pay the integer work of the content hash, about 7.3 TB/s for the hash alone, and the compare: see profiles/instruction_rates_b200.md)",
                 "kernel": "ragged_kernel" if ragged else "dense_kernel",
                 "achieved": achieved, "peak": peak, "peak_kind": peak_kind + " (STREAM-style copy)",
                 "unit": "GB/s", "frac": achieved / peak, "traffic": NCU_TRAFFIC_BYTES.get(args.workload),

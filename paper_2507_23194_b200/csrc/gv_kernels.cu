@@ -95,10 +95,16 @@ struct DenseParams {
 //   * Candidates: each lane streams its own 16 bytes of every candidate with asynchronous 16-byte
 //     copies into a private ring in shared memory, kRing copies in flight per lane, and reads them
 //     back itself -- no registers are spent on data in flight and no barrier on its arrival.
-//   * Accumulators: the 64-bit hash partial of every (candidate of the chunk, lane) lives in a
-//     shared-memory slot for the whole chunk; max |d|, max relative error, counts and the first
-//     index go to per-CTA shared accumulators only when they can change them. One block combine
-//     and one set of global integer atomics per (CTA, candidate).
+//   * Hash: a candidate vector that is bit-identical to the reference vector has the reference
+//     vector's hash terms, so the lane hashes its reference vector once per tile and a 64-bit
+//     shared-memory slot per (candidate of the chunk, lane) only collects the corrections
+//     hash(c) - hash(r) of the vectors that differ.
+//   * Compare: identical vectors are done after the identity test. Differing vectors of sparse
+//     visits are queued per warp and compared 32 at a time, one per lane; visits in which most
+//     lanes differ are compared in place against values derived from the reference once per tile.
+//   * Accumulators: max |d|, max relative error, counts and the first index go to per-CTA shared
+//     accumulators only when they can change them. One block combine and one set of global
+//     integer atomics per (CTA, candidate).
 #ifndef GV_UNROLL
 #define GV_UNROLL 4
 #endif
@@ -137,8 +143,10 @@ struct DenseSmem {
     static constexpr size_t kTotal = kRefHashOff + 8;
 };
 
-// CTA shapes: integer kernels need ~72 registers and run 3 CTAs of 8 warps per SM; float kernels hold
-// the derived reference values as well and run 2 CTAs of GV_FLOAT_WARPS warps within the register file.
+// CTA shapes: 8 warps and about 98 KB of shared memory per CTA (ring 32, reference stages 8, hash slots
+// 32, queue 24, accumulators 1.3), hence 2 CTAs per SM for every dtype; the float kernels also need
+// the whole register file at that occupancy (up to 128 registers per thread); the integer ones are
+// compiled for 3 CTAs per SM, which keeps them at 80 registers.
 #ifndef GV_FLOAT_WARPS
 #define GV_FLOAT_WARPS 8
 #endif

@@ -19,7 +19,8 @@
 //
 // Every function here is pinned by tests/test_oracle_*.py against values fixed outside this
 // file (published SplitMix64 outputs, a hand-derived truth table, torch.isclose / numpy on the
-// host, closed forms and by-construction counts).
+// host, closed forms and by-construction counts; the grouping by a hand-worked example, its
+// degenerate cases and a dictionary of byte strings).
 
 #include <cstdint>
 #include <cstring>
@@ -246,6 +247,32 @@ int gvo_verify_ragged(const void* ref_base, const int64_t* ref_off, const void* 
             if (rc) return rc;
         }
     }
+    return 0;
+}
+
+// Grouping of duplicate candidates (the use the content hash is computed for: parallel sampling
+// of many generation runs per reference, Section 4.2 "parallel scaling", yields identical
+// candidates, which need to be examined only once). Two candidates belong to one group exactly
+// when their 64-byte records are identical byte for byte -- same content hash and same statistics.
+//   group_id[j]    = the smallest index i whose record equals record j (so the representative of a
+//                    group is its first member, and group_id[j] == j marks representatives)
+//   group_count[j] = number of members of the group when j is its representative, else 0
+//   *n_groups      = number of representatives
+// Written as the definition: a double loop over whole records.
+int gvo_group(const gvo_result* results, int64_t N, int32_t* group_id, int32_t* group_count,
+              int32_t* n_groups) {
+    int32_t groups = 0;
+    for (int64_t j = 0; j < N; ++j) group_count[j] = 0;
+    for (int64_t j = 0; j < N; ++j) {
+        int64_t first = j;
+        for (int64_t i = 0; i < j; ++i) {
+            if (std::memcmp(&results[i], &results[j], sizeof(gvo_result)) == 0) { first = i; break; }
+        }
+        group_id[j] = static_cast<int32_t>(first);
+        group_count[first] += 1;
+        if (first == j) ++groups;
+    }
+    *n_groups = groups;
     return 0;
 }
 

@@ -77,6 +77,8 @@ def lib() -> ctypes.CDLL:
             ctypes.c_void_p, ctypes.c_int64, ctypes.c_int32, ctypes.c_double, ctypes.c_double, ctypes.c_int,
             ctypes.c_void_p,
         ]
+        L.gvo_group.restype = ctypes.c_int
+        L.gvo_group.argtypes = [ctypes.c_void_p, ctypes.c_int64, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
         _lib = L
     return _lib
 
@@ -157,3 +159,16 @@ def verify_ragged(ref_buf: np.ndarray, ref_off: np.ndarray, cand_buf: np.ndarray
     if rc != 0:
         raise ValueError("oracle rejected a dtype code in the ragged batch")
     return out
+
+
+def group(records: np.ndarray):
+    """Duplicate groups of N result records -> (group_id[N] int32, group_count[N] int32, n_groups)."""
+    rec = np.ascontiguousarray(records, dtype=RESULT_DTYPE)
+    n = rec.shape[0]
+    gid = np.zeros(max(n, 1), dtype=np.int32)
+    cnt = np.zeros(max(n, 1), dtype=np.int32)
+    ng = np.zeros(1, dtype=np.int32)
+    rc = lib().gvo_group(rec.ctypes.data, n, gid.ctypes.data, cnt.ctypes.data, ng.ctypes.data)
+    if rc:
+        raise RuntimeError(f"gvo_group failed with {rc}")
+    return gid[:n], cnt[:n], int(ng[0])

@@ -443,3 +443,67 @@ def test_config5_reduced_by_construction(oracle, align):
         tight = all(int(wl.ref_off[t + 1] - wl.ref_off[t]) == wl.n_elems[t] * esz[int(wl.dtypes[t])] for t in range(wl.T))
         if tight:
             assert res2.tobytes() == res.tobytes()
+
+
+# --------------------------------------------------------------------------------------------
+# grouping of duplicate candidates
+# --------------------------------------------------------------------------------------------
+def _records(rows):
+    """rows: tuples (n_mismatch, first, n_nan, n_inf, hash, maxint, maxabs, maxrel)."""
+    from oracle import gv_oracle as O
+    rec = np.zeros(len(rows), dtype=O.RESULT_DTYPE)
+    for j, r in enumerate(rows):
+        (rec[j]["n_mismatch"], rec[j]["first_mismatch"], rec[j]["n_nan_disagree"], rec[j]["n_inf_disagree"],
+         rec[j]["hash"], rec[j]["max_abs_diff_int"], rec[j]["max_abs_err"], rec[j]["max_rel_err"]) = r
+    return rec
+
+
+def test_group_hand_worked_example(oracle):
+    # seven candidates: A B A C B A D  ->  groups {0,2,5} {1,4} {3} {6}
+    A = (0, M64, 0, 0, 0x1111, 0, 0.0, 0.0)
+    B = (3, 17, 0, 0, 0x2222, 0, 0.5, 0.25)
+    C = (3, 17, 0, 0, 0x2222, 0, 0.5, 0.125)        # same hash and counts as B, one statistic differs
+    D = (0, M64, 0, 0, 0x1112, 0, 0.0, 0.0)         # differs from A in one bit of the hash
+    gid, cnt, ng = oracle.group(_records([A, B, A, C, B, A, D]))
+    assert gid.tolist() == [0, 1, 0, 3, 1, 0, 6]
+    assert cnt.tolist() == [3, 2, 0, 1, 0, 0, 1]
+    assert ng == 4
+
+
+def test_group_degenerate_cases(oracle):
+    gid, cnt, ng = oracle.group(_records([]))
+    assert gid.size == 0 and cnt.size == 0 and ng == 0
+    one = (1, 2, 3, 4, 5, 6, 7.0, 8.0)
+    gid, cnt, ng = oracle.group(_records([one] * 9))
+    assert gid.tolist() == [0] * 9 and cnt.tolist() == [9] + [0] * 8 and ng == 1
+    distinct = [(0, M64, 0, 0, h, 0, 0.0, 0.0) for h in range(12)]
+    gid, cnt, ng = oracle.group(_records(distinct))
+    assert gid.tolist() == list(range(12)) and cnt.tolist() == [1] * 12 and ng == 12
+    # -0.0 and +0.0 in a float field are different bytes, hence different records
+    gid, _, ng = oracle.group(_records([(0, M64, 0, 0, 9, 0, 0.0, 0.0), (0, M64, 0, 0, 9, 0, -0.0, 0.0)]))
+    assert gid.tolist() == [0, 1] and ng == 2
+
+
+@pytest.mark.parametrize("seed", [0, 1, 2])
+def test_group_against_python_dict(oracle, seed):
+    # independent restatement: first index of each distinct byte string, via a dict
+    rng = np.random.default_rng(seed)
+    from oracle import gv_oracle as O
+    pool = rng.integers(0, 256, size=(40, 64), dtype=np.uint8)
+    pick = rng.integers(0, 40, size=500)
+    rec = pool[pick].copy().view(O.RESULT_DTYPE).reshape(-1)
+    gid, cnt, ng = oracle.group(rec)
+    first = {}
+    want = []
+    for j in range(500):
+        want.append(first.setdefault(rec[j].tobytes(), j))
+    assert gid.tolist() == want
+    assert ng == len(first)
+    for j in range(500):
+        assert cnt[j] == (want.count(j) if want[j] == j else 0)
+    # relabelling invariance: reversing the order maps each group onto the same member set
+    gid_r, _, ng_r = oracle.group(rec[::-1].copy())
+    assert ng_r == ng
+    groups = {frozenset(np.nonzero(gid == g)[0].tolist()) for g in set(gid.tolist())}
+    groups_r = {frozenset((499 - np.nonzero(gid_r == g)[0]).tolist()) for g in set(gid_r.tolist())}
+    assert groups == groups_r

@@ -163,6 +163,28 @@ gv_status gv_verify_ragged_noalloc(const void* ref_base, const int64_t* ref_off,
  * The same function the verifier applies to each candidate (used to de-duplicate candidates). */
 gv_status gv_hash(const void* buf, uint64_t nbytes, uint64_t* out, void* cuda_stream);
 
+/* Groups of duplicate candidates (what the content hash is for: the paper's parallel scaling,
+ * Section 4.2, samples many generation runs per reference, and identical candidates need to be
+ * examined only once). Candidates i and j are duplicates exactly when their 64-byte records are
+ * identical byte for byte: same content hash and same statistics against the reference.
+ *   results      device, N records as a verify call wrote them (read only, 16-byte aligned).
+ *   group_id     device, int32[N]: the smallest index whose record equals record j. Representatives
+ *                are the j with group_id[j] == j.
+ *   group_count  device, int32[N], nullable: size of the group at its representative's index, 0
+ *                elsewhere.
+ *   n_groups     device, int32[1], nullable: number of groups.
+ *   workspace    device, >= gv_group_workspace_bytes(N) bytes, 16-byte aligned; carries a status word
+ *                for gv_check() (GV_ERR_DEVICE_TIMEOUT would mean a bounded table probe gave up, which
+ *                the table's load factor of at most 1/2 rules out).
+ * N == 0 is legal (n_groups = 0). N > GV_GROUP_MAX returns GV_ERR_UNSUPPORTED and enqueues nothing.
+ * Up to 2048 records are grouped by one launch with the table in shared memory; beyond that the
+ * table lives in the workspace and the call enqueues three launches. The outputs do not depend on
+ * thread scheduling. Enqueue it on the stream of the verify call that writes `results`. */
+#define GV_GROUP_MAX (1ll << 28)
+size_t gv_group_workspace_bytes(int64_t N);
+gv_status gv_group_candidates(const gv_result* results, int64_t N, int32_t* group_id, int32_t* group_count,
+                              int32_t* n_groups, void* workspace, size_t workspace_bytes, void* cuda_stream);
+
 /* Host-buffer convenience for callers whose outputs live in host memory: copies the reference and
  * the candidates host->device in slabs through `staging` (device, staging_bytes), verifies them and
  * copies the N records (and the reference hash) back to host memory. Copies and kernels are

@@ -17,6 +17,7 @@
 
 #include "gv.h"
 #include "gv_device.cuh"
+#include "gv_group.cuh"
 
 namespace gv {
 
@@ -1333,6 +1334,57 @@ gv_status gv_hash(const void* buf, uint64_t nbytes, uint64_t* out, void* cuda_st
 
 static size_t round256(size_t x) { return (x + 255) / 256 * 256; }
 
+// ---- grouping of duplicate candidates ----
+static uint32_t group_slots(int64_t N) {
+    uint32_t s = 16;
+    while (static_cast<int64_t>(s) < 2 * N) s <<= 1;
+    return s;
+}
+size_t gv_group_workspace_bytes(int64_t N) {
+    if (N < 0 || N > GV_GROUP_MAX) return 0;
+    return 256 + (N > gv::kGroupFusedMax ? static_cast<size_t>(group_slots(N)) * 8 : 0);
+}
+gv_status gv_group_candidates(const gv_result* results, int64_t N, int32_t* group_id, int32_t* group_count,
+                              int32_t* n_groups, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    if (N < 0 || (N > 0 && (!results || !group_id))) return GV_ERR_INVALID_ARG;
+    if (N > GV_GROUP_MAX) {
+        snprintf(g_last_error, sizeof(g_last_error), "gv_group_candidates: N = %lld exceeds GV_GROUP_MAX = %lld",
+                 static_cast<long long>(N), static_cast<long long>(GV_GROUP_MAX));
+        return GV_ERR_UNSUPPORTED;
+    }
+    if (reinterpret_cast<uintptr_t>(results) & 15u) return GV_ERR_MISALIGNED;
+    if ((reinterpret_cast<uintptr_t>(group_id) & 3u) || (reinterpret_cast<uintptr_t>(group_count) & 3u) ||
+        (reinterpret_cast<uintptr_t>(n_groups) & 3u))
+        return GV_ERR_MISALIGNED;
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 15u) || workspace_bytes < gv_group_workspace_bytes(N))
+        return GV_ERR_WORKSPACE;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    gv::GroupParams p;
+    p.results = results;
+    p.N = N;
+    p.group_id = group_id;
+    p.group_count = group_count;
+    p.n_groups = n_groups;
+    p.status = static_cast<uint32_t*>(workspace);
+    p.slots = group_slots(N);
+    p.owner = reinterpret_cast<int*>(static_cast<unsigned char*>(workspace) + 256);
+    p.min_index = p.owner + p.slots;
+    if (N <= gv::kGroupFusedMax) {
+        gv::group_fused_kernel<<<1, gv::kGroupThreads, 0, st>>>(p);     // also covers N == 0: clears n_groups and the status
+    } else {
+        int sm_count = 0;
+        gv_status rc = device_info(&sm_count);
+        if (rc != GV_OK) return rc;
+        const long long want = (static_cast<long long>(p.slots) + gv::kGroupThreads - 1) / gv::kGroupThreads;
+        const unsigned grid = static_cast<unsigned>(want < 8LL * sm_count ? want : 8LL * sm_count);
+        gv::group_clear_kernel<<<grid, gv::kGroupThreads, 0, st>>>(p);
+        gv::group_insert_kernel<<<grid, gv::kGroupThreads, 0, st>>>(p);
+        gv::group_finish_kernel<<<grid, gv::kGroupThreads, 0, st>>>(p);
+    }
+    GV_CUDA(cudaGetLastError());
+    return GV_OK;
+}
+
 size_t gv_host_staging_bytes(uint64_t n_elems, gv_dtype dt, int32_t slab) {
     const int esz = gv::elem_size(dt);
     if (esz == 0 || slab < 1) return 0;
@@ -1402,6 +1454,7 @@ gv_status gv_check(const void* workspace, void* cuda_stream) {
     GV_CUDA(cudaStreamSynchronize(st));
     if (word & gv::kStatusTimeout) return GV_ERR_DEVICE_TIMEOUT;
     if (word & gv::kStatusBadTable) return GV_ERR_BAD_TABLE;
+    if (word & gv::kStatusGroupOverflow) return GV_ERR_DEVICE_TIMEOUT;      // a bounded probe gave up
     return GV_OK;
 }
 

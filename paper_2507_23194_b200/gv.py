@@ -37,7 +37,8 @@ class gv_tol(ctypes.Structure):
                 ("equal_nan", ctypes.c_int32), ("reserved", ctypes.c_int32)]
 
 
-EXPORTS = ["gv_verify_batch", "gv_verify_ragged", "gv_verify_ragged_noalloc", "gv_hash", "gv_verify_batch_host", "gv_host_staging_bytes",
+EXPORTS = ["gv_verify_batch", "gv_verify_ragged", "gv_verify_ragged_noalloc", "gv_hash", "gv_group_candidates",
+           "gv_group_workspace_bytes", "gv_verify_batch_host", "gv_host_staging_bytes",
            "gv_workspace_bytes", "gv_check", "gv_status_string", "gv_last_cuda_error", "gv_version"]
 
 
@@ -57,6 +58,10 @@ def _load() -> ctypes.CDLL:
     L.gv_verify_ragged_noalloc.argtypes = [vp, vp, vp, vp, vp, vp, i64, i32, ctypes.POINTER(gv_tol), vp, vp, vp]
     L.gv_hash.restype = ctypes.c_int
     L.gv_hash.argtypes = [vp, u64, vp, vp]
+    L.gv_group_candidates.restype = ctypes.c_int
+    L.gv_group_candidates.argtypes = [vp, i64, vp, vp, vp, vp, sz, vp]
+    L.gv_group_workspace_bytes.restype = sz
+    L.gv_group_workspace_bytes.argtypes = [i64]
     L.gv_verify_batch_host.restype = ctypes.c_int
     L.gv_verify_batch_host.argtypes = [vp, vp, i32, u64, ctypes.c_int, ctypes.POINTER(gv_tol), vp, vp, vp, sz, vp]
     L.gv_host_staging_bytes.restype = sz
@@ -193,6 +198,31 @@ def gv_hash(buf: torch.Tensor, out: Optional[torch.Tensor] = None,
     rc = lib.gv_hash(buf.data_ptr(), buf.numel() * buf.element_size(), out.data_ptr(), _stream_ptr(stream))
     _raise(rc)
     return out
+
+
+def gv_group_workspace_bytes(N: int) -> int:
+    return int(lib.gv_group_workspace_bytes(N))
+
+
+def gv_group_candidates(results: torch.Tensor, group_id: Optional[torch.Tensor] = None,
+                        group_count: Optional[torch.Tensor] = None, n_groups: Optional[torch.Tensor] = None,
+                        workspace: Optional[torch.Tensor] = None, stream: Optional[torch.cuda.Stream] = None):
+    """Enqueue the grouping of the N records in ``results`` (device uint8 tensor of shape (N, 64));
+    returns device tensors (group_id int32[N], group_count int32[N], n_groups int32[1])."""
+    N = results.shape[0]
+    dev = results.device
+    if group_id is None:
+        group_id = torch.empty(max(N, 1), dtype=torch.int32, device=dev)
+    if group_count is None:
+        group_count = torch.empty(max(N, 1), dtype=torch.int32, device=dev)
+    if n_groups is None:
+        n_groups = torch.empty(1, dtype=torch.int32, device=dev)
+    if workspace is None:
+        workspace = torch.empty(gv_group_workspace_bytes(N), dtype=torch.uint8, device=dev)
+    rc = lib.gv_group_candidates(results.data_ptr(), N, group_id.data_ptr(), group_count.data_ptr(), n_groups.data_ptr(),
+                                 workspace.data_ptr(), workspace.numel(), _stream_ptr(stream))
+    _raise(rc)
+    return group_id[:N], group_count[:N], n_groups
 
 
 def gv_check(workspace: torch.Tensor, stream: Optional[torch.cuda.Stream] = None) -> int:

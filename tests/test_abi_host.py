@@ -103,3 +103,24 @@ def test_ragged_and_hash_argument_errors(gvlib):
     assert gv.lib.gv_hash(None, 16, 0x1000, None) == gv.GV_ERR_INVALID_ARG
     assert gv.lib.gv_hash(0x1000, 16, 0x1004, None) == gv.GV_ERR_MISALIGNED
     assert gv.lib.gv_check(None, None) == gv.GV_ERR_INVALID_ARG
+
+
+def test_group_argument_errors_return_before_any_launch(gvlib):
+    gv = gvlib
+    call = lambda res=0x1000, N=4, gid=0x2000, cnt=0x3000, ng=0x4000, ws=0x5000, wsb=4096: gv.lib.gv_group_candidates(
+        res, N, gid, cnt, ng, ws, wsb, None)
+    assert call(N=-1) == gv.GV_ERR_INVALID_ARG
+    assert call(res=None) == gv.GV_ERR_INVALID_ARG
+    assert call(gid=None) == gv.GV_ERR_INVALID_ARG
+    assert call(res=0x1008) == gv.GV_ERR_MISALIGNED
+    assert call(gid=0x2002) == gv.GV_ERR_MISALIGNED
+    assert call(ws=None) == gv.GV_ERR_WORKSPACE
+    assert call(ws=0x5004) == gv.GV_ERR_WORKSPACE
+    assert call(wsb=128) == gv.GV_ERR_WORKSPACE
+    assert call(N=5000, wsb=4096) == gv.GV_ERR_WORKSPACE            # beyond one CTA the table lives in the workspace
+    assert call(N=(1 << 28) + 1, wsb=1 << 40) == gv.GV_ERR_UNSUPPORTED
+    assert b"GV_GROUP_MAX" in gv.lib.gv_last_cuda_error()
+    assert gv.gv_group_workspace_bytes(0) == 256
+    assert gv.gv_group_workspace_bytes(2048) == 256
+    assert gv.gv_group_workspace_bytes(2049) == 256 + 8192 * 8
+    assert gv.gv_group_workspace_bytes(-1) == 0

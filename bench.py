@@ -359,6 +359,32 @@ def main():
         v, sample = time_oracle_sample(wl, 15.0)
         cpu_baseline = {"value": v, "unit": "GB/s", "cores": 1, "kind": "oracle", "sample": sample}
 
+    # ---- duplicate groups of the step's records (follow-on stage; outside the timed step) ----
+    n_rec = res.shape[0]
+    gws = torch.empty(gv.gv_group_workspace_bytes(n_rec), dtype=torch.uint8, device=device)
+    gid = torch.empty(max(n_rec, 1), dtype=torch.int32, device=device)
+    gcnt = torch.empty(max(n_rec, 1), dtype=torch.int32, device=device)
+    gn = torch.empty(1, dtype=torch.int32, device=device)
+    for _ in range(3):
+        gv.gv_group_candidates(res, gid, gcnt, gn, gws)
+    torch.cuda.synchronize()
+    g_ev = [torch.cuda.Event(enable_timing=True) for _ in range(21)]
+    g_ev[0].record(stream)
+    for i in range(20):
+        gv.gv_group_candidates(res, gid, gcnt, gn, gws)
+        g_ev[i + 1].record(stream)
+    torch.cuda.synchronize()
+    grouping = {"records": n_rec, "groups": int(gn.cpu()[0]),
+                "us_per_call": 1e3 * statistics.median(g_ev[i].elapsed_time(g_ev[i + 1]) for i in range(20)),
+                "launches_per_call": 1 if n_rec <= 2048 else 3}
+    if not args.no_cpu_baseline:
+        from oracle import gv_oracle as O
+        rec_np = gv.results_to_numpy(res)[:min(n_rec, 4096)]
+        t0 = time.perf_counter()
+        O.group(rec_np)
+        grouping["cpu_oracle_us"] = 1e6 * (time.perf_counter() - t0)
+        grouping["cpu_oracle_records"] = int(rec_np.shape[0])
+
     line = {
         "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
@@ -369,7 +395,7 @@ def main():
                    "parallelism": "independent replicas per GPU" if world > 1 else "one GPU"},
         "frac_of_measured_hbm": value / world / peak, "frac_of_nominal_8000": value / world / 8000.0,
         "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
-        "roofline": roofline, "cpu_baseline": cpu_baseline,
+        "roofline": roofline, "cpu_baseline": cpu_baseline, "grouping": grouping,
     }
     print(json.dumps(line))
     if dist is not None:

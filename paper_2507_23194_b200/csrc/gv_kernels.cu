@@ -129,7 +129,7 @@ constexpr int kQCap = 64;                           // entries (a power of two, 
 constexpr uint32_t kQPlane = kQCap * 16;            // bytes of one plane (candidate / reference / meta)
 constexpr size_t kQueueBytes = 3 * size_t(kQPlane);
 #ifndef GV_QDIRECT
-#define GV_QDIRECT 20                               // visits with at least this many differing lanes are compared in place
+#define GV_QDIRECT 18                               // visits with at least this many differing lanes are compared in place
 #endif
 
 template <int WARPS>

@@ -276,4 +276,113 @@ int gvo_group(const gvo_result* results, int64_t N, int32_t* group_id, int32_t* 
     return 0;
 }
 
+// Error profile of ONE candidate against the reference: the richer "error trace" an Evaluator can
+// hand to the Reflector when the functionality test fails (Section 4.1: the trace of a failing run
+// is fed back; Section 4.2, Reflexion) -- where the errors are and how large, not just that there
+// are some. The paper does not define such a profile; this is the reading used here, written out
+// element by element with the same close rule as gvo_verify:
+//   ulp_hist[b]   all n elements, by the distance between candidate and reference in units of the
+//                 dtype's own spacing: float dtypes order their bit patterns (negative values
+//                 mirrored, so -0 and +0 coincide and the distance counts representable values
+//                 in between); integer dtypes use |c - r|. b = 0: distance 0; b = 1 + floor(log2
+//                 distance) for distance >= 1 (b <= 64); b = 65: a NaN is involved.
+//   n_mismatch    elements that are not close (same as the record's)
+//   worst_*       the mismatching element with the largest error, ties to the smallest index.
+//                 Error of a float element: |fl(c - r)|, with NaN ranking above everything (bit
+//                 patterns compared as unsigned, NaN taken as all ones); of an integer: |c - r|.
+//   first_*       the (up to) 8 mismatching elements of smallest index, in order
+//   *_raw         the element's own bits, zero-extended
+//   rows          optional: mismatches per row of row_len elements (row i = elements
+//                 [i*row_len, (i+1)*row_len)), ceil(n / row_len) counters
+struct gvo_profile {
+    uint64_t ulp_hist[66];
+    uint64_t n_mismatch;
+    uint64_t worst_index;
+    uint64_t worst_c_raw, worst_r_raw;
+    uint64_t n_first;
+    uint64_t first_index[8];
+    uint64_t first_c_raw[8];
+    uint64_t first_r_raw[8];
+};
+
+int gvo_profile_pair(const void* ref, const void* cand, uint64_t n, int dtype, double atol, double rtol,
+                     int equal_nan, uint64_t row_len, gvo_profile* out, uint32_t* rows) {
+    const int esz = elem_size(dtype);
+    if (esz == 0) return 1;
+    gvo_profile p;
+    std::memset(&p, 0, sizeof(p));
+    p.worst_index = ~0ull;
+    for (int i = 0; i < 8; ++i) p.first_index[i] = ~0ull;
+    if (rows && row_len)
+        for (uint64_t i = 0; i < (n + row_len - 1) / row_len; ++i) rows[i] = 0;
+    const float atol_f = static_cast<float>(atol), rtol_f = static_cast<float>(rtol);
+    const float pos_inf = bits_to_float(0x7F800000u);
+    uint64_t worst_key = 0;
+    bool have_worst = false;
+
+    for (uint64_t i = 0; i < n; ++i) {
+        uint64_t c_raw = 0, r_raw = 0;
+        std::memcpy(&c_raw, static_cast<const char*>(cand) + esz * i, esz);      // little-endian host
+        std::memcpy(&r_raw, static_cast<const char*>(ref) + esz * i, esz);
+        bool close;
+        uint64_t key;        // error used to rank mismatches
+        int bucket;
+        if (dtype == I32 || dtype == I64) {
+            const int64_t c = dtype == I32 ? static_cast<int64_t>(static_cast<int32_t>(c_raw)) : static_cast<int64_t>(c_raw);
+            const int64_t r = dtype == I32 ? static_cast<int64_t>(static_cast<int32_t>(r_raw)) : static_cast<int64_t>(r_raw);
+            const uint64_t diff = (c > r) ? static_cast<uint64_t>(c) - static_cast<uint64_t>(r)
+                                          : static_cast<uint64_t>(r) - static_cast<uint64_t>(c);
+            close = (c == r);
+            key = diff;
+            bucket = 0;
+            for (uint64_t d = diff; d; d >>= 1) ++bucket;                          // 1 + floor(log2 diff)
+        } else {
+            float c, r;
+            const int width = esz * 8;
+            if (dtype == F32) { c = bits_to_float(static_cast<uint32_t>(c_raw)); r = bits_to_float(static_cast<uint32_t>(r_raw)); }
+            else if (dtype == BF16) { c = widen_bf16(static_cast<uint16_t>(c_raw)); r = widen_bf16(static_cast<uint16_t>(r_raw)); }
+            else { c = widen_f16(static_cast<uint16_t>(c_raw)); r = widen_f16(static_cast<uint16_t>(r_raw)); }
+            const float d = c - r;
+            const float ad = f_abs(d);
+            const float prod = rtol_f * f_abs(r);
+            const float tol = atol_f + prod;
+            const bool c_nan = is_nan(c), r_nan = is_nan(r);
+            close = (c == r);
+            if (equal_nan && c_nan && r_nan) close = true;
+            if (ad < pos_inf && ad <= tol) close = true;
+            key = is_nan(ad) ? 0xFFFFFFFFull : static_cast<uint64_t>(float_to_bits(ad));
+            if (c_nan || r_nan) {
+                bucket = 65;
+            } else {
+                const uint64_t sign_bit = 1ull << (width - 1);
+                const int64_t oc = (c_raw & sign_bit) ? -static_cast<int64_t>(c_raw & (sign_bit - 1)) : static_cast<int64_t>(c_raw);
+                const int64_t orf = (r_raw & sign_bit) ? -static_cast<int64_t>(r_raw & (sign_bit - 1)) : static_cast<int64_t>(r_raw);
+                const uint64_t dist = static_cast<uint64_t>(oc > orf ? oc - orf : orf - oc);
+                bucket = 0;
+                for (uint64_t dd = dist; dd; dd >>= 1) ++bucket;
+            }
+        }
+        p.ulp_hist[bucket] += 1;
+        if (!close) {
+            if (p.n_first < 8) {
+                p.first_index[p.n_first] = i;
+                p.first_c_raw[p.n_first] = c_raw;
+                p.first_r_raw[p.n_first] = r_raw;
+                p.n_first += 1;
+            }
+            p.n_mismatch += 1;
+            if (!have_worst || key > worst_key) {
+                have_worst = true;
+                worst_key = key;
+                p.worst_index = i;
+                p.worst_c_raw = c_raw;
+                p.worst_r_raw = r_raw;
+            }
+            if (rows && row_len) rows[i / row_len] += 1;
+        }
+    }
+    *out = p;
+    return 0;
+}
+
 }  // extern "C"

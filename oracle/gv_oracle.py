@@ -39,6 +39,23 @@ assert RESULT_DTYPE.itemsize == 64
 
 NO_INDEX = 0xFFFFFFFFFFFFFFFF
 
+PROFILE_BUCKETS = 66
+PROFILE_LIST = 8
+PROFILE_DTYPE = np.dtype(
+    [
+        ("ulp_hist", "<u8", (PROFILE_BUCKETS,)),
+        ("n_mismatch", "<u8"),
+        ("worst_index", "<u8"),
+        ("worst_c_raw", "<u8"),
+        ("worst_r_raw", "<u8"),
+        ("n_first", "<u8"),
+        ("first_index", "<u8", (PROFILE_LIST,)),
+        ("first_c_raw", "<u8", (PROFILE_LIST,)),
+        ("first_r_raw", "<u8", (PROFILE_LIST,)),
+    ]
+)
+assert PROFILE_DTYPE.itemsize == 8 * (66 + 5 + 24)
+
 
 def build(force: bool = False) -> str:
     """Compile the oracle into a shared object beside its source (a second or two with g++)."""
@@ -77,6 +94,9 @@ def lib() -> ctypes.CDLL:
             ctypes.c_void_p, ctypes.c_int64, ctypes.c_int32, ctypes.c_double, ctypes.c_double, ctypes.c_int,
             ctypes.c_void_p,
         ]
+        L.gvo_profile_pair.restype = ctypes.c_int
+        L.gvo_profile_pair.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_uint64, ctypes.c_int, ctypes.c_double,
+                                       ctypes.c_double, ctypes.c_int, ctypes.c_uint64, ctypes.c_void_p, ctypes.c_void_p]
         L.gvo_group.restype = ctypes.c_int
         L.gvo_group.argtypes = [ctypes.c_void_p, ctypes.c_int64, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
         _lib = L
@@ -172,3 +192,20 @@ def group(records: np.ndarray):
     if rc:
         raise RuntimeError(f"gvo_group failed with {rc}")
     return gid[:n], cnt[:n], int(ng[0])
+
+
+def profile(ref: np.ndarray, cand: np.ndarray, dtype: int, atol: float = 0.0, rtol: float = 0.0,
+            equal_nan: bool = False, row_len: int = 0):
+    """Error profile of one candidate -> (PROFILE_DTYPE scalar, per-row mismatch counts or None)."""
+    r, c = _as_bytes_array(ref), _as_bytes_array(cand)
+    assert r.nbytes == c.nbytes and r.nbytes % ELEM_SIZE[dtype] == 0
+    n = r.nbytes // ELEM_SIZE[dtype]
+    out = np.zeros(1, dtype=PROFILE_DTYPE)
+    rows = np.zeros(max(1, (n + row_len - 1) // row_len), dtype=np.uint32) if row_len else None
+    rc = lib().gvo_profile_pair(r.ctypes.data, c.ctypes.data, n, dtype, atol, rtol, int(equal_nan), row_len,
+                                out.ctypes.data, rows.ctypes.data if rows is not None else None)
+    if rc:
+        raise RuntimeError(f"gvo_profile_pair failed with {rc}")
+    if rows is not None:
+        rows = rows[:(n + row_len - 1) // row_len]
+    return out[0], rows

@@ -507,3 +507,115 @@ def test_group_against_python_dict(oracle, seed):
     groups = {frozenset(np.nonzero(gid == g)[0].tolist()) for g in set(gid.tolist())}
     groups_r = {frozenset((499 - np.nonzero(gid_r == g)[0]).tolist()) for g in set(gid_r.tolist())}
     assert groups == groups_r
+
+
+# --------------------------------------------------------------------------------------------
+# error profile of one candidate (ulp histogram, worst element, first mismatches, per-row counts)
+# --------------------------------------------------------------------------------------------
+def test_profile_hand_worked_example(oracle):
+    # element:        0     1      2      3      4           5
+    r = np.array([1.0, 2.0, -0.0, np.nan, 3.0, -1.0], dtype=np.float32)
+    c = np.array([1.0, 2.5, 0.0, 1.0, 3.0000002, 1.0], dtype=np.float32)
+    # distances: 0; 0x40200000-0x40000000 = 2^21 -> bucket 22; -0/+0 coincide -> 0; NaN -> bucket 65;
+    # next float after 3.0 -> 1 -> bucket 1; -1.0 to +1.0 = 2 * 0x3F800000 = 2^31 - 2^24 -> bucket 31
+    p, rows = oracle.profile(r, c, oracle.F32, 1e-3, 1e-3, False, row_len=4)
+    want = np.zeros(66, dtype=np.uint64)
+    want[0], want[22], want[65], want[1], want[31] = 2, 1, 1, 1, 1
+    assert p["ulp_hist"].tolist() == want.tolist()
+    assert int(p["n_mismatch"]) == 3                       # 2.5 vs 2, 1 vs NaN, 1 vs -1
+    assert int(p["worst_index"]) == 3                      # the NaN pair ranks above every finite error
+    assert int(p["worst_c_raw"]) == 0x3F800000 and int(p["worst_r_raw"]) == 0x7FC00000
+    assert int(p["n_first"]) == 3 and p["first_index"].tolist()[:3] == [1, 3, 5]
+    assert p["first_index"].tolist()[3:] == [oracle.NO_INDEX] * 5
+    assert p["first_c_raw"].tolist()[:3] == [0x40200000, 0x3F800000, 0x3F800000]
+    assert p["first_r_raw"].tolist()[:3] == [0x40000000, 0x7FC00000, 0xBF800000]
+    assert rows.tolist() == [2, 1]
+    # with equal_nan nothing changes here (only one side is NaN); without the NaN pair the worst is 1 vs -1
+    p2, _ = oracle.profile(r[[0, 1, 2, 4, 5]], c[[0, 1, 2, 4, 5]], oracle.F32, 1e-3, 1e-3, True)
+    assert int(p2["worst_index"]) == 4 and int(p2["n_mismatch"]) == 2
+
+
+def test_profile_ulp_distance_counts_representable_steps(oracle):
+    # k steps of nextafter away from x are at distance k, in every dtype's own spacing
+    x = np.float32(0.7)
+    for k in (1, 2, 3, 4, 7, 8, 1000, 1 << 20):
+        y = x
+        if k <= 1000:
+            for _ in range(k):
+                y = np.nextafter(y, np.float32(np.inf))
+        else:
+            y = (np.array([x]).view(np.uint32) + np.uint32(k)).view(np.float32)[0]
+        p, _ = oracle.profile(np.array([x]), np.array([y]), oracle.F32)
+        assert int(p["ulp_hist"][1 + int(np.floor(np.log2(k)))]) == 1
+    # across zero: smallest negative to smallest positive subnormal is two steps
+    p, _ = oracle.profile(np.array([0x80000001], dtype=np.uint32), np.array([0x00000001], dtype=np.uint32), oracle.F32)
+    assert int(p["ulp_hist"][2]) == 1
+    # 16-bit dtypes: same-sign patterns a < b are b - a steps apart; +Inf is one step above the largest finite
+    for code in (oracle.BF16, oracle.F16):
+        inf = 0x7F80 if code == oracle.BF16 else 0x7C00
+        a = np.array([0x3C00, 0x0001, inf - 1, 0x8005], dtype=np.uint16)
+        b = np.array([0x3C07, 0x0009, inf, 0x0003], dtype=np.uint16)      # 7, 8, 1 and 5 + 3 = 8 steps
+        p, _ = oracle.profile(a, b, code)
+        assert int(p["ulp_hist"][3]) == 1 and int(p["ulp_hist"][4]) == 2 and int(p["ulp_hist"][1]) == 1
+
+
+@pytest.mark.parametrize("code,tdt", [(0, torch.float32), (1, torch.bfloat16), (2, torch.float16)])
+def test_profile_against_torch_and_numpy(oracle, code, tdt):
+    g = torch.Generator().manual_seed(77 + code)
+    n = 5000
+    r = torch.randn(n, generator=g).to(tdt)
+    c = (r.float() * (1 + 2e-2 * torch.randn(n, generator=g))).to(tdt)
+    c[::97] = r[::97] + 1.0
+    atol = rtol = 1e-2
+    p, rows = oracle.profile(r.view(torch.uint8).numpy(), c.view(torch.uint8).numpy(), code, atol, rtol, False, row_len=128)
+    close = torch.isclose(c.float(), r.float(), rtol=rtol, atol=atol)
+    bad = (~close).numpy()
+    assert int(p["n_mismatch"]) == int(bad.sum())
+    idx = np.nonzero(bad)[0]
+    assert p["first_index"].tolist() == idx[:8].tolist()
+    ad = (c.float() - r.float()).abs().numpy()
+    ad_bad = np.where(bad, ad, -1.0)
+    assert int(p["worst_index"]) == int(np.argmax(ad_bad))          # argmax returns the first of equal maxima
+    pad = np.zeros((n + 127) // 128 * 128, dtype=bool)
+    pad[:n] = bad
+    assert rows.tolist() == pad.reshape(-1, 128).sum(axis=1).tolist()
+    assert int(p["ulp_hist"].sum()) == n and int(p["ulp_hist"][65]) == 0
+    # the histogram restated with integer views (no NaN here)
+    bits = (r.view(torch.int16 if code else torch.int32).numpy().astype(np.int64),
+            c.view(torch.int16 if code else torch.int32).numpy().astype(np.int64))
+    width = 16 if code else 32
+    def order(b):
+        u = b & ((1 << width) - 1)
+        return np.where(u >> (width - 1), -(u & ((1 << (width - 1)) - 1)), u)
+    dist = np.abs(order(bits[1]) - order(bits[0]))
+    want = np.bincount(np.where(dist == 0, 0, 1 + np.floor(np.log2(np.maximum(dist, 1))).astype(np.int64)), minlength=66)
+    assert p["ulp_hist"].tolist() == want.tolist()
+    # consistency with the verifier's record
+    rec = oracle.verify(r.view(torch.uint8).numpy(), c.view(torch.uint8).numpy(), code, atol, rtol, False)
+    assert int(rec["n_mismatch"]) == int(p["n_mismatch"]) and int(rec["first_mismatch"]) == int(p["first_index"][0])
+
+
+def test_profile_integers_and_degenerate_cases(oracle):
+    i64 = np.iinfo(np.int64)
+    r = np.array([0, 5, i64.min, -3, 7, 7], dtype=np.int64)
+    c = np.array([0, 6, i64.max, 1, 7, 9], dtype=np.int64)
+    p, rows = oracle.profile(r, c, oracle.I64, row_len=2)
+    want = np.zeros(66, dtype=np.uint64)
+    want[0], want[1], want[64], want[3], want[2] = 2, 1, 1, 1, 1        # 0; 1; 2^64-1; 4; 2
+    assert p["ulp_hist"].tolist() == want.tolist()
+    assert int(p["n_mismatch"]) == 4 and int(p["worst_index"]) == 2
+    assert int(p["worst_c_raw"]) == i64.max and int(p["worst_r_raw"]) == 1 << 63
+    assert p["first_index"].tolist()[:4] == [1, 2, 3, 5] and int(p["n_first"]) == 4
+    assert rows.tolist() == [1, 2, 1]
+    r32 = np.array([-1, 2], dtype=np.int32)
+    p, _ = oracle.profile(r32, r32 + 1, oracle.I32)
+    assert int(p["ulp_hist"][1]) == 2 and int(p["first_r_raw"][0]) == 0xFFFFFFFF       # raw bits, zero-extended
+    # empty and identical inputs
+    p, rows = oracle.profile(np.zeros(0, dtype=np.float32), np.zeros(0, dtype=np.float32), oracle.F32, row_len=4)
+    assert int(p["ulp_hist"].sum()) == 0 and int(p["worst_index"]) == oracle.NO_INDEX and rows.size == 0
+    x = np.linspace(-1, 1, 100, dtype=np.float32)
+    p, _ = oracle.profile(x, x.copy(), oracle.F32)
+    assert int(p["ulp_hist"][0]) == 100 and int(p["n_mismatch"]) == 0 and int(p["n_first"]) == 0
+    # more than eight mismatches: the list keeps the first eight, the count goes on
+    p, _ = oracle.profile(np.zeros(20, dtype=np.int32), np.ones(20, dtype=np.int32), oracle.I32)
+    assert int(p["n_mismatch"]) == 20 and p["first_index"].tolist() == list(range(8))

@@ -185,6 +185,44 @@ size_t gv_group_workspace_bytes(int64_t N);
 gv_status gv_group_candidates(const gv_result* results, int64_t N, int32_t* group_id, int32_t* group_count,
                               int32_t* n_groups, void* workspace, size_t workspace_bytes, void* cuda_stream);
 
+/* Error profile of ONE candidate against the reference: a richer error trace for a candidate that
+ * failed the functionality test (the paper feeds the trace of a failing run back to the Reflector,
+ * Sections 4.1 and 4.2; it does not define such a profile -- this is this library's reading). Meant to be
+ * called on demand for the few failing candidates; the verify calls carry none of its cost.
+ *   ulp_hist[b]   every element, by the distance between candidate and reference in units of the dtype's
+ *                 own spacing: float dtypes order their bit patterns (negative values mirrored, so -0 and
+ *                 +0 coincide); integer dtypes use |c - r|. b = 0: distance 0; b = 1 + floor(log2
+ *                 distance) otherwise (b <= 64); b = 65: a NaN is involved. The buckets sum to n_elems.
+ *   n_mismatch    elements that are not close (the verify record's count, same rule, same tolerances).
+ *   worst_*       the mismatching element with the largest error, ties to the smallest index; error of a
+ *                 float element = bits of |fl(c - r)| with NaN above everything, of an integer = |c - r|.
+ *                 worst_index = GV_NO_INDEX (raw values 0) when nothing mismatches.
+ *   first_*       the n_first <= 8 mismatching elements of smallest index, ascending; unused entries have
+ *                 index GV_NO_INDEX and raw values 0.
+ *   *_raw         the element's own bits, zero-extended to 64.
+ *   row_mismatch  device, uint32[ceil(n_elems / row_len)], mismatches per row of row_len consecutive
+ *                 elements; pass row_len = 0 and NULL to skip.
+ *   out           device, one gv_profile, fully overwritten.   tol as in gv_verify_batch.
+ *   workspace     device, >= gv_profile_workspace_bytes() bytes, 16-byte aligned.
+ * Bases must be multiples of the element size (16-byte aligned bases take 128-bit loads). n_elems == 0
+ * is legal (all zero, indices GV_NO_INDEX). Enqueues two memsets and two kernels. */
+#define GV_PROFILE_BUCKETS 66
+#define GV_PROFILE_LIST 8
+typedef struct gv_profile {
+    uint64_t ulp_hist[GV_PROFILE_BUCKETS];
+    uint64_t n_mismatch;
+    uint64_t worst_index;
+    uint64_t worst_c_raw, worst_r_raw;
+    uint64_t n_first;
+    uint64_t first_index[GV_PROFILE_LIST];
+    uint64_t first_c_raw[GV_PROFILE_LIST];
+    uint64_t first_r_raw[GV_PROFILE_LIST];
+} gv_profile;
+size_t gv_profile_workspace_bytes(void);
+gv_status gv_error_profile(const void* ref, const void* cand, uint64_t n_elems, gv_dtype dt, const gv_tol* tol,
+                           uint64_t row_len, gv_profile* out, uint32_t* row_mismatch, void* workspace,
+                           size_t workspace_bytes, void* cuda_stream);
+
 /* Host-buffer convenience for callers whose outputs live in host memory: copies the reference and
  * the candidates host->device in slabs through `staging` (device, staging_bytes), verifies them and
  * copies the N records (and the reference hash) back to host memory. Copies and kernels are

@@ -18,6 +18,7 @@
 #include "gv.h"
 #include "gv_device.cuh"
 #include "gv_group.cuh"
+#include "gv_profile.cuh"
 
 namespace gv {
 
@@ -1091,6 +1092,14 @@ extern "C" void gv_debug_counters(unsigned long long* out, int reset) {
 }
 #endif
 
+template <int DT>
+gv_status launch_profile(gv::ProfileParams p, unsigned grid, cudaStream_t st) {
+    gv::profile_kernel<DT><<<grid, gv::kProfileThreads, 0, st>>>(p);
+    gv::profile_finalize_kernel<DT><<<1, gv::kProfileThreads, 0, st>>>(p, grid);
+    GV_CUDA(cudaGetLastError());
+    return GV_OK;
+}
+
 extern "C" {
 
 size_t gv_workspace_bytes(int64_t T, int32_t N) {
@@ -1333,6 +1342,59 @@ gv_status gv_hash(const void* buf, uint64_t nbytes, uint64_t* out, void* cuda_st
 }
 
 static size_t round256(size_t x) { return (x + 255) / 256 * 256; }
+
+// ---- error profile of one candidate ----
+size_t gv_profile_workspace_bytes(void) {
+    return 256 + static_cast<size_t>(gv::kProfileMaxCtas) *
+                     (sizeof(gv::ProfileWorst) + gv::kProfileWarps * GV_PROFILE_LIST * sizeof(unsigned long long));
+}
+gv_status gv_error_profile(const void* ref, const void* cand, uint64_t n_elems, gv_dtype dt, const gv_tol* tol,
+                           uint64_t row_len, gv_profile* out, uint32_t* row_mismatch, void* workspace,
+                           size_t workspace_bytes, void* cuda_stream) {
+    const int esz = gv::elem_size(dt);
+    if (esz == 0) return GV_ERR_UNSUPPORTED;
+    if (!out || (n_elems > 0 && (!ref || !cand)) || (row_len > 0 && !row_mismatch)) return GV_ERR_INVALID_ARG;
+    const bool is_float = dt <= GV_F16;
+    if (is_float && !tol_valid(tol)) return GV_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(ref) % esz) || (reinterpret_cast<uintptr_t>(cand) % esz) ||
+        (reinterpret_cast<uintptr_t>(out) & 7u) || (reinterpret_cast<uintptr_t>(row_mismatch) & 3u))
+        return GV_ERR_MISALIGNED;
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 15u) || workspace_bytes < gv_profile_workspace_bytes())
+        return GV_ERR_WORKSPACE;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    int sm_count = 0;
+    gv_status rc = device_info(&sm_count);
+    if (rc != GV_OK) return rc;
+    gv::ProfileParams p;
+    p.ref = static_cast<const unsigned char*>(ref);
+    p.cand = static_cast<const unsigned char*>(cand);
+    p.n = n_elems;
+    p.atol = is_float ? static_cast<float>(tol->atol) : 0.0f;
+    p.rtol = is_float ? static_cast<float>(tol->rtol) : 0.0f;
+    p.equal_nan = is_float ? (tol->equal_nan != 0) : 0;
+    p.aligned = ((reinterpret_cast<uintptr_t>(ref) | reinterpret_cast<uintptr_t>(cand)) & 15u) == 0;
+    p.row_len = row_len;
+    p.out = out;
+    p.rows = row_mismatch;
+    unsigned char* ws = static_cast<unsigned char*>(workspace) + 256;
+    p.cta_worst = reinterpret_cast<gv::ProfileWorst*>(ws);
+    p.warp_first = reinterpret_cast<unsigned long long*>(ws + static_cast<size_t>(gv::kProfileMaxCtas) * sizeof(gv::ProfileWorst));
+    const uint64_t tiles = (n_elems * esz + 511) / 512;
+    uint64_t grid = (tiles + gv::kProfileWarps - 1) / gv::kProfileWarps;
+    const uint64_t cap = static_cast<uint64_t>(sm_count) * 8 < gv::kProfileMaxCtas ? static_cast<uint64_t>(sm_count) * 8 : gv::kProfileMaxCtas;
+    if (grid > cap) grid = cap;
+    if (grid == 0) grid = 1;
+    GV_CUDA(cudaMemsetAsync(out, 0, sizeof(gv_profile), st));
+    if (row_len > 0 && n_elems > 0)
+        GV_CUDA(cudaMemsetAsync(row_mismatch, 0, sizeof(uint32_t) * ((n_elems + row_len - 1) / row_len), st));
+    switch (dt) {
+        case GV_F32: return launch_profile<GV_F32>(p, static_cast<unsigned>(grid), st);
+        case GV_BF16: return launch_profile<GV_BF16>(p, static_cast<unsigned>(grid), st);
+        case GV_F16: return launch_profile<GV_F16>(p, static_cast<unsigned>(grid), st);
+        case GV_I32: return launch_profile<GV_I32>(p, static_cast<unsigned>(grid), st);
+        default: return launch_profile<GV_I64>(p, static_cast<unsigned>(grid), st);
+    }
+}
 
 // ---- grouping of duplicate candidates ----
 static uint32_t group_slots(int64_t N) {

@@ -31,6 +31,15 @@ RESULT_DTYPE = np.dtype([
     ("reserved", "<u8")])
 assert RESULT_DTYPE.itemsize == 64
 
+#: gv_profile as a numpy structured dtype (760 bytes)
+GV_PROFILE_BUCKETS, GV_PROFILE_LIST = 66, 8
+PROFILE_DTYPE = np.dtype([
+    ("ulp_hist", "<u8", (GV_PROFILE_BUCKETS,)), ("n_mismatch", "<u8"), ("worst_index", "<u8"),
+    ("worst_c_raw", "<u8"), ("worst_r_raw", "<u8"), ("n_first", "<u8"),
+    ("first_index", "<u8", (GV_PROFILE_LIST,)), ("first_c_raw", "<u8", (GV_PROFILE_LIST,)),
+    ("first_r_raw", "<u8", (GV_PROFILE_LIST,))])
+assert PROFILE_DTYPE.itemsize == 760
+
 
 class gv_tol(ctypes.Structure):
     _fields_ = [("atol", ctypes.c_double), ("rtol", ctypes.c_double),
@@ -38,7 +47,7 @@ class gv_tol(ctypes.Structure):
 
 
 EXPORTS = ["gv_verify_batch", "gv_verify_ragged", "gv_verify_ragged_noalloc", "gv_hash", "gv_group_candidates",
-           "gv_group_workspace_bytes", "gv_verify_batch_host", "gv_host_staging_bytes",
+           "gv_group_workspace_bytes", "gv_error_profile", "gv_profile_workspace_bytes", "gv_verify_batch_host", "gv_host_staging_bytes",
            "gv_workspace_bytes", "gv_check", "gv_status_string", "gv_last_cuda_error", "gv_version"]
 
 
@@ -62,6 +71,10 @@ def _load() -> ctypes.CDLL:
     L.gv_group_candidates.argtypes = [vp, i64, vp, vp, vp, vp, sz, vp]
     L.gv_group_workspace_bytes.restype = sz
     L.gv_group_workspace_bytes.argtypes = [i64]
+    L.gv_error_profile.restype = ctypes.c_int
+    L.gv_error_profile.argtypes = [vp, vp, u64, ctypes.c_int, ctypes.POINTER(gv_tol), u64, vp, vp, vp, sz, vp]
+    L.gv_profile_workspace_bytes.restype = sz
+    L.gv_profile_workspace_bytes.argtypes = []
     L.gv_verify_batch_host.restype = ctypes.c_int
     L.gv_verify_batch_host.argtypes = [vp, vp, i32, u64, ctypes.c_int, ctypes.POINTER(gv_tol), vp, vp, vp, sz, vp]
     L.gv_host_staging_bytes.restype = sz
@@ -198,6 +211,37 @@ def gv_hash(buf: torch.Tensor, out: Optional[torch.Tensor] = None,
     rc = lib.gv_hash(buf.data_ptr(), buf.numel() * buf.element_size(), out.data_ptr(), _stream_ptr(stream))
     _raise(rc)
     return out
+
+
+def gv_profile_workspace_bytes() -> int:
+    return int(lib.gv_profile_workspace_bytes())
+
+
+def gv_error_profile(ref: torch.Tensor, cand: torch.Tensor, atol: float = 0.0, rtol: float = 0.0,
+                     equal_nan: bool = False, row_len: int = 0, out: Optional[torch.Tensor] = None,
+                     rows: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None,
+                     stream: Optional[torch.cuda.Stream] = None):
+    """Enqueue the error profile of one candidate; returns (device uint8[760] holding a gv_profile,
+    device int32 per-row mismatch counts or None). Read the profile with ``profile_to_numpy``."""
+    dt = DTYPE_OF[ref.dtype]
+    n = ref.numel()
+    dev = ref.device
+    if out is None:
+        out = torch.empty(PROFILE_DTYPE.itemsize, dtype=torch.uint8, device=dev)
+    if row_len and rows is None:
+        rows = torch.empty(max(1, (n + row_len - 1) // row_len), dtype=torch.int32, device=dev)
+    if workspace is None:
+        workspace = torch.empty(gv_profile_workspace_bytes(), dtype=torch.uint8, device=dev)
+    t = _tol(atol, rtol, equal_nan)
+    rc = lib.gv_error_profile(ref.data_ptr(), cand.data_ptr(), n, dt, ctypes.byref(t), row_len, out.data_ptr(),
+                              rows.data_ptr() if rows is not None else None, workspace.data_ptr(), workspace.numel(),
+                              _stream_ptr(stream))
+    _raise(rc)
+    return out, (rows[:(n + row_len - 1) // row_len] if rows is not None else None)
+
+
+def profile_to_numpy(out: torch.Tensor) -> np.ndarray:
+    return out.cpu().numpy().view(PROFILE_DTYPE)[0]
 
 
 def gv_group_workspace_bytes(N: int) -> int:

@@ -124,3 +124,25 @@ def test_group_argument_errors_return_before_any_launch(gvlib):
     assert gv.gv_group_workspace_bytes(2048) == 256
     assert gv.gv_group_workspace_bytes(2049) == 256 + 8192 * 8
     assert gv.gv_group_workspace_bytes(-1) == 0
+
+
+def test_profile_argument_errors_return_before_any_launch(gvlib):
+    gv = gvlib
+    wsb = gv.gv_profile_workspace_bytes()
+    assert wsb > 256
+    t = gv.gv_tol(1e-3, 1e-3, 0, 0)
+
+    def call(ref=0x1000, cand=0x2000, n=16, dt=0, tol=t, row_len=0, out=0x3000, rows=None, ws=0x4000, wsb=wsb):
+        return gv.lib.gv_error_profile(ref, cand, n, dt, ctypes.byref(tol) if tol is not None else None, row_len, out,
+                                       rows, ws, wsb, None)
+    assert call(dt=7) == gv.GV_ERR_UNSUPPORTED
+    assert call(out=None) == gv.GV_ERR_INVALID_ARG
+    assert call(ref=None) == gv.GV_ERR_INVALID_ARG
+    assert call(row_len=8) == gv.GV_ERR_INVALID_ARG                  # row counts asked for, no buffer given
+    assert call(tol=None) == gv.GV_ERR_INVALID_ARG
+    assert call(tol=gv.gv_tol(-1.0, 0.0, 0, 0)) == gv.GV_ERR_INVALID_ARG
+    assert call(ref=0x1002) == gv.GV_ERR_MISALIGNED
+    assert call(out=0x3004) == gv.GV_ERR_MISALIGNED
+    assert call(ws=None) == gv.GV_ERR_WORKSPACE
+    assert call(wsb=1024) == gv.GV_ERR_WORKSPACE
+    assert gv.PROFILE_DTYPE.itemsize == 760

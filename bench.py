@@ -385,6 +385,29 @@ def main():
         grouping["cpu_oracle_us"] = 1e6 * (time.perf_counter() - t0)
         grouping["cpu_oracle_records"] = int(rec_np.shape[0])
 
+    # ---- error profile of one failing candidate (follow-on stage; outside the timed step) ----
+    error_profile = None
+    if not ragged:
+        j_bad = next((j for j, f in enumerate(wl.facts) if f["class"] != "copy"), 0)
+        pws = torch.empty(gv.gv_profile_workspace_bytes(), dtype=torch.uint8, device=device)
+        pout = torch.empty(gv.PROFILE_DTYPE.itemsize, dtype=torch.uint8, device=device)
+        prow = torch.empty((wl.n + 4095) // 4096, dtype=torch.int32, device=device)
+        for _ in range(3):
+            gv.gv_error_profile(wl.ref, wl.cands[j_bad], wl.atol, wl.rtol, wl.equal_nan, 4096, pout, prow, pws)
+        torch.cuda.synchronize()
+        p_ev = [torch.cuda.Event(enable_timing=True) for _ in range(11)]
+        p_ev[0].record(stream)
+        for i in range(10):
+            gv.gv_error_profile(wl.ref, wl.cands[j_bad], wl.atol, wl.rtol, wl.equal_nan, 4096, pout, prow, pws)
+            p_ev[i + 1].record(stream)
+        torch.cuda.synchronize()
+        p_ms = statistics.median(p_ev[i].elapsed_time(p_ev[i + 1]) for i in range(10))
+        pbytes = 2 * wl.n * W.ELEM_SIZE[wl.dtype]
+        error_profile = {"candidate": j_bad, "class": wl.facts[j_bad]["class"], "us_per_call": 1e3 * p_ms,
+                         "bytes_read": pbytes, "GB/s": pbytes / (p_ms * 1e-3) / 1e9,
+                         "frac_of_measured_hbm": pbytes / (p_ms * 1e-3) / 1e9 / peak,
+                         "note": "one candidate + the reference, both read once; fits L2 when the pair is below 126 MB"}
+
     line = {
         "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
@@ -396,6 +419,7 @@ def main():
         "frac_of_measured_hbm": value / world / peak, "frac_of_nominal_8000": value / world / 8000.0,
         "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
         "roofline": roofline, "cpu_baseline": cpu_baseline, "grouping": grouping,
+        "error_profile": error_profile,
     }
     print(json.dumps(line))
     if dist is not None:

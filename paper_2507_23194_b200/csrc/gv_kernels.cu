@@ -1346,7 +1346,7 @@ static size_t round256(size_t x) { return (x + 255) / 256 * 256; }
 // ---- error profile of one candidate ----
 size_t gv_profile_workspace_bytes(void) {
     return 256 + static_cast<size_t>(gv::kProfileMaxCtas) *
-                     (sizeof(gv::ProfileWorst) + gv::kProfileWarps * GV_PROFILE_LIST * sizeof(unsigned long long));
+                     (sizeof(gv::ProfileWorst) + GV_PROFILE_LIST * sizeof(unsigned long long));
 }
 gv_status gv_error_profile(const void* ref, const void* cand, uint64_t n_elems, gv_dtype dt, const gv_tol* tol,
                            uint64_t row_len, gv_profile* out, uint32_t* row_mismatch, void* workspace,
@@ -1378,7 +1378,7 @@ gv_status gv_error_profile(const void* ref, const void* cand, uint64_t n_elems, 
     p.rows = row_mismatch;
     unsigned char* ws = static_cast<unsigned char*>(workspace) + 256;
     p.cta_worst = reinterpret_cast<gv::ProfileWorst*>(ws);
-    p.warp_first = reinterpret_cast<unsigned long long*>(ws + static_cast<size_t>(gv::kProfileMaxCtas) * sizeof(gv::ProfileWorst));
+    p.cta_first = reinterpret_cast<unsigned long long*>(ws + static_cast<size_t>(gv::kProfileMaxCtas) * sizeof(gv::ProfileWorst));
     const uint64_t tiles = (n_elems * esz + 511) / 512;
     uint64_t grid = (tiles + gv::kProfileWarps - 1) / gv::kProfileWarps;
     const uint64_t cap = static_cast<uint64_t>(sm_count) * 8 < gv::kProfileMaxCtas ? static_cast<uint64_t>(sm_count) * 8 : gv::kProfileMaxCtas;

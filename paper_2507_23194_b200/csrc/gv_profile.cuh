@@ -37,7 +37,7 @@ struct ProfileParams {
     gv_profile* out;
     uint32_t* rows;
     ProfileWorst* cta_worst;       // [gridDim.x]
-    unsigned long long* warp_first;  // [gridDim.x * kProfileWarps][GV_PROFILE_LIST], ascending, all ones = unused
+    unsigned long long* cta_first;   // [gridDim.x][GV_PROFILE_LIST]: the CTA's smallest mismatching indices, all ones = unused
 };
 
 // bucket of a distance: 0 for 0, else 1 + floor(log2 distance)
@@ -102,11 +102,11 @@ template <int DT>
 __global__ void __launch_bounds__(kProfileThreads) profile_kernel(ProfileParams p) {
     constexpr int ESZ = Traits<DT>::ESZ;
     constexpr int EPV = 16 / ESZ;
-    __shared__ unsigned int s_hist[GV_PROFILE_BUCKETS];
+    __shared__ unsigned int s_hist[kProfileWarps][GV_PROFILE_BUCKETS];     // one per warp: fewer same-address collisions
     __shared__ unsigned long long s_first[kProfileWarps][GV_PROFILE_LIST];
     __shared__ ProfileWorst s_worst[kProfileWarps];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    for (int b = tid; b < GV_PROFILE_BUCKETS; b += kProfileThreads) s_hist[b] = 0u;
+    for (int b = tid; b < kProfileWarps * GV_PROFILE_BUCKETS; b += kProfileThreads) (&s_hist[0][0])[b] = 0u;
     if (lane < GV_PROFILE_LIST) s_first[warp][lane] = ~0ull;
     __syncthreads();
 
@@ -161,7 +161,7 @@ __global__ void __launch_bounds__(kProfileThreads) profile_kernel(ProfileParams 
                     int bucket;
                     profile_element<DT>(c_raw, r_raw, tol, close, key, bucket);
                     if (bucket == 0) zero_cnt += 1;
-                    else atomicAdd(&s_hist[bucket], 1u);
+                    else atomicAdd(&s_hist[warp][bucket], 1u);
                     if (!close) {
                         bad |= 1u << e;
                         mism_cnt += 1;
@@ -224,21 +224,40 @@ __global__ void __launch_bounds__(kProfileThreads) profile_kernel(ProfileParams 
         if (mism_cnt) atomicAdd(reinterpret_cast<unsigned long long*>(&p.out->n_mismatch), mism_cnt);
         s_worst[warp] = {best_key, best_idx, best_c, best_r};
     }
-    __syncwarp();
-    if (lane < GV_PROFILE_LIST) p.warp_first[gw * GV_PROFILE_LIST + lane] = s_first[warp][lane];
     __syncthreads();
-    for (int b = tid; b < GV_PROFILE_BUCKETS; b += kProfileThreads)
-        if (s_hist[b]) atomicAdd(reinterpret_cast<unsigned long long*>(&p.out->ulp_hist[b]), static_cast<unsigned long long>(s_hist[b]));
+    for (int b = tid; b < GV_PROFILE_BUCKETS; b += kProfileThreads) {
+        unsigned long long h = 0;
+        for (int i = 0; i < kProfileWarps; ++i) h += s_hist[i][b];
+        if (h) atomicAdd(reinterpret_cast<unsigned long long*>(&p.out->ulp_hist[b]), h);
+    }
     if (tid == 0) {
         ProfileWorst w = s_worst[0];
         for (int i = 1; i < kProfileWarps; ++i)
             if (profile_better(s_worst[i].key, s_worst[i].index, w.key, w.index)) w = s_worst[i];
         p.cta_worst[blockIdx.x] = w;
     }
+    // the CTA's eight smallest mismatching indices out of its warps' lists: warp 0, two entries per lane,
+    // eight rounds of a warp-wide minimum above the previous pick
+    if (warp == 0) {
+        __syncwarp();
+        static_assert(kProfileWarps * GV_PROFILE_LIST == 64, "two entries per lane");
+        const unsigned long long e0 = s_first[lane >> 3][lane & 7], e1 = s_first[4 + (lane >> 3)][lane & 7];
+        unsigned long long last = 0;
+        bool have_last = false;
+        for (int round = 0; round < GV_PROFILE_LIST; ++round) {
+            unsigned long long m = ~0ull;
+            if (e0 < m && (!have_last || e0 > last)) m = e0;
+            if (e1 < m && (!have_last || e1 > last)) m = e1;
+            m = warp_min_u64(m);
+            if (lane == 0) p.cta_first[static_cast<size_t>(blockIdx.x) * GV_PROFILE_LIST + round] = m;
+            last = m;
+            have_last = true;
+        }
+    }
 }
 
 // One CTA: the worst element over the per-CTA partials, the eight smallest indices over the
-// per-warp lists (eight rounds of a block-wide minimum above the previous pick), and their raw values.
+// per-CTA lists (eight rounds of a block-wide minimum above the previous pick), and their raw values.
 template <int DT>
 __global__ void __launch_bounds__(kProfileThreads) profile_finalize_kernel(ProfileParams p, unsigned int n_ctas) {
     constexpr int ESZ = Traits<DT>::ESZ;
@@ -269,28 +288,35 @@ __global__ void __launch_bounds__(kProfileThreads) profile_finalize_kernel(Profi
         p.out->worst_c_raw = w.index == ~0ull ? 0ull : w.c_raw;
         p.out->worst_r_raw = w.index == ~0ull ? 0ull : w.r_raw;
     }
-    const uint64_t entries = static_cast<uint64_t>(n_ctas) * kProfileWarps * GV_PROFILE_LIST;
-    unsigned long long last = 0;
-    bool have_last = false;
-    for (int round = 0; round < GV_PROFILE_LIST; ++round) {
-        unsigned long long m = ~0ull;
-        for (uint64_t i = tid; i < entries; i += kProfileThreads) {
-            const unsigned long long x = p.warp_first[i];
-            if (x < m && (!have_last || x > last)) m = x;
+    // each thread keeps the eight smallest of the entries it reads (one pass, independent loads) ...
+    const uint64_t entries = static_cast<uint64_t>(n_ctas) * GV_PROFILE_LIST;
+    unsigned long long t8[GV_PROFILE_LIST];
+#pragma unroll
+    for (int j = 0; j < GV_PROFILE_LIST; ++j) t8[j] = ~0ull;
+    for (uint64_t i = tid; i < entries; i += kProfileThreads) {
+        unsigned long long x = p.cta_first[i];
+        if (x < t8[GV_PROFILE_LIST - 1]) {
+#pragma unroll
+            for (int j = 0; j < GV_PROFILE_LIST; ++j) {        // insertion into the ascending list
+                const unsigned long long y = t8[j];
+                if (x < y) { t8[j] = x; x = y; }
+            }
         }
-        m = warp_min_u64(m);
+    }
+    // ... then eight rounds of a block-wide minimum over the threads' current heads (indices are unique)
+    for (int round = 0; round < GV_PROFILE_LIST; ++round) {
+        unsigned long long m = warp_min_u64(t8[0]);
         if (lane == 0) s_min[warp] = m;
         __syncthreads();
         m = s_min[0];
         for (int i = 1; i < kProfileWarps; ++i) m = s_min[i] < m ? s_min[i] : m;
         if (tid == 0) s_pick[round] = m;
-        __syncthreads();
-        last = m;
-        have_last = true;
-        if (m == ~0ull) {
-            for (int r2 = round + 1; r2 < GV_PROFILE_LIST; ++r2) if (tid == 0) s_pick[r2] = ~0ull;
-            break;
+        if (m != ~0ull && t8[0] == m) {                        // the owner drops its head
+#pragma unroll
+            for (int j = 0; j + 1 < GV_PROFILE_LIST; ++j) t8[j] = t8[j + 1];
+            t8[GV_PROFILE_LIST - 1] = ~0ull;
         }
+        __syncthreads();
     }
     __syncthreads();
     if (tid < GV_PROFILE_LIST) {

@@ -385,4 +385,72 @@ int gvo_profile_pair(const void* ref, const void* cand, uint64_t n, int dtype, d
     return 0;
 }
 
+// Pass/fail summary of one kernel's candidates and the pass@k estimate (Section 3.3: a generated
+// kernel counts as correct when it satisfies ALL unit tests -- Execution Accuracy; Section 4.2:
+// accuracy under parallel sampling is estimated with the pass@k metric).
+// results is tensor-major, T unit-test tensors x N candidates (results[t*N + j], the layout the
+// ragged verifier writes). pass[j] = 1 when candidate j has n_mismatch == 0 on every one of the T
+// tensors (with T == 0 every candidate passes vacuously). c = number of passing candidates.
+// pass_at_k[k-1], k = 1..kmax, is the standard unbiased estimator 1 - C(N-c, k) / C(N, k), evaluated
+// in binary64 as 1 - prod_{i=0}^{k-1} (N-c-i)/(N-i), factors multiplied left to right, each factor one
+// division; it is exactly 1 when N - c < k, and k > N is not allowed.
+int gvo_exec_summary(const gvo_result* results, int64_t T, int32_t N, int32_t kmax, uint8_t* pass,
+                     int32_t* n_pass, double* pass_at_k) {
+    if (T < 0 || N < 0 || kmax < 0 || kmax > N) return 1;
+    int32_t c = 0;
+    for (int32_t j = 0; j < N; ++j) {
+        bool ok = true;
+        for (int64_t t = 0; t < T; ++t) ok = ok && results[t * N + j].n_mismatch == 0;
+        pass[j] = ok ? 1 : 0;
+        c += ok ? 1 : 0;
+    }
+    *n_pass = c;
+    for (int32_t k = 1; k <= kmax; ++k) {
+        if (N - c < k) { pass_at_k[k - 1] = 1.0; continue; }
+        double prod = 1.0;
+        for (int32_t i = 0; i < k; ++i) prod = prod * (static_cast<double>(N - c - i) / static_cast<double>(N - i));
+        pass_at_k[k - 1] = 1.0 - prod;
+    }
+    return 0;
+}
+
+// Speedup of a generated kernel over the reference kernel (Section 3.3: the expectation, over the
+// unit tests, of the ratio of the median reference latency to the generated kernel's latency;
+// computed only for kernels that pass). ref_lat is T x S_ref, gen_lat T x S_gen latency samples
+// (binary32, row per unit test). Reading: both latencies are summarised by their medians (the
+// evaluator times each kernel several times); median of an even count = fl32((a + b) / 2) of the two
+// middle values, computed as fl32(fl32(a + b) * 0.5); ratio[t] = fl32(median_ref[t] / median_gen[t]);
+// speedup = (sum over t of ratio[t], accumulated in binary64 in index order) / T. NaN samples are not
+// allowed. T == 0 gives speedup 0.
+int gvo_speedup(const float* ref_lat, const float* gen_lat, int64_t T, int32_t S_ref, int32_t S_gen,
+                float* median_ref, float* median_gen, float* ratio, double* speedup) {
+    if (T < 0 || S_ref < 1 || S_gen < 1) return 1;
+    double sum = 0.0;
+    for (int64_t t = 0; t < T; ++t) {
+        float med[2];
+        for (int which = 0; which < 2; ++which) {
+            const float* row = which == 0 ? ref_lat + t * S_ref : gen_lat + t * S_gen;
+            const int32_t S = which == 0 ? S_ref : S_gen;
+            // selection by counting: the value of rank q is the x with (#smaller) <= q < (#smaller or equal)
+            float picked[2] = {0.0f, 0.0f};
+            const int32_t want[2] = {(S - 1) / 2, S / 2};
+            for (int w = 0; w < 2; ++w) {
+                for (int32_t a = 0; a < S; ++a) {
+                    int32_t less = 0, leq = 0;
+                    for (int32_t b = 0; b < S; ++b) { less += row[b] < row[a]; leq += row[b] <= row[a]; }
+                    if (less <= want[w] && want[w] < leq) { picked[w] = row[a]; break; }
+                }
+            }
+            const float s2 = picked[0] + picked[1];
+            med[which] = (S & 1) ? picked[0] : s2 * 0.5f;
+        }
+        median_ref[t] = med[0];
+        median_gen[t] = med[1];
+        ratio[t] = med[0] / med[1];
+        sum += static_cast<double>(ratio[t]);
+    }
+    *speedup = T ? sum / static_cast<double>(T) : 0.0;
+    return 0;
+}
+
 }  // extern "C"

@@ -97,6 +97,12 @@ def lib() -> ctypes.CDLL:
         L.gvo_profile_pair.restype = ctypes.c_int
         L.gvo_profile_pair.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_uint64, ctypes.c_int, ctypes.c_double,
                                        ctypes.c_double, ctypes.c_int, ctypes.c_uint64, ctypes.c_void_p, ctypes.c_void_p]
+        L.gvo_exec_summary.restype = ctypes.c_int
+        L.gvo_exec_summary.argtypes = [ctypes.c_void_p, ctypes.c_int64, ctypes.c_int32, ctypes.c_int32, ctypes.c_void_p,
+                                       ctypes.c_void_p, ctypes.c_void_p]
+        L.gvo_speedup.restype = ctypes.c_int
+        L.gvo_speedup.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64, ctypes.c_int32, ctypes.c_int32,
+                                  ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
         L.gvo_group.restype = ctypes.c_int
         L.gvo_group.argtypes = [ctypes.c_void_p, ctypes.c_int64, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
         _lib = L
@@ -209,3 +215,31 @@ def profile(ref: np.ndarray, cand: np.ndarray, dtype: int, atol: float = 0.0, rt
     if rows is not None:
         rows = rows[:(n + row_len - 1) // row_len]
     return out[0], rows
+
+
+def exec_summary(records: np.ndarray, T: int, N: int, kmax: int):
+    """(pass[N] uint8, n_pass, pass_at_k[kmax] float64) for T x N tensor-major records."""
+    rec = np.ascontiguousarray(records, dtype=RESULT_DTYPE)
+    assert rec.shape[0] == T * N
+    ok = np.zeros(max(N, 1), dtype=np.uint8)
+    c = np.zeros(1, dtype=np.int32)
+    pk = np.zeros(max(kmax, 1), dtype=np.float64)
+    rc = lib().gvo_exec_summary(rec.ctypes.data, T, N, kmax, ok.ctypes.data, c.ctypes.data, pk.ctypes.data)
+    if rc:
+        raise RuntimeError(f"gvo_exec_summary failed with {rc}")
+    return ok[:N], int(c[0]), pk[:kmax]
+
+
+def speedup(ref_lat: np.ndarray, gen_lat: np.ndarray):
+    """(median_ref[T], median_gen[T], ratio[T] float32, speedup float64) for T x S latency samples."""
+    a = np.ascontiguousarray(ref_lat, dtype=np.float32)
+    b = np.ascontiguousarray(gen_lat, dtype=np.float32)
+    T = a.shape[0]
+    assert a.ndim == 2 and b.ndim == 2 and b.shape[0] == T
+    mr, mg, ra = (np.zeros(max(T, 1), dtype=np.float32) for _ in range(3))
+    sp = np.zeros(1, dtype=np.float64)
+    rc = lib().gvo_speedup(a.ctypes.data, b.ctypes.data, T, a.shape[1], b.shape[1], mr.ctypes.data, mg.ctypes.data,
+                           ra.ctypes.data, sp.ctypes.data)
+    if rc:
+        raise RuntimeError(f"gvo_speedup failed with {rc}")
+    return mr[:T], mg[:T], ra[:T], float(sp[0])

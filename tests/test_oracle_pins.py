@@ -619,3 +619,54 @@ def test_profile_integers_and_degenerate_cases(oracle):
     # more than eight mismatches: the list keeps the first eight, the count goes on
     p, _ = oracle.profile(np.zeros(20, dtype=np.int32), np.ones(20, dtype=np.int32), oracle.I32)
     assert int(p["n_mismatch"]) == 20 and p["first_index"].tolist() == list(range(8))
+
+
+# --------------------------------------------------------------------------------------------
+# pass/fail summary, pass@k and speedup
+# --------------------------------------------------------------------------------------------
+def test_exec_summary_and_pass_at_k_exact(oracle):
+    from math import comb
+    rng = np.random.default_rng(8)
+    for T, N in [(1, 1), (3, 5), (6, 20), (2, 64), (0, 4)]:
+        rec = np.zeros(T * N, dtype=oracle.RESULT_DTYPE)
+        fail = rng.random((T, N)) < 0.15
+        rec["n_mismatch"] = np.where(fail, rng.integers(1, 100, (T, N)), 0).reshape(-1)
+        ok, c, pk = oracle.exec_summary(rec, T, N, N)
+        want_ok = (~fail).all(axis=0) if T else np.ones(N, dtype=bool)
+        assert ok.astype(bool).tolist() == want_ok.tolist() and c == int(want_ok.sum())
+        for k in range(1, N + 1):
+            exact = 1 - Fraction(comb(N - c, k), comb(N, k))           # the estimator in exact rationals
+            assert abs(pk[k - 1] - float(exact)) <= 1e-14, (T, N, k)
+        if c:
+            assert pk[0] == 1.0 - (N - c) / N                           # k = 1 is the plain pass fraction, one rounding each
+        assert all(pk[k - 1] == 1.0 for k in range(N - c + 1, N + 1))   # more draws than failures: certain
+        assert np.all(np.diff(pk) >= 0)
+    # nobody passes / everybody passes
+    rec = np.zeros(12, dtype=oracle.RESULT_DTYPE)
+    rec["n_mismatch"][:4] = 1                                            # test 0 fails for all four candidates
+    ok, c, pk = oracle.exec_summary(rec, 3, 4, 4)
+    assert ok.tolist() == [0, 0, 0, 0] and c == 0 and pk.tolist() == [0.0] * 4
+    ok, c, pk = oracle.exec_summary(np.zeros(12, dtype=oracle.RESULT_DTYPE), 3, 4, 2)
+    assert ok.tolist() == [1] * 4 and c == 4 and pk.tolist() == [1.0, 1.0]
+
+
+def test_speedup_hand_worked_and_numpy(oracle):
+    ref = np.array([[3.0, 1.0, 2.0], [8.0, 8.0, 2.0]], dtype=np.float32)          # medians 2, 8
+    gen = np.array([[1.0, 4.0, 1.0, 2.0], [4.0, 1.0, 16.0, 4.0]], dtype=np.float32)  # medians (1+2)/2 = 1.5, 4
+    mr, mg, ra, sp = oracle.speedup(ref, gen)
+    assert mr.tolist() == [2.0, 8.0] and mg.tolist() == [1.5, 4.0]
+    assert ra.tolist() == [np.float32(2.0) / np.float32(1.5), 2.0]
+    assert sp == (float(np.float32(2.0) / np.float32(1.5)) + 2.0) / 2
+    rng = np.random.default_rng(2)
+    for T, sr, sg in [(1, 1, 1), (7, 5, 8), (40, 16, 9), (3, 2, 2)]:
+        ref = rng.lognormal(0, 0.3, (T, sr)).astype(np.float32)
+        gen = rng.lognormal(-0.2, 0.3, (T, sg)).astype(np.float32)
+        ref[0, :] = ref[0, 0]                                          # ties
+        mr, mg, ra, sp = oracle.speedup(ref, gen)
+        sref, sgen = np.sort(ref, axis=1), np.sort(gen, axis=1)
+        wr = sref[:, sr // 2] if sr & 1 else ((sref[:, sr // 2 - 1] + sref[:, sr // 2]) * np.float32(0.5))
+        wg = sgen[:, sg // 2] if sg & 1 else ((sgen[:, sg // 2 - 1] + sgen[:, sg // 2]) * np.float32(0.5))
+        assert mr.tolist() == wr.tolist() and mg.tolist() == wg.tolist()
+        assert ra.tolist() == (wr / wg).tolist()
+        assert abs(sp - float(np.mean((wr / wg).astype(np.float64)))) <= 1e-12
+    assert oracle.speedup(np.zeros((0, 3), dtype=np.float32), np.zeros((0, 2), dtype=np.float32))[3] == 0.0

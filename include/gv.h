@@ -223,6 +223,32 @@ gv_status gv_error_profile(const void* ref, const void* cand, uint64_t n_elems, 
                            uint64_t row_len, gv_profile* out, uint32_t* row_mismatch, void* workspace,
                            size_t workspace_bytes, void* cuda_stream);
 
+/* Pass/fail summary of one kernel's candidates and the pass@k estimate (paper Section 3.3: a generated
+ * kernel is correct when it satisfies all unit tests; Section 4.2: accuracy under parallel sampling is
+ * estimated with pass@k).
+ *   results     device, T x N records, tensor-major (results[t*N + j]: unit-test tensor t, candidate j --
+ *               the layout gv_verify_ragged writes; a dense call's N records are the case T = 1).
+ *   pass        device, uint8[N]: 1 when candidate j has n_mismatch == 0 on all T tensors (T == 0: all 1).
+ *   n_pass      device, int32[1]: c, the number of passing candidates.
+ *   pass_at_k   device, double[kmax]: entry k-1 = 1 - C(N-c, k) / C(N, k), evaluated in binary64 as
+ *               1 - prod_{i<k} (N-c-i)/(N-i) (factors multiplied left to right); exactly 1 when N-c < k.
+ * 0 <= kmax <= N and kmax <= GV_PASSK_MAX, else GV_ERR_INVALID_ARG. One launch. */
+#define GV_PASSK_MAX 65536
+gv_status gv_exec_summary(const gv_result* results, int64_t T, int32_t N, int32_t kmax, uint8_t* pass,
+                          int32_t* n_pass, double* pass_at_k, void* cuda_stream);
+
+/* Speedup of a generated kernel over the reference kernel from latency samples (paper Section 3.3: the
+ * expectation over the unit tests of the ratio of the median reference latency to the generated kernel's
+ * latency; meaningful only for kernels that pass). Reading: both latencies are summarised by medians.
+ *   ref_lat     device, float[T][S_ref]; gen_lat device, float[T][S_gen]: samples per unit test (no NaNs).
+ *   median_ref, median_gen, ratio   device, float[T]: medians (even count: fl((a + b) * 0.5) of the two
+ *               middle values, the sum rounded first) and ratio[t] = fl(median_ref[t] / median_gen[t]).
+ *   speedup     device, double[1]: the mean of ratio[] accumulated in binary64 in index order; 0 for T == 0.
+ * 1 <= S_ref, S_gen <= GV_SAMPLES_MAX. Two launches (one CTA per unit test, then one thread for the mean). */
+#define GV_SAMPLES_MAX 4096
+gv_status gv_speedup(const float* ref_lat, const float* gen_lat, int64_t T, int32_t S_ref, int32_t S_gen,
+                     float* median_ref, float* median_gen, float* ratio, double* speedup, void* cuda_stream);
+
 /* Host-buffer convenience for callers whose outputs live in host memory: copies the reference and
  * the candidates host->device in slabs through `staging` (device, staging_bytes), verifies them and
  * copies the N records (and the reference hash) back to host memory. Copies and kernels are

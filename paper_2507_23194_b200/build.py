@@ -16,7 +16,7 @@ _INCLUDE = os.path.join(os.path.dirname(_PKG), "include")
 LIB_PATH = os.path.join(_PKG, "libgv.so")
 
 SOURCES = ["gv_kernels.cu"]
-HEADERS = ["gv_device.cuh", "gv_group.cuh", "gv_profile.cuh"]
+HEADERS = ["gv_device.cuh", "gv_group.cuh", "gv_profile.cuh", "gv_stats.cuh"]
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",

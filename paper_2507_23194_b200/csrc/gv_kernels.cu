@@ -19,6 +19,7 @@
 #include "gv_device.cuh"
 #include "gv_group.cuh"
 #include "gv_profile.cuh"
+#include "gv_stats.cuh"
 
 namespace gv {
 
@@ -1342,6 +1343,37 @@ gv_status gv_hash(const void* buf, uint64_t nbytes, uint64_t* out, void* cuda_st
 }
 
 static size_t round256(size_t x) { return (x + 255) / 256 * 256; }
+
+// ---- aggregates: pass/fail summary with pass@k, speedup from latency samples ----
+gv_status gv_exec_summary(const gv_result* results, int64_t T, int32_t N, int32_t kmax, uint8_t* pass,
+                          int32_t* n_pass, double* pass_at_k, void* cuda_stream) {
+    if (T < 0 || N < 0 || kmax < 0 || kmax > N || kmax > GV_PASSK_MAX || !n_pass) return GV_ERR_INVALID_ARG;
+    if ((N > 0 && !pass) || (kmax > 0 && !pass_at_k) || (T > 0 && N > 0 && !results)) return GV_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(results) & 7u) || (reinterpret_cast<uintptr_t>(n_pass) & 3u) ||
+        (reinterpret_cast<uintptr_t>(pass_at_k) & 7u))
+        return GV_ERR_MISALIGNED;
+    gv::exec_summary_kernel<<<1, gv::kStatsThreads, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
+        results, T, N, kmax, pass, n_pass, pass_at_k);
+    GV_CUDA(cudaGetLastError());
+    return GV_OK;
+}
+gv_status gv_speedup(const float* ref_lat, const float* gen_lat, int64_t T, int32_t S_ref, int32_t S_gen,
+                     float* median_ref, float* median_gen, float* ratio, double* speedup, void* cuda_stream) {
+    if (T < 0 || T > 0x7FFFFFFFll || S_ref < 1 || S_gen < 1 || S_ref > GV_SAMPLES_MAX || S_gen > GV_SAMPLES_MAX || !speedup)
+        return GV_ERR_INVALID_ARG;
+    if (T > 0 && (!ref_lat || !gen_lat || !median_ref || !median_gen || !ratio)) return GV_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(ref_lat) & 3u) || (reinterpret_cast<uintptr_t>(gen_lat) & 3u) ||
+        (reinterpret_cast<uintptr_t>(median_ref) & 3u) || (reinterpret_cast<uintptr_t>(median_gen) & 3u) ||
+        (reinterpret_cast<uintptr_t>(ratio) & 3u) || (reinterpret_cast<uintptr_t>(speedup) & 7u))
+        return GV_ERR_MISALIGNED;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    if (T > 0)
+        gv::median_ratio_kernel<<<static_cast<unsigned>(T), gv::kStatsThreads, 0, st>>>(ref_lat, gen_lat, S_ref, S_gen,
+                                                                                       median_ref, median_gen, ratio);
+    gv::speedup_mean_kernel<<<1, 1, 0, st>>>(ratio, T, speedup);
+    GV_CUDA(cudaGetLastError());
+    return GV_OK;
+}
 
 // ---- error profile of one candidate ----
 size_t gv_profile_workspace_bytes(void) {

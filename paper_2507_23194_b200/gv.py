@@ -47,7 +47,7 @@ class gv_tol(ctypes.Structure):
 
 
 EXPORTS = ["gv_verify_batch", "gv_verify_ragged", "gv_verify_ragged_noalloc", "gv_hash", "gv_group_candidates",
-           "gv_group_workspace_bytes", "gv_error_profile", "gv_profile_workspace_bytes", "gv_verify_batch_host", "gv_host_staging_bytes",
+           "gv_group_workspace_bytes", "gv_error_profile", "gv_profile_workspace_bytes", "gv_exec_summary", "gv_speedup", "gv_verify_batch_host", "gv_host_staging_bytes",
            "gv_workspace_bytes", "gv_check", "gv_status_string", "gv_last_cuda_error", "gv_version"]
 
 
@@ -73,6 +73,10 @@ def _load() -> ctypes.CDLL:
     L.gv_group_workspace_bytes.argtypes = [i64]
     L.gv_error_profile.restype = ctypes.c_int
     L.gv_error_profile.argtypes = [vp, vp, u64, ctypes.c_int, ctypes.POINTER(gv_tol), u64, vp, vp, vp, sz, vp]
+    L.gv_exec_summary.restype = ctypes.c_int
+    L.gv_exec_summary.argtypes = [vp, i64, i32, i32, vp, vp, vp, vp]
+    L.gv_speedup.restype = ctypes.c_int
+    L.gv_speedup.argtypes = [vp, vp, i64, i32, i32, vp, vp, vp, vp, vp]
     L.gv_profile_workspace_bytes.restype = sz
     L.gv_profile_workspace_bytes.argtypes = []
     L.gv_verify_batch_host.restype = ctypes.c_int
@@ -211,6 +215,30 @@ def gv_hash(buf: torch.Tensor, out: Optional[torch.Tensor] = None,
     rc = lib.gv_hash(buf.data_ptr(), buf.numel() * buf.element_size(), out.data_ptr(), _stream_ptr(stream))
     _raise(rc)
     return out
+
+
+def gv_exec_summary(results: torch.Tensor, T: int, N: int, kmax: int, stream: Optional[torch.cuda.Stream] = None):
+    """Enqueue the pass/fail summary of T x N tensor-major records; returns device tensors
+    (pass uint8[N], n_pass int32[1], pass_at_k float64[kmax])."""
+    dev = results.device
+    ok = torch.empty(max(N, 1), dtype=torch.uint8, device=dev)
+    c = torch.empty(1, dtype=torch.int32, device=dev)
+    pk = torch.empty(max(kmax, 1), dtype=torch.float64, device=dev)
+    _raise(lib.gv_exec_summary(results.data_ptr(), T, N, kmax, ok.data_ptr(), c.data_ptr(), pk.data_ptr(),
+                               _stream_ptr(stream)))
+    return ok[:N], c, pk[:kmax]
+
+
+def gv_speedup(ref_lat: torch.Tensor, gen_lat: torch.Tensor, stream: Optional[torch.cuda.Stream] = None):
+    """Enqueue medians, ratios and the speedup for float32 latency samples of shape (T, S_ref) and
+    (T, S_gen); returns device tensors (median_ref[T], median_gen[T], ratio[T], speedup float64[1])."""
+    T = ref_lat.shape[0]
+    dev = ref_lat.device
+    mr, mg, ra = (torch.empty(max(T, 1), dtype=torch.float32, device=dev) for _ in range(3))
+    sp = torch.empty(1, dtype=torch.float64, device=dev)
+    _raise(lib.gv_speedup(ref_lat.data_ptr(), gen_lat.data_ptr(), T, ref_lat.shape[1], gen_lat.shape[1], mr.data_ptr(),
+                          mg.data_ptr(), ra.data_ptr(), sp.data_ptr(), _stream_ptr(stream)))
+    return mr[:T], mg[:T], ra[:T], sp
 
 
 def gv_profile_workspace_bytes() -> int:

@@ -146,3 +146,22 @@ def test_profile_argument_errors_return_before_any_launch(gvlib):
     assert call(ws=None) == gv.GV_ERR_WORKSPACE
     assert call(wsb=1024) == gv.GV_ERR_WORKSPACE
     assert gv.PROFILE_DTYPE.itemsize == 760
+
+
+def test_stats_argument_errors_return_before_any_launch(gvlib):
+    gv = gvlib
+    es = lambda res=0x1000, T=2, N=4, kmax=4, ok=0x2000, c=0x3000, pk=0x4000: gv.lib.gv_exec_summary(res, T, N, kmax, ok, c, pk, None)
+    assert es(T=-1) == gv.GV_ERR_INVALID_ARG
+    assert es(kmax=5) == gv.GV_ERR_INVALID_ARG                       # more draws than candidates
+    assert es(N=100000, kmax=70000) == gv.GV_ERR_INVALID_ARG         # beyond GV_PASSK_MAX
+    assert es(c=None) == gv.GV_ERR_INVALID_ARG
+    assert es(res=None) == gv.GV_ERR_INVALID_ARG
+    assert es(pk=0x4004) == gv.GV_ERR_MISALIGNED
+    sp = lambda a=0x1000, b=0x2000, T=3, sr=5, sg=5, mr=0x3000, mg=0x4000, ra=0x5000, out=0x6000: gv.lib.gv_speedup(
+        a, b, T, sr, sg, mr, mg, ra, out, None)
+    assert sp(sr=0) == gv.GV_ERR_INVALID_ARG
+    assert sp(sg=4097) == gv.GV_ERR_INVALID_ARG
+    assert sp(out=None) == gv.GV_ERR_INVALID_ARG
+    assert sp(a=None) == gv.GV_ERR_INVALID_ARG
+    assert sp(a=0x1002) == gv.GV_ERR_MISALIGNED
+    assert sp(out=0x6004) == gv.GV_ERR_MISALIGNED

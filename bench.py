@@ -273,7 +273,7 @@ def main():
         def step():
             gv.gv_verify_batch(wl.ref, wl.cands, wl.atol, wl.rtol, wl.equal_nan, results=res, ref_hash=rh,
                                workspace=ws, cand_ptrs=ptrs)
-        launches_per_step = 1 + (n_cands + 255) // 256
+        launches_per_step = 1 + 2 * ((n_cands + 255) // 256)      # init + (classify + verify) per 256 candidates
         ref_bytes = wl.n * W.ELEM_SIZE[wl.dtype]
     cand_bytes = wl.cand_bytes
 

@@ -15,6 +15,8 @@
 #include <stdio.h>
 #include <string.h>
 
+#include <type_traits>
+
 #include "gv.h"
 #include "gv_device.cuh"
 #include "gv_group.cuh"
@@ -85,6 +87,7 @@ struct DenseParams {
     int equal_nan;
     int N;                      // candidates in this launch (<= kMaxPtrs)
     int all_aligned;            // reference and every candidate base are 16-byte aligned
+    const unsigned char* flags; // device, one byte per candidate of this launch: 1 = differs from the reference nearly everywhere
     const unsigned char* cands[kMaxPtrs];
 };
 
@@ -208,25 +211,54 @@ __device__ __forceinline__ void batch_entries(uint32_t qbase, uint32_t head, uin
         const uint64_t hs = pack64(sl.x, sl.y) + (h - h_ref);
         slots[k * 32] = make_uint2(static_cast<uint32_t>(hs), static_cast<uint32_t>(hs >> 32));
         CtaAcc* s = &acc[k];
+        uint32_t cnt = 0u;                                       // elements of this entry that are not close
         if constexpr (Traits<DT>::IS_FLOAT) {
             RefVec<16 / ESZ> rv;
-            uint32_t rflags = 0u, cnt = 0u;
+            uint32_t rflags = 0u;
             hoist_ref<DT>(r, tol, rv, rflags);
             if (!vec_fast_float<DT>(c, rv, rflags, tol, s, voff / ESZ, cnt)) settle_vector_exact<DT>(c, rv, voff / ESZ, tol, s);
-            if (cnt) atomicAdd(&s->cnt, static_cast<unsigned long long>(cnt));
         } else {
             Acc a;
             a.clear();
             vec_int<DT>(c, r, voff / ESZ, 16 / ESZ, a);
             push_rare(s, a);
-            if (a.cnt) atomicAdd(&s->cnt, static_cast<unsigned long long>(a.cnt));
+            cnt = a.cnt;
         }
+        // (one shared atomic per lane that found mismatches: these do not stall the warp, and a vote plus a
+        // match over the candidate slots measured slower even when every entry mismatches)
+        if (cnt) atomicAdd(&s->cnt, static_cast<unsigned long long>(cnt));
     }
 }
 template <int DT, bool BIGK>
 __device__ __noinline__ void process_batch(uint32_t qbase, uint32_t head, uint32_t n, uint2* slots, CtaAcc* cacc,
                                            TolF tol) {
     batch_entries<DT, BIGK>(qbase, head, n, slots, cacc, tol);
+}
+
+// Which candidates differ from the reference nearly everywhere? One CTA per candidate compares a
+// sample of its 512-byte tiles (evenly spread) with the reference, bytes only, and writes 1 when on
+// average at least GV_QDIRECT of the 32 vectors of a tile differ. The verdict only selects which of
+// the dense kernel's two loops handles the candidate; both are correct for any data.
+constexpr int kSampleTiles = 64;
+__global__ void __launch_bounds__(kThreads) classify_kernel(const __grid_constant__ DenseParams p, uint64_t full_tiles,
+                                                            unsigned char* flags) {
+    __shared__ unsigned int s_total;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    if (tid == 0) s_total = 0u;
+    __syncthreads();
+    const unsigned char* cand = p.cands[blockIdx.x];
+    const uint64_t S = full_tiles < kSampleTiles ? full_tiles : kSampleTiles;
+    unsigned int mine = 0u;
+    for (uint64_t i = warp; i < S; i += kThreads / 32) {
+        const uint64_t off = (i * full_tiles / S) * kWarpTile + lane * 16;
+        const uint4 c = ldg_stream(cand + off);
+        const uint4 r = *reinterpret_cast<const uint4*>(p.ref + off);
+        const bool differs = (c.x != r.x) || (c.y != r.y) || (c.z != r.z) || (c.w != r.w);
+        mine += __popc(__ballot_sync(0xFFFFFFFFu, differs));
+    }
+    if (lane == 0 && mine) atomicAdd(&s_total, mine);
+    __syncthreads();
+    if (tid == 0) flags[blockIdx.x] = (S > 0 && s_total >= GV_QDIRECT * S) ? 1 : 0;
 }
 
 // BIGK: word indices of the hash need more than 32 bits (tensors of 32 GiB and more).
@@ -255,8 +287,44 @@ dense_kernel(const __grid_constant__ DenseParams p) {
     const uint64_t all_tiles = (nbytes + kWarpTile - 1) / kWarpTile;
     const uint64_t gw = static_cast<uint64_t>(blockIdx.x) * kWarps + warp;   // this warp in the grid
     const uint64_t GW = static_cast<uint64_t>(gridDim.x) * kWarps;
-    const int num_groups = (p.N + kChunk - 1) / kChunk;
     const TolF tol = {p.atol, p.rtol, p.equal_nan};
+
+    // Candidates in processing order: those flagged "differs nearly everywhere" last. Chunks of 16 are
+    // formed within each class, so every chunk runs one of the two loops below.
+    static_assert(kWarps * 32 >= kMaxPtrs, "one thread per candidate");
+    __shared__ unsigned char s_list[kMaxPtrs];
+    __shared__ int s_wcount[2][kWarps];
+    __shared__ __align__(16) const unsigned char* s_cptr[kChunk];
+    {
+        const bool dn = tid < p.N && p.flags != nullptr && p.flags[tid] != 0;
+        const bool sp = tid < p.N && !dn;
+        const uint32_t bs = __ballot_sync(0xFFFFFFFFu, sp), bd = __ballot_sync(0xFFFFFFFFu, dn);
+        if (lane == 0) { s_wcount[0][warp] = __popc(bs); s_wcount[1][warp] = __popc(bd); }
+        __syncthreads();
+        int off_s = 0, off_d = 0, tot_s = 0;
+        for (int w = 0; w < kWarps; ++w) {
+            if (w < warp) { off_s += s_wcount[0][w]; off_d += s_wcount[1][w]; }
+            tot_s += s_wcount[0][w];
+        }
+        if (sp) s_list[off_s + __popc(bs & lanes_below)] = static_cast<unsigned char>(tid);
+        if (dn) s_list[tot_s + off_d + __popc(bd & lanes_below)] = static_cast<unsigned char>(tid);
+    }
+    int n_sparse = 0;
+    for (int w = 0; w < kWarps; ++w) n_sparse += s_wcount[0][w];
+    // Chunks of the ordered list: full chunks of 16, then the rest as one chunk of 4, 8 or 12 (the block
+    // loop takes multiples of 4) and one of the last 1 to 3 candidates (one visit at a time). A chunk takes
+    // the in-place loop only when all its candidates are flagged; the one chunk that straddles the two
+    // classes takes the queueing loop, which is correct (if slower) for flagged candidates too. Small
+    // chunks are costly whatever the loop -- the reference's share of the work is spread over fewer
+    // candidates -- so the classes are not padded to chunk boundaries.
+    auto chunks_of = [](int n) { return n / kChunk + ((n % kChunk) >= 4 ? 1 : 0) + ((n & 3) ? 1 : 0); };
+    auto chunk_at = [](int n, int gi, int& start, int& size) {
+        const int full = n / kChunk, rest = n % kChunk;
+        if (gi < full) { start = gi * kChunk; size = kChunk; }
+        else if (gi == full && rest >= 4) { start = full * kChunk; size = rest & ~3; }
+        else { start = n - (rest & 3); size = rest & 3; }
+    };
+    const int num_groups = chunks_of(p.N);
 
     if (lane == 0) {
         mbar_init(&bars[0], 1);
@@ -274,12 +342,19 @@ dense_kernel(const __grid_constant__ DenseParams p) {
     hc.init();
 
     for (int g = 0; g < num_groups; ++g) {
-        const int kg = min(kChunk, p.N - g * kChunk);
-        const int cand0 = g * kChunk;          // first candidate of the chunk (pointers are read straight from the parameters)
+        int cand0, kg;                                         // first entry of the chunk in s_list, its size
+        chunk_at(p.N, g, cand0, kg);
+        const bool chunk_dense = cand0 >= n_sparse;
+        if (tid < kg) s_cptr[tid] = p.cands[s_list[cand0 + tid]];
+        __syncthreads();
         for (int k = 0; k < kg; ++k) slots[k * 32] = make_uint2(0u, 0u);
 
         // ================= fast loop: full warp-tiles, every base 16-byte aligned =================
-        if (gw < full_tiles && !timed_out) {
+        // Two instances of the same loop: MODE 0 queues every differing vector (candidates that mostly
+        // agree with the reference), MODE 1 compares every differing vector in place against values
+        // hoisted per tile (candidates that differ nearly everywhere). Both are correct for any data.
+        auto fast_loop = [&](auto mode_tag) {
+            constexpr int MODE = decltype(mode_tag)::value;
             const uint32_t my_tiles = static_cast<uint32_t>(min((full_tiles - gw + GW - 1) / GW, uint64_t(0xFFFFFFFFu)));
             const uint64_t tile_stride = GW * kWarpTile;
             uint64_t voff = gw * kWarpTile + lane * 16;          // this lane's vector in the tensor (current tile)
@@ -379,8 +454,7 @@ dense_kernel(const __grid_constant__ DenseParams p) {
                 const bool differs = (c.x != r.x) || (c.y != r.y) || (c.z != r.z) || (c.w != r.w);
                 if (__any_sync(0xFFFFFFFFu, differs) || tile_forced) {
                     const bool want = differs || force != 0u;
-                    const uint32_t bal = __ballot_sync(0xFFFFFFFFu, want);
-                    if (__popc(bal) >= GV_QDIRECT) {
+                    if constexpr (MODE == 1) {
                         ensure_hoisted(r);
                         uint32_t lane_cnt = 0u;
                         if (differs) correct_slot(c, k);
@@ -388,8 +462,9 @@ dense_kernel(const __grid_constant__ DenseParams p) {
                         if constexpr (IS_FLOAT) {
                             if (__any_sync(0xFFFFFFFFu, lane_cnt != 0u)) merge_counts_converged(&cacc[k], lane_cnt);
                         }
-                    } else if (bal) {
-                        enqueue(c, r, k, want, bal);
+                    } else {
+                        const uint32_t bal = __ballot_sync(0xFFFFFFFFu, want);
+                        if (bal) enqueue(c, r, k, want, bal);
                     }
                 }
             };
@@ -416,16 +491,19 @@ dense_kernel(const __grid_constant__ DenseParams p) {
                 bulk_load(ref_stage, p.ref + gw * kWarpTile, kWarpTile, &bars[0]);
             }
 
-            if (kg == kChunk) {
-                // ---- full chunk: ring depth 8 = half a chunk. While candidate k of a tile is consumed
-                // from stage k & 7, that stage is refilled with candidate k + 8 of the same tile
-                // (k < 8) or candidate k - 8 of the next tile (k >= 8).
+            if ((kg & 3) == 0) {
+                // ---- chunk of 4, 8, 12 or 16 candidates: blocks of U = 4 visits, ring depth 8 = two blocks.
+                // The visits of the warp form one sequence (tile by tile, candidate by candidate); while a
+                // block is consumed its stages are refilled with the block two further on, which lies in
+                // the same tile, the next one or (4 candidates) the one after.
                 constexpr int U = GV_UNROLL;               // visits per unrolled block (divides kRing)
 #pragma unroll 1
-                for (int k = 0; k < kRing; ++k) {
-                    cp_async16(ring_base + k * 512u, p.cands[cand0 + k] + voff);
-                    if ((k % U) == U - 1) cp_async_commit();
+                for (int j = 0; j < kRing; ++j) {
+                    const int tt = j / kg, cc = j - tt * kg;
+                    if (static_cast<uint32_t>(tt) < my_tiles) cp_async16(ring_base + j * 512u, s_cptr[cc] + voff + tt * tile_stride);
+                    if ((j % U) == U - 1) cp_async_commit();
                 }
+                uint32_t vstage = 0u;                      // first stage of the current block: 0 or 4
 #pragma unroll 1
                 for (uint32_t i = 0; i < my_tiles; ++i) {
                     uint4 r;
@@ -433,13 +511,22 @@ dense_kernel(const __grid_constant__ DenseParams p) {
                     h_ref = hash_of(r);
                     ref_sum += h_ref;
                     new_tile(r);
-                    const bool has_next = i + 1 < my_tiles;
 #pragma unroll 1
-                    for (int k0 = 0; k0 < kChunk; k0 += U) {
-                        const uint32_t stage0 = ring_base + (k0 & (kRing - 1)) * 512u;
-                        const int refill = cand0 + ((k0 + kRing) & (kChunk - 1));
-                        const uint64_t refill_off = k0 < kRing ? voff : voff + tile_stride;
-                        const bool live = k0 < kRing || has_next;
+                    for (int k0 = 0; k0 < kg; k0 += U) {
+                        const uint32_t stage0 = ring_base + vstage * 512u;
+                        vstage ^= 4u;
+                        int refill = k0 + kRing;           // candidate and tile of the block two further on
+                        uint32_t ahead = 0u;
+                        if (refill >= kg) { refill -= kg; ahead = 1u; }
+                        if (refill >= kg) { refill -= kg; ahead = 2u; }
+                        const uint64_t refill_off = voff + ahead * tile_stride;
+                        const bool live = i + ahead < my_tiles;
+                        // the U refill pointers, two per 128-bit shared load, issued ahead of the wait
+                        static_assert(U == 4, "two pointer pairs per block");
+                        const uint4 pp0 = lds128(smem_u32(&s_cptr[refill])), pp1 = lds128(smem_u32(&s_cptr[refill + 2]));
+                        const unsigned char* const rp[U] = {
+                            reinterpret_cast<const unsigned char*>(pack64(pp0.x, pp0.y)), reinterpret_cast<const unsigned char*>(pack64(pp0.z, pp0.w)),
+                            reinterpret_cast<const unsigned char*>(pack64(pp1.x, pp1.y)), reinterpret_cast<const unsigned char*>(pack64(pp1.z, pp1.w))};
                         cp_async_wait<kRing / U - 1>();     // the block of U stages issued kRing visits ago has landed
                         uint4 c[U];
 #pragma unroll
@@ -452,33 +539,26 @@ dense_kernel(const __grid_constant__ DenseParams p) {
                             diffmask |= differs ? (1u << u) : 0u;
                         }
                         if (__any_sync(0xFFFFFFFFu, diffmask != 0u) || tile_forced) {
-                            // How many lanes want a compare, for all U visits at once: one byte per
-                            // visit, summed over the warp. Visits with GV_QDIRECT lanes or more are dense
-                            // (bit 7 of their byte in `dense`); the other non-empty ones go to the queue.
-                            static_assert(U == 4, "one byte per visit of the block");
-                            const uint32_t wantmask = force != 0u ? 0xFu : diffmask;
-                            const uint32_t counts = __reduce_add_sync(0xFFFFFFFFu, (wantmask * 0x00204081u) & 0x01010101u);
-                            const uint32_t dense = (counts + (0x80u - GV_QDIRECT) * 0x01010101u) & 0x80808080u;
+                            if constexpr (MODE == 0) {
+                                // every visit with a lane that wants a compare appends to the queue
 #pragma unroll
-                            for (int u = 0; u < U; ++u) {
-                                if (!(dense & (0x80u << (8 * u))) && (counts & (0xFFu << (8 * u)))) {
-                                    const bool want = (wantmask >> u) & 1u;
-                                    enqueue(c[u], r, k0 + u, want, __ballot_sync(0xFFFFFFFFu, want));
+                                for (int u = 0; u < U; ++u) {
+                                    const bool want = ((diffmask >> u) & 1u) || force != 0u;
+                                    const uint32_t bal = __ballot_sync(0xFFFFFFFFu, want);
+                                    if (bal) enqueue(c[u], r, k0 + u, want, bal);
                                 }
-                            }
-                            if (dense) {
+                            } else {
+                                // in place, U visits interleaved: hash chain and compare share one block
                                 ensure_hoisted(r);
                                 uint32_t lane_cnt[U];
 #pragma unroll
                                 for (int u = 0; u < U; ++u) {
                                     lane_cnt[u] = 0u;
-                                    if (dense & (0x80u << (8 * u))) {
-                                        if (diffmask & (1u << u)) {
-                                            correct_slot(c[u], k0 + u);        // hash chain and compare share one block
-                                            differing(c[u], r, k0 + u, lane_cnt[u]);
-                                        } else if (force != 0u) {
-                                            differing(c[u], r, k0 + u, lane_cnt[u]);   // identical, but the reference holds a NaN
-                                        }
+                                    if (diffmask & (1u << u)) {
+                                        correct_slot(c[u], k0 + u);
+                                        differing(c[u], r, k0 + u, lane_cnt[u]);
+                                    } else if (force != 0u) {
+                                        differing(c[u], r, k0 + u, lane_cnt[u]);   // identical, but the reference holds a NaN
                                     }
                                 }
                                 if constexpr (IS_FLOAT) {
@@ -496,21 +576,21 @@ dense_kernel(const __grid_constant__ DenseParams p) {
                         }
 #pragma unroll
                         for (int u = 0; u < U; ++u) {
-                            if (live) cp_async16(stage0 + u * 512u, p.cands[refill + u] + refill_off);
+                            if (live) cp_async16(stage0 + u * 512u, rp[u] + refill_off);
                         }
                         cp_async_commit();                  // one group per block of U refills
                     }
                     voff += tile_stride;
                 }
             } else {
-                // ---- partial chunk (fewer than 16 candidates): same ring, one visit at a time. The stage a
+                // ---- the last 1 to 3 candidates of a class: same ring, one visit at a time. The stage a
                 // visit has just consumed is refilled at once with the copy kRing visits ahead.
                 uint64_t issue_off = voff;
                 int issue_k = 0;
                 uint32_t tiles_left = my_tiles;            // tiles whose copies have not all been issued
                 auto issue_one = [&](uint32_t stage_addr) {
                     if (tiles_left) {
-                        cp_async16(stage_addr, p.cands[cand0 + issue_k] + issue_off);
+                        cp_async16(stage_addr, s_cptr[issue_k] + issue_off);
                         if (++issue_k == kg) { issue_k = 0; issue_off += tile_stride; --tiles_left; }
                     }
                     cp_async_commit();          // one group per visit, possibly empty near the end
@@ -561,6 +641,14 @@ dense_kernel(const __grid_constant__ DenseParams p) {
                 }
                 __syncwarp();
             }
+        };
+        if (gw < full_tiles && !timed_out) {
+#ifdef GV_ONLY_MODE0
+            fast_loop(std::integral_constant<int, 0>{});
+#else
+            if (chunk_dense) fast_loop(std::integral_constant<int, 1>{});
+            else fast_loop(std::integral_constant<int, 0>{});
+#endif
         }
 
         // ================= general loop: ragged tail, or some base not 16-byte aligned =================
@@ -574,7 +662,7 @@ dense_kernel(const __grid_constant__ DenseParams p) {
                 const int nwords = nvalid * ESZ > 8 ? 2 : 1;
                 if (g == 0 && p.ref_hash) my_ref_hash += hash_vec(r, voff / 8, nwords);
                 for (int k = 0; k < kg; ++k) {
-                    const uint4 c = load_vec_generic<ESZ>(p.cands[cand0 + k], voff, nbytes);
+                    const uint4 c = load_vec_generic<ESZ>(s_cptr[k], voff, nbytes);
                     Acc a;
                     a.clear();
                     a.hash = hash_vec(c, voff / 8, nwords);
@@ -596,7 +684,7 @@ dense_kernel(const __grid_constant__ DenseParams p) {
             if (lane == 0 && h) atomicAdd(&cacc[k].hash, static_cast<unsigned long long>(h));
         }
         __syncthreads();
-        if (tid < kg) push_global(&p.results[g * kChunk + tid], cacc[tid]);
+        if (tid < kg) push_global(&p.results[s_list[cand0 + tid]], cacc[tid]);
         if (tid < kChunk) cacc[tid].clear();
         __syncthreads();
     }
@@ -1104,8 +1192,9 @@ gv_status launch_profile(gv::ProfileParams p, unsigned grid, cudaStream_t st) {
 extern "C" {
 
 size_t gv_workspace_bytes(int64_t T, int32_t N) {
-    (void)N;
-    const size_t table = T > 0 ? static_cast<size_t>(T + 1) * sizeof(int64_t) : 0;
+    // status word (256 bytes), then either the ragged tile-prefix table (T + 1 entries) or the dense
+    // kernel's one classification byte per candidate
+    const size_t table = T > 0 ? static_cast<size_t>(T + 1) * sizeof(int64_t) : static_cast<size_t>(N > 0 ? N : 0);
     return 256 + ((table + 255) / 256) * 256;
 }
 
@@ -1168,6 +1257,16 @@ gv_status gv_verify_batch(const void* ref, const void* const* cands, int32_t N, 
             all_bits |= reinterpret_cast<uintptr_t>(p.cands[k]);
         }
         p.all_aligned = (all_bits & 15u) == 0;
+        // one sampling pass decides which candidates take the in-place loop (skipped for small inputs and
+        // when the fast loop cannot run at all: everything then takes the queueing loop)
+        unsigned char* flags = static_cast<unsigned char*>(workspace) + 256 + j0;
+        const uint64_t full_tiles = p.all_aligned ? n_elems * esz / gv::kWarpTile : 0;
+        p.flags = nullptr;
+        if (full_tiles >= 4096) {
+            p.flags = flags;
+            gv::classify_kernel<<<p.N, gv::kThreads, 0, st>>>(p, full_tiles, flags);
+            GV_CUDA(cudaGetLastError());
+        }
         rc = launch_dense(dt, p, sm_count, st);
         if (rc != GV_OK) return rc;
     }

@@ -258,14 +258,17 @@ def test_results_independent_of_schedule(oracle):
 # ------------------------------------------------------------------------------------------------
 # differing vectors at every density: from none to all 32 lanes of a warp-tile, several tiles per warp
 # ------------------------------------------------------------------------------------------------
-@pytest.mark.parametrize("code,equal_nan", [(1, True), (0, False), (2, True), (3, False)])
-def test_differing_lane_densities(oracle, code, equal_nan):
-    """Candidate j differs from the reference in a fraction j/15 of its 16-byte vectors, so the
-    kernel meets visits with anything from 0 to 32 differing lanes (queued and in-place compares,
-    queue wrap-around, drains at chunk ends). The differing vectors mix noise inside the tolerance,
-    plain mismatches and, for float dtypes, NaN/Inf, and the reference itself holds a few NaNs."""
+@pytest.mark.parametrize("code,equal_nan,n_cands", [(1, True, 16), (0, False, 16), (2, True, 16), (3, False, 16),
+                                                    (1, False, 37), (0, True, 37), (3, False, 21)])
+def test_differing_lane_densities(oracle, code, equal_nan, n_cands):
+    """Candidate j differs from the reference in a fraction (j mod 16)/15 of its 16-byte vectors, so the
+    kernel meets visits with anything from 0 to 32 differing lanes. The tensors are large enough for
+    the sampling pass to classify the candidates; with 37 or 21 of them both loops run (queued and
+    in-place compares), one chunk straddles the classes, the last chunks hold 4 and 1 candidates,
+    queues wrap around and are drained at chunk ends. The differing vectors mix noise inside the
+    tolerance, plain mismatches and, for float dtypes, NaN/Inf; the reference itself holds a few NaNs."""
     g = torch.Generator().manual_seed(4242 + code)
-    n = 6 * (1 << 20) + 1000 if ESZ[code] == 2 else 3 * (1 << 20) + 1000
+    n = (6 * (1 << 20) + 1000 if ESZ[code] == 2 else 3 * (1 << 20) + 1000) // (1 if n_cands == 16 else 2)
     epv = 16 // ESZ[code]
     nv = n // epv
     if code == 3:
@@ -274,8 +277,8 @@ def test_differing_lane_densities(oracle, code, equal_nan):
         r = torch.randn(n, generator=g).to(TDT[code])
         r[torch.randint(0, n, (64,), generator=g)] = float("nan")
     cands = []
-    for j in range(16):
-        pick = torch.rand(nv, generator=g) < (j / 15.0)
+    for j in range(n_cands):
+        pick = torch.rand(nv, generator=g) < (((j * 7) % 16) / 15.0)
         elem = pick.repeat_interleave(epv)
         elem = torch.cat([elem, torch.zeros(n - nv * epv, dtype=torch.bool)])
         elem &= torch.rand(n, generator=g) < 0.6                      # not every element of a picked vector

@@ -311,20 +311,45 @@ dense_kernel(const __grid_constant__ DenseParams p) {
     }
     int n_sparse = 0;
     for (int w = 0; w < kWarps; ++w) n_sparse += s_wcount[0][w];
-    // Chunks of the ordered list: full chunks of 16, then the rest as one chunk of 4, 8 or 12 (the block
-    // loop takes multiples of 4) and one of the last 1 to 3 candidates (one visit at a time). A chunk takes
-    // the in-place loop only when all its candidates are flagged; the one chunk that straddles the two
-    // classes takes the queueing loop, which is correct (if slower) for flagged candidates too. Small
-    // chunks are costly whatever the loop -- the reference's share of the work is spread over fewer
-    // candidates -- so the classes are not padded to chunk boundaries.
-    auto chunks_of = [](int n) { return n / kChunk + ((n % kChunk) >= 4 ? 1 : 0) + ((n & 3) ? 1 : 0); };
-    auto chunk_at = [](int n, int gi, int& start, int& size) {
-        const int full = n / kChunk, rest = n % kChunk;
-        if (gi < full) { start = gi * kChunk; size = kChunk; }
-        else if (gi == full && rest >= 4) { start = full * kChunk; size = rest & ~3; }
-        else { start = n - (rest & 3); size = rest & 3; }
-    };
-    const int num_groups = chunks_of(p.N);
+    // Chunks of the ordered list. A run of candidates is cut into full chunks of 16, then one chunk of 4, 8
+    // or 12 (the block loop takes multiples of 4) and one of the last 1 to 3 candidates (one visit at a
+    // time). A chunk takes the in-place loop only when all its candidates are flagged; a chunk holding
+    // both classes takes the queueing loop, which is correct (if slower) for flagged candidates too. So
+    // when a plain cut would put three or more flagged candidates into such a chunk, the list is cut at
+    // the class boundary instead (the unflagged ones up to a multiple of 4, a chunk of 4 across the
+    // boundary, then the flagged ones). Small chunks are costly whatever the loop -- the reference's
+    // share of the work is spread over fewer candidates -- so this is done only when it pays.
+    constexpr int kMaxChunks = 2 * (kMaxPtrs / kChunk) + 8;
+    __shared__ unsigned char s_cstart[kMaxChunks], s_csize[kMaxChunks];
+    __shared__ int s_nchunks;
+    if (tid == 0) {
+        int nc = 0;
+        auto emit = [&](int start, int n) {
+            while (n >= kChunk) { s_cstart[nc] = static_cast<unsigned char>(start); s_csize[nc++] = kChunk; start += kChunk; n -= kChunk; }
+            if (n >= 4) { s_cstart[nc] = static_cast<unsigned char>(start); s_csize[nc++] = static_cast<unsigned char>(n & ~3); start += n & ~3; n &= 3; }
+            if (n > 0) { s_cstart[nc] = static_cast<unsigned char>(start); s_csize[nc++] = static_cast<unsigned char>(n); }
+        };
+        const int nd = p.N - n_sparse;
+        const int in_last = n_sparse % kChunk;                                  // unflagged candidates in the chunk a plain cut puts across the boundary
+        const int flagged_there = in_last ? min(nd, kChunk - in_last) : 0;      // flagged ones it would take along
+        if (flagged_there >= 3) {
+            const int head = n_sparse & ~3;
+            emit(0, head);
+            int next = head;
+            if (n_sparse & 3) {
+                const int size = (n_sparse & 3) + min(nd, 4 - (n_sparse & 3));
+                s_cstart[nc] = static_cast<unsigned char>(head);
+                s_csize[nc++] = static_cast<unsigned char>(size);
+                next = head + size;
+            }
+            emit(next, p.N - next);
+        } else {
+            emit(0, p.N);
+        }
+        s_nchunks = nc;
+    }
+    __syncthreads();
+    const int num_groups = s_nchunks;
 
     if (lane == 0) {
         mbar_init(&bars[0], 1);
@@ -342,9 +367,8 @@ dense_kernel(const __grid_constant__ DenseParams p) {
     hc.init();
 
     for (int g = 0; g < num_groups; ++g) {
-        int cand0, kg;                                         // first entry of the chunk in s_list, its size
-        chunk_at(p.N, g, cand0, kg);
-        const bool chunk_dense = cand0 >= n_sparse;
+        const int cand0 = s_cstart[g], kg = s_csize[g];       // first entry of the chunk in s_list, its size
+        const bool chunk_dense = cand0 >= n_sparse;            // every candidate of the chunk is flagged
         if (tid < kg) s_cptr[tid] = p.cands[s_list[cand0 + tid]];
         __syncthreads();
         for (int k = 0; k < kg; ++k) slots[k * 32] = make_uint2(0u, 0u);

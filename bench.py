@@ -38,19 +38,22 @@ FALLBACK_HBM_GBS = 6650.0
 # tensors of the same shapes; the figures here are scaled to the full launch in proportion to the
 # units processed (traffic is proportional to them: every candidate byte is read once, the reference
 # once per chunk of 16 candidates).
-def _scaled(measured, ref_bytes, cap_cands, full_cands):
+def _scaled(measured, ref_bytes, cap_cands, full_cands, cap_chunks=None, full_chunks=None):
     """Capture on cap_cands candidates -> full launch: the candidate part scales with the number of
-    candidates, the reference part with the number of 16-candidate chunks."""
+    candidates, the reference part with the number of chunks the kernel forms (16 candidates each
+    unless the chunk table cuts at the class boundary, which the profile summary states)."""
     chunks = lambda n: (n + 15) // 16
-    per_cand = (measured - chunks(cap_cands) * ref_bytes) / cap_cands
-    return per_cand * full_cands + chunks(full_cands) * ref_bytes
+    cap_chunks = chunks(cap_cands) if cap_chunks is None else cap_chunks
+    full_chunks = chunks(full_cands) if full_chunks is None else full_chunks
+    per_cand = (measured - cap_chunks * ref_bytes) / cap_cands
+    return per_cand * full_cands + full_chunks * ref_bytes
 
 
 NCU_TRAFFIC_BYTES = {
-    "cfg2": _scaled(2.282e9 + 5.5e6, 33554432, 64, 256),      # profiles/dense_kernel_bf16_cfg2.md
-    "cfg3": _scaled(4.563e9 + 5.3e6, 268435456, 16, 32),      # profiles/dense_kernel_f16_cfg3.md
-    "cfg4": _scaled(4.564e9 + 6.7e6, 268435456, 16, 64),      # profiles/dense_kernel_i32_cfg4.md
-    "cfg5": (2.291e9 + 11.3e6) * 10000 / 2000,                # profiles/ragged_kernel_cfg5.md (2000 of 10000 tensors)
+    "cfg2": _scaled(2.282e9 + 6.5e6, 33554432, 64, 256),      # profiles/dense_kernel_bf16_cfg2.md
+    "cfg3": _scaled(5.101e9 + 4.6e6, 268435456, 16, 32, cap_chunks=3, full_chunks=2),   # profiles/dense_kernel_f16_cfg3.md
+    "cfg4": _scaled(4.563e9 + 5.5e6, 268435456, 16, 64),      # profiles/dense_kernel_i32_cfg4.md
+    "cfg5": (2.291e9 + 11.8e6) * 10000 / 2000,                # profiles/ragged_kernel_cfg5.md (2000 of 10000 tensors)
 }
 
 
@@ -352,7 +355,7 @@ def main():
                 "achieved": achieved, "peak": peak, "peak_kind": peak_kind + " (STREAM-style copy)",
                 "unit": "GB/s", "frac": achieved / peak, "traffic": NCU_TRAFFIC_BYTES.get(args.workload),
                 "algorithmic_bytes_per_launch": algo_bytes,
-                "note": "duration = median CUDA-event time of one call (init kernel + verify kernel) on the launch stream"}
+                "note": "duration = median CUDA-event time of one call (init, classify and verify kernels) on the launch stream"}
 
     cpu_baseline = None
     if not args.no_cpu_baseline:

@@ -105,9 +105,12 @@ struct DenseParams {
 //     vector's hash terms, so the lane hashes its reference vector once per tile and a 64-bit
 //     shared-memory slot per (candidate of the chunk, lane) only collects the corrections
 //     hash(c) - hash(r) of the vectors that differ.
-//   * Compare: identical vectors are done after the identity test. Differing vectors of sparse
-//     visits are queued per warp and compared 32 at a time, one per lane; visits in which most
-//     lanes differ are compared in place against values derived from the reference once per tile.
+//   * Compare: identical vectors are done after the identity test. A sampling pass (classify_kernel)
+//     flags the candidates that differ from the reference nearly everywhere; the kernel orders the
+//     candidates, cuts them into chunks and runs one of two instances of its loop per chunk: one
+//     queues differing vectors per warp and compares them 32 at a time, one per lane (candidates
+//     that mostly agree with the reference); the other compares every differing vector in place
+//     against values derived from the reference once per tile (chunks of flagged candidates).
 //   * Accumulators: max |d|, max relative error, counts and the first index go to per-CTA shared
 //     accumulators only when they can change them. One block combine and one set of global
 //     integer atomics per (CTA, candidate).

@@ -587,3 +587,29 @@ def test_ragged_differing_lane_densities(oracle):
         want = oracle.verify_ragged(ref_buf.numpy(), ref_off_t.numpy(), cand_buf.numpy(), cand_off_t.numpy(),
                                     dtypes_t.numpy(), N, 1e-2, 1e-2, en, n_elems=n_el.numpy())
         assert_records_equal(gv.results_to_numpy(res), want, f"ragged densities equal_nan {en}")
+
+
+@pytest.mark.parametrize("code", [1, 0])
+def test_candidates_that_fool_the_sampling_pass(oracle, code):
+    """The sampling pass that picks a loop per candidate looks at 64 evenly spread 512-byte tiles. Here
+    candidates differ from the reference exactly in those tiles and nowhere else (flagged as differing
+    everywhere, in fact almost identical), everywhere but in those tiles (the opposite), in the first
+    or second half only, plus plain copies and fully noisy ones, in an order that mixes the classes:
+    the records must not depend on which loop a candidate was given."""
+    g = torch.Generator().manual_seed(31 + code)
+    per_tile = 512 // ESZ[code]
+    tiles = 16384
+    n = tiles * per_tile
+    r = torch.randn(n, generator=g).to(TDT[code])
+    noisy = (r.float() * (1 + 3e-2 * torch.randn(n, generator=g)) + 1e-3).to(TDT[code])
+    tile_of = torch.arange(n) // per_tile
+    sampled = (tile_of % (tiles // 64)) == 0
+    first_half = tile_of < tiles // 2
+    cands = [r.clone(), torch.where(sampled, noisy, r), torch.where(sampled, r, noisy), noisy.clone(),
+             torch.where(first_half, noisy, r), torch.where(first_half, r, noisy), r.clone(), noisy.clone(),
+             torch.where(sampled, noisy, r), noisy.clone(), torch.where(sampled, r, noisy)]
+    got, rh = run_dense(r.to(DEV), [c.to(DEV) for c in cands], 1e-2, 1e-2, False)
+    want = oracle_batch(oracle, r, cands, code, 1e-2, 1e-2, False)
+    assert_records_equal(got, want, f"sampling dtype {code}")
+    assert rh == oracle.hash_bytes(host_bytes(r))
+    assert got[1].tobytes() == got[8].tobytes() and got[3].tobytes() == got[7].tobytes() == got[9].tobytes()

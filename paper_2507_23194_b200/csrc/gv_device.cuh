@@ -174,6 +174,12 @@ __device__ __forceinline__ void sts128(uint32_t smem_addr, const uint4& v) {
     asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(smem_addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w)
                  : "memory");
 }
+// the same store under a predicate (no branch: the lanes of a warp that store and those that do not stay together)
+__device__ __forceinline__ void sts128_if(uint32_t smem_addr, const uint4& v, bool on) {
+    asm volatile("{ .reg .pred p; setp.ne.u32 p, %5, 0; @p st.shared.v4.u32 [%0], {%1,%2,%3,%4}; }"
+                 ::"r"(smem_addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w), "r"(static_cast<uint32_t>(on))
+                 : "memory");
+}
 __device__ __forceinline__ uint4 lds128(uint32_t smem_addr) {
     uint4 v;
     asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];"
@@ -490,7 +496,12 @@ __device__ __forceinline__ bool vec_fast_float(const uint4& c, const RefVec<16 /
         vw = fmaxf(max3(w[0], w[1], w[2]), w[3]);
     }
     const uint32_t vab = __float_as_uint(va);
-    if (!(va <= r.tolmin)) {
+    // Common case: every element within the smallest tolerance, no running maximum raised -> one test.
+    const bool over_tol = !(va <= r.tolmin);
+    const bool raise_abs = vab > run.x;
+    const bool maybe_rel = vw > 0.0f || ((flags & 2u) && vab != 0u);
+    if (!(over_tol || raise_abs || maybe_rel)) return true;
+    if (over_tol) {
         // Some |d| exceeds the smallest tolerance of the vector, or a NaN is present. NaN or Inf:
         // the caller runs the exact rule. Otherwise every pair is finite and an element is close
         // exactly when |d| <= its own tolc.
@@ -508,8 +519,8 @@ __device__ __forceinline__ bool vec_fast_float(const uint4& c, const RefVec<16 /
             if (idx < *reinterpret_cast<volatile unsigned long long*>(&s->first)) atomicMin(&s->first, idx);
         }
     }
-    if (vab > run.x) raise_maxabs(s, vab);
-    if (vw > 0.0f || ((flags & 2u) && vab != 0u)) {
+    if (raise_abs) raise_maxabs(s, vab);
+    if (maybe_rel) {
         // some element may raise the relative maximum M: each one that passes the filter is examined
         GV_COUNT(2);
         const float M = __uint_as_float(run.y);

@@ -456,14 +456,12 @@ dense_kernel(const __grid_constant__ DenseParams p) {
             // Append this lane's vector (if it wants a compare) to the warp's queue; bal = ballot of the
             // lanes that do. Compares the 32 oldest entries as soon as 32 have gathered.
             auto enqueue = [&](const uint4& c, const uint4& r, int k, bool want, uint32_t bal) {
-                if (want) {
-                    const uint32_t at = qbase + ((qhead + qcount + __popc(bal & lanes_below)) & (kQCap - 1)) * 16u;
-                    const uint64_t meta = voff | static_cast<uint64_t>(k);
-                    sts128(at, c);
-                    sts128(at + kQPlane, r);
-                    sts128(at + 2 * kQPlane, make_uint4(static_cast<uint32_t>(meta), static_cast<uint32_t>(meta >> 32),
-                                                        static_cast<uint32_t>(h_ref), static_cast<uint32_t>(h_ref >> 32)));
-                }
+                const uint32_t at = qbase + ((qhead + qcount + __popc(bal & lanes_below)) & (kQCap - 1)) * 16u;
+                const uint64_t meta = voff | static_cast<uint64_t>(k);
+                sts128_if(at, c, want);
+                sts128_if(at + kQPlane, r, want);
+                sts128_if(at + 2 * kQPlane, make_uint4(static_cast<uint32_t>(meta), static_cast<uint32_t>(meta >> 32),
+                                                       static_cast<uint32_t>(h_ref), static_cast<uint32_t>(h_ref >> 32)), want);
                 qcount += __popc(bal);
                 if (qcount >= 32u) {
                     __syncwarp();
@@ -959,13 +957,13 @@ __device__ __forceinline__ void ragged_stretch(const RaggedParams& p, int dt, co
         const bool want = (c.x != r.x) || (c.y != r.y) || (c.z != r.z) || (c.w != r.w) || force;
         const uint32_t bal = __ballot_sync(0xFFFFFFFFu, want);
         if (bal == 0u) return;
-        if (want) {
+        {
             const uint32_t at = qbase + ((qhead + qcount + __popc(bal & lanes_below)) & (kQCap - 1)) * 16u;
             const uint64_t meta = voff | static_cast<uint64_t>(k);
-            sts128(at, c);
-            sts128(at + kQPlane, r);
-            sts128(at + 2 * kQPlane, make_uint4(static_cast<uint32_t>(meta), static_cast<uint32_t>(meta >> 32),
-                                                static_cast<uint32_t>(h_ref), static_cast<uint32_t>(h_ref >> 32)));
+            sts128_if(at, c, want);
+            sts128_if(at + kQPlane, r, want);
+            sts128_if(at + 2 * kQPlane, make_uint4(static_cast<uint32_t>(meta), static_cast<uint32_t>(meta >> 32),
+                                                   static_cast<uint32_t>(h_ref), static_cast<uint32_t>(h_ref >> 32)), want);
         }
         qcount += __popc(bal);
         if (qcount >= 32u) {

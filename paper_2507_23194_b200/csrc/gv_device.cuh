@@ -473,7 +473,9 @@ __device__ __noinline__ uint32_t rel_candidate_bits(float ad, float ar, float M,
 // n_not_close: the number of elements found not close is ADDED to this per-lane counter; the caller
 // merges it into the accumulator at a point where the whole warp is converged (one reduction and one
 // atomic per warp) -- inside this function the set of lanes present is not known reliably.
-template <int DT>
+// ADD_NOW: add the count to the accumulator at once (callers whose lanes each work for their own
+// candidate) instead of returning it in n_not_close.
+template <int DT, bool ADD_NOW = false>
 __device__ __forceinline__ bool vec_fast_float(const uint4& c, const RefVec<16 / Traits<DT>::ESZ>& r, uint32_t flags,
                                                const TolF& t, CtaAcc* s, uint64_t elem0, uint32_t& n_not_close) {
     constexpr int EPV = 16 / Traits<DT>::ESZ;
@@ -514,7 +516,8 @@ __device__ __forceinline__ bool vec_fast_float(const uint4& c, const RefVec<16 /
         }
         if (cnt) {
             GV_COUNT(3);
-            n_not_close += cnt;
+            if (ADD_NOW) atomicAdd(&s->cnt, static_cast<unsigned long long>(cnt));
+            else n_not_close += cnt;
             const unsigned long long idx = elem0 + first_e;
             if (idx < *reinterpret_cast<volatile unsigned long long*>(&s->first)) atomicMin(&s->first, idx);
         }

@@ -214,22 +214,20 @@ __device__ __forceinline__ void batch_entries(uint32_t qbase, uint32_t head, uin
         const uint64_t hs = pack64(sl.x, sl.y) + (h - h_ref);
         slots[k * 32] = make_uint2(static_cast<uint32_t>(hs), static_cast<uint32_t>(hs >> 32));
         CtaAcc* s = &acc[k];
-        uint32_t cnt = 0u;                                       // elements of this entry that are not close
+        // (mismatch counts: one shared atomic per lane that found some -- these do not stall the warp, and a
+        // vote plus a match over the candidate slots measured slower even when every entry mismatches)
         if constexpr (Traits<DT>::IS_FLOAT) {
             RefVec<16 / ESZ> rv;
-            uint32_t rflags = 0u;
+            uint32_t rflags = 0u, unused = 0u;
             hoist_ref<DT>(r, tol, rv, rflags);
-            if (!vec_fast_float<DT>(c, rv, rflags, tol, s, voff / ESZ, cnt)) settle_vector_exact<DT>(c, rv, voff / ESZ, tol, s);
+            if (!vec_fast_float<DT, true>(c, rv, rflags, tol, s, voff / ESZ, unused)) settle_vector_exact<DT>(c, rv, voff / ESZ, tol, s);
         } else {
             Acc a;
             a.clear();
             vec_int<DT>(c, r, voff / ESZ, 16 / ESZ, a);
             push_rare(s, a);
-            cnt = a.cnt;
+            if (a.cnt) atomicAdd(&s->cnt, static_cast<unsigned long long>(a.cnt));
         }
-        // (one shared atomic per lane that found mismatches: these do not stall the warp, and a vote plus a
-        // match over the candidate slots measured slower even when every entry mismatches)
-        if (cnt) atomicAdd(&s->cnt, static_cast<unsigned long long>(cnt));
     }
 }
 template <int DT, bool BIGK>

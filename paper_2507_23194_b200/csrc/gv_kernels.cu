@@ -814,7 +814,8 @@ struct RaggedSmem {
     static constexpr size_t kAccOff = kSlotOff + size_t(kWarps) * kChunk * 32 * 8;         // [warp][kChunk] CtaAcc
     static constexpr size_t kPtrOff = kAccOff + size_t(kWarps) * kChunk * sizeof(CtaAcc);  // [warp][kChunk + 2] reference + candidate pointers
     static constexpr size_t kQueueOff = kPtrOff + size_t(kWarps) * (kChunk + 2) * 8;       // [warp][3][kQCap] uint4
-    static constexpr size_t kTotal = kQueueOff + size_t(kWarps) * kQueueBytes;
+    static constexpr size_t kRefOff = kQueueOff + size_t(kWarps) * kQueueBytes;            // [warp][2][32] uint4 (four-candidate loop)
+    static constexpr size_t kTotal = kRefOff + size_t(kWarps) * 2 * kWarpTile;
 };
 
 // A full candidate vector that differs from its reference vector, any dtype. Out of line and
@@ -921,7 +922,7 @@ __device__ __forceinline__ bool vec_has_nan(int dt, const uint4& r) {
 __device__ __forceinline__ void ragged_stretch(const RaggedParams& p, int dt, const unsigned char* ref, uint64_t n,
                                                uint64_t tile_begin, uint64_t tile_end, int kg, uint2* slots,
                                                CtaAcc* wacc, const unsigned char* const* wsrc, int lane,
-                                               uint32_t ring_base, uint32_t qbase) {
+                                               uint32_t ring_base, uint32_t qbase, uint32_t refst_base) {
     const unsigned char* const* wptr = wsrc + 1;        // wsrc[0] = the reference, wsrc[1 + k] = candidate k
     const int esz = elem_size(dt);
     const uint64_t nbytes = n * esz;
@@ -973,8 +974,56 @@ __device__ __forceinline__ void ragged_stretch(const RaggedParams& p, int dt, co
         }
     };
 
-    if (full_end > tile_begin) {
-        // ---- streamed part ----
+    if (full_end > tile_begin && kg == 4) {
+        // ---- streamed part, exactly four candidates (the usual handful of sampled runs): tile by tile,
+        // the reference vector in a two-deep stage of its own and the four candidate vectors as one block
+        // of the ring, two tiles in flight; one wait, one vote and one commit per tile, pointers in registers.
+        const unsigned char* src_r = ref + lane * 16;
+        const unsigned char* src_c[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) src_c[u] = wptr[u] + lane * 16;
+        auto issue_tile = [&](uint64_t tile, uint32_t half) {     // half: 0 or 1, which half of the ring / reference stage
+            if (tile < full_end) {
+                const uint64_t off = tile * kWarpTile;
+                cp_async16(refst_base + half * 512u, src_r + off);
+#pragma unroll
+                for (int u = 0; u < 4; ++u) cp_async16(ring_base + (half * 4u + u) * 512u, src_c[u] + off);
+            }
+            cp_async_commit();
+        };
+        issue_tile(tile_begin, 0u);
+        issue_tile(tile_begin + 1, 1u);
+        uint32_t half = 0u;
+#pragma unroll 1
+        for (uint64_t tile = tile_begin; tile < full_end; ++tile) {
+            const uint64_t voff = tile * kWarpTile + lane * 16;
+            cp_async_wait<1>();                                   // this tile's group has landed
+            const uint4 r = lds128(refst_base + half * 512u);
+            uint4 c[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) c[u] = lds128(ring_base + (half * 4u + u) * 512u);
+            issue_tile(tile + 2, half);                           // refill the stages just read
+            half ^= 1u;
+            const bool force = nan_matters && vec_has_nan(dt, r);
+            const uint64_t h_ref = hash_vec_full(r, voff / 8);
+            ref_sum += h_ref;
+            uint32_t diffmask = force ? 0xFu : 0u;
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+                diffmask |= ((c[u].x != r.x) || (c[u].y != r.y) || (c[u].z != r.z) || (c[u].w != r.w)) ? (1u << u) : 0u;
+            if (__any_sync(0xFFFFFFFFu, diffmask != 0u)) {
+#pragma unroll
+                for (int u = 0; u < 4; ++u) queued_visit(c[u], r, h_ref, (diffmask >> u) & 1u, voff, u);
+            }
+        }
+        cp_async_wait<0>();
+        if (qcount) {                                   // the tensor's accumulators close: drain the queue
+            __syncwarp();
+            ragged_batch(dt, qbase, qhead, qcount, slots, wacc, tol);
+            __syncwarp();
+        }
+    } else if (full_end > tile_begin) {
+        // ---- streamed part, any number of candidates ----
         // The copies form one sequence: per tile the reference vector, then the kg candidate vectors.
         // The stage a visit has just consumed is refilled at once with the copy kRing places ahead,
         // so consumer and producer share one stage counter. src[0] is the reference, src[1 + k]
@@ -1060,6 +1109,7 @@ __global__ void __launch_bounds__(kThreads, 2) ragged_kernel(const __grid_consta
     const unsigned char** wsrc = reinterpret_cast<const unsigned char**>(smem + RaggedSmem::kPtrOff) + warp * (kChunk + 2);
     const uint32_t ring_base = smem_u32(smem + RaggedSmem::kRingOff) + (warp * kRing * 32 + lane) * 16;
     const uint32_t qbase = smem_u32(smem + RaggedSmem::kQueueOff) + warp * static_cast<uint32_t>(kQueueBytes);
+    const uint32_t refst_base = smem_u32(smem + RaggedSmem::kRefOff) + (warp * 2 * 32 + lane) * 16;
 
     const uint64_t total = static_cast<uint64_t>(p.tile_prefix[p.T]);
     const uint64_t gw = static_cast<uint64_t>(blockIdx.x) * kWarps + warp;
@@ -1099,7 +1149,7 @@ __global__ void __launch_bounds__(kThreads, 2) ragged_kernel(const __grid_consta
             if (lane == 0) wsrc[0] = ref;
             for (int k = 0; k < kg; ++k) slots[k * 32] = make_uint2(0u, 0u);
             __syncwarp();
-            ragged_stretch(p, dt, ref, n, tile_begin, tile_end, kg, slots, wacc, wsrc, lane, ring_base, qbase);
+            ragged_stretch(p, dt, ref, n, tile_begin, tile_end, kg, slots, wacc, wsrc, lane, ring_base, qbase, refst_base);
             __syncwarp();
             // leave the tensor (or this group of its candidates): combine and publish
             for (int k = 0; k < kg; ++k) {

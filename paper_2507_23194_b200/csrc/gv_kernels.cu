@@ -1330,12 +1330,13 @@ gv_status gv_verify_batch(const void* ref, const void* const* cands, int32_t N, 
             all_bits |= reinterpret_cast<uintptr_t>(p.cands[k]);
         }
         p.all_aligned = (all_bits & 15u) == 0;
-        // one sampling pass decides which candidates take the in-place loop (skipped for small inputs and
-        // when the fast loop cannot run at all: everything then takes the queueing loop)
+        // one sampling pass decides which candidates take the in-place loop (skipped when the launch is
+        // too small for it to pay, below 64 MB of candidates, and when the fast loop cannot run at all:
+        // everything then takes the queueing loop)
         unsigned char* flags = static_cast<unsigned char*>(workspace) + 256 + j0;
         const uint64_t full_tiles = p.all_aligned ? n_elems * esz / gv::kWarpTile : 0;
         p.flags = nullptr;
-        if (full_tiles >= 4096) {
+        if (full_tiles >= 64 && full_tiles * gv::kWarpTile * static_cast<uint64_t>(p.N) >= (64ull << 20)) {
             p.flags = flags;
             gv::classify_kernel<<<p.N, gv::kThreads, 0, st>>>(p, full_tiles, flags);
             GV_CUDA(cudaGetLastError());

@@ -4,7 +4,7 @@
 // the "tolerance based tensor comparison of output tensors produced by test functions" of the
 // paper's Section 3.1 (TritonBench-revised, second bullet), applied to one candidate output
 // against one reference output, as the inner step of the Evaluator's functionality test
-// (Section 4.1) whose verdict feeds Execution Accuracy (Section 3.3: a kernel passes when it
+// (Section 4.1) whose outcome feeds Execution Accuracy (Section 3.3: a kernel passes when it
 // satisfies all unit tests, i.e. n_mismatch == 0 for every test tensor).
 //
 // The paper states the comparison in one phrase and prints no formula. The rule below is the

@@ -238,7 +238,7 @@ __device__ __noinline__ void process_batch(uint32_t qbase, uint32_t head, uint32
 
 // Which candidates differ from the reference nearly everywhere? One CTA per candidate compares a
 // sample of its 512-byte tiles (evenly spread) with the reference, bytes only, and writes 1 when on
-// average at least GV_QDIRECT of the 32 vectors of a tile differ. The verdict only selects which of
+// average at least GV_QDIRECT of the 32 vectors of a tile differ. The flag only selects which of
 // the dense kernel's two loops handles the candidate; both are correct for any data.
 constexpr int kSampleTiles = 64;
 __global__ void __launch_bounds__(kThreads) classify_kernel(const __grid_constant__ DenseParams p, uint64_t full_tiles,

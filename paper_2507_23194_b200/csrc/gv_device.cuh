@@ -180,6 +180,21 @@ __device__ __forceinline__ void sts128_if(uint32_t smem_addr, const uint4& v, bo
                  ::"r"(smem_addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w), "r"(static_cast<uint32_t>(on))
                  : "memory");
 }
+// three such stores, `plane` bytes apart, under one predicate (one queue entry)
+__device__ __forceinline__ void sts128x3_if(uint32_t smem_addr, uint32_t plane, const uint4& a, const uint4& b, const uint4& c,
+                                            bool on) {
+    asm volatile(
+        "{ .reg .pred p; .reg .u32 a1, a2;\n\t"
+        "setp.ne.u32 p, %14, 0;\n\t"
+        "add.u32 a1, %0, %13;\n\t"
+        "add.u32 a2, a1, %13;\n\t"
+        "@p st.shared.v4.u32 [%0], {%1,%2,%3,%4};\n\t"
+        "@p st.shared.v4.u32 [a1], {%5,%6,%7,%8};\n\t"
+        "@p st.shared.v4.u32 [a2], {%9,%10,%11,%12}; }"
+        ::"r"(smem_addr), "r"(a.x), "r"(a.y), "r"(a.z), "r"(a.w), "r"(b.x), "r"(b.y), "r"(b.z), "r"(b.w), "r"(c.x), "r"(c.y),
+          "r"(c.z), "r"(c.w), "r"(plane), "r"(static_cast<uint32_t>(on))
+        : "memory");
+}
 __device__ __forceinline__ uint4 lds128(uint32_t smem_addr) {
     uint4 v;
     asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];"

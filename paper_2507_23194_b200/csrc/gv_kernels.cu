@@ -456,10 +456,8 @@ dense_kernel(const __grid_constant__ DenseParams p) {
             auto enqueue = [&](const uint4& c, const uint4& r, int k, bool want, uint32_t bal) {
                 const uint32_t at = qbase + ((qhead + qcount + __popc(bal & lanes_below)) & (kQCap - 1)) * 16u;
                 const uint64_t meta = voff | static_cast<uint64_t>(k);
-                sts128_if(at, c, want);
-                sts128_if(at + kQPlane, r, want);
-                sts128_if(at + 2 * kQPlane, make_uint4(static_cast<uint32_t>(meta), static_cast<uint32_t>(meta >> 32),
-                                                       static_cast<uint32_t>(h_ref), static_cast<uint32_t>(h_ref >> 32)), want);
+                sts128x3_if(at, kQPlane, c, r, make_uint4(static_cast<uint32_t>(meta), static_cast<uint32_t>(meta >> 32),
+                                                          static_cast<uint32_t>(h_ref), static_cast<uint32_t>(h_ref >> 32)), want);
                 qcount += __popc(bal);
                 if (qcount >= 32u) {
                     __syncwarp();
@@ -959,10 +957,8 @@ __device__ __forceinline__ void ragged_stretch(const RaggedParams& p, int dt, co
         {
             const uint32_t at = qbase + ((qhead + qcount + __popc(bal & lanes_below)) & (kQCap - 1)) * 16u;
             const uint64_t meta = voff | static_cast<uint64_t>(k);
-            sts128_if(at, c, want);
-            sts128_if(at + kQPlane, r, want);
-            sts128_if(at + 2 * kQPlane, make_uint4(static_cast<uint32_t>(meta), static_cast<uint32_t>(meta >> 32),
-                                                   static_cast<uint32_t>(h_ref), static_cast<uint32_t>(h_ref >> 32)), want);
+            sts128x3_if(at, kQPlane, c, r, make_uint4(static_cast<uint32_t>(meta), static_cast<uint32_t>(meta >> 32),
+                                                      static_cast<uint32_t>(h_ref), static_cast<uint32_t>(h_ref >> 32)), want);
         }
         qcount += __popc(bal);
         if (qcount >= 32u) {

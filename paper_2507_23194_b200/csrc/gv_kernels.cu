@@ -506,7 +506,7 @@ dense_kernel(const __grid_constant__ DenseParams p) {
                 }
                 return true;
             };
-            if (lane == 0) {
+            if (lane == 0 && (kg & 3) == 0) {                  // (the loop for 1 to 3 candidates streams the reference itself)
                 fence_proxy_async();
                 mbar_expect_tx(&bars[0], kWarpTile);
                 bulk_load(ref_stage, p.ref + gw * kWarpTile, kWarpTile, &bars[0]);
@@ -604,37 +604,40 @@ dense_kernel(const __grid_constant__ DenseParams p) {
                     voff += tile_stride;
                 }
             } else {
-                // ---- the last 1 to 3 candidates of a class: same ring, one visit at a time. The stage a
-                // visit has just consumed is refilled at once with the copy kRing visits ahead.
-                uint64_t issue_off = voff;
-                int issue_k = 0;
-                uint32_t tiles_left = my_tiles;            // tiles whose copies have not all been issued
-                auto issue_one = [&](uint32_t stage_addr) {
-                    if (tiles_left) {
-                        cp_async16(stage_addr, s_cptr[issue_k] + issue_off);
-                        if (++issue_k == kg) { issue_k = 0; issue_off += tile_stride; --tiles_left; }
+                // ---- the last 1 to 3 candidates (or a call with so few): tile by tile. The reference vector
+                // travels through the ring like the candidates, a tile occupies kg + 1 stages, and as many
+                // tiles as fit in the ring are in flight (4 for one candidate, else 2); one wait and one
+                // commit per tile.
+                const uint32_t per = static_cast<uint32_t>(kg) + 1u;
+                const uint32_t depth = kg == 1 ? 4u : 2u;
+                const uint64_t first_off = voff;                       // this lane's vector in the warp's first tile
+                auto issue_tile = [&](uint32_t t, uint32_t into) {
+                    if (t < my_tiles) {
+                        const uint64_t off = first_off + static_cast<uint64_t>(t) * tile_stride;
+                        const uint32_t at = ring_base + into * per * 512u;
+                        cp_async16(at, p.ref + off);
+                        for (int u = 0; u < kg; ++u) cp_async16(at + (1u + u) * 512u, s_cptr[u] + off);
                     }
-                    cp_async_commit();          // one group per visit, possibly empty near the end
+                    cp_async_commit();
                 };
-#pragma unroll 1
-                for (int j = 0; j < kRing; ++j) issue_one(ring_base + j * 512u);
-                uint32_t stage = 0;
+                for (uint32_t t = 0; t < depth; ++t) issue_tile(t, t);
+                uint32_t slot = 0u;
 #pragma unroll 1
                 for (uint32_t i = 0; i < my_tiles; ++i) {
-                    uint4 r;
-                    if (!next_ref(i, r)) { timed_out = true; break; }
+                    if (depth == 4u) cp_async_wait<3>(); else cp_async_wait<1>();
+                    const uint32_t at = ring_base + slot * per * 512u;
+                    const uint4 r = lds128(at);
+                    uint4 c[3];
+#pragma unroll
+                    for (int u = 0; u < 3; ++u) c[u] = u < kg ? lds128(at + (1u + u) * 512u) : r;
+                    issue_tile(i + depth, slot);                       // refill the stages just read
+                    slot = slot + 1u == depth ? 0u : slot + 1u;
                     h_ref = hash_of(r);
                     ref_sum += h_ref;
                     new_tile(r);
-#pragma unroll 1
-                    for (int k = 0; k < kg; ++k) {
-                        cp_async_wait<kRing - 1>();
-                        const uint32_t at = ring_base + stage * 512u;
-                        const uint4 c = lds128(at);
-                        stage = (stage + 1) & (kRing - 1);
-                        issue_one(at);
-                        visit(c, r, k);
-                    }
+#pragma unroll
+                    for (int u = 0; u < 3; ++u)
+                        if (u < kg) visit(c[u], r, u);
                     voff += tile_stride;
                 }
             }

@@ -313,8 +313,8 @@ dense_kernel(const __grid_constant__ DenseParams p) {
     int n_sparse = 0;
     for (int w = 0; w < kWarps; ++w) n_sparse += s_wcount[0][w];
     // Chunks of the ordered list. A run of candidates is cut into full chunks of 16, then one chunk of 4, 8
-    // or 12 (the block loop takes multiples of 4) and one of the last 1 to 3 candidates (one visit at a
-    // time). A chunk takes the in-place loop only when all its candidates are flagged; a chunk holding
+    // or 12 (the block loop takes multiples of 4) and one of the last 1 to 3 candidates (a tile-by-tile
+    // loop of its own). A chunk takes the in-place loop only when all its candidates are flagged; a chunk holding
     // both classes takes the queueing loop, which is correct (if slower) for flagged candidates too. So
     // when a plain cut would put three or more flagged candidates into such a chunk, the list is cut at
     // the class boundary instead (the unflagged ones up to a multiple of 4, a chunk of 4 across the

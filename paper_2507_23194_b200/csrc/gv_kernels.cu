@@ -51,7 +51,26 @@ __global__ void __launch_bounds__(kThreads) hash_kernel(const unsigned char* buf
     const uint64_t nvec = (nbytes + 15) / 16;
     const bool aligned = (reinterpret_cast<uintptr_t>(buf) & 15u) == 0;
     const uint64_t stride = static_cast<uint64_t>(gridDim.x) * blockDim.x;
-    for (uint64_t v = blockIdx.x * static_cast<uint64_t>(blockDim.x) + threadIdx.x; v < nvec; v += stride) {
+    uint64_t v = blockIdx.x * static_cast<uint64_t>(blockDim.x) + threadIdx.x;
+    if (aligned) {
+        // main part: four full vectors per thread and iteration, all loads issued before the first hash
+        // (eight independent mixing chains per thread); 32-bit word indices while they suffice
+        const uint64_t nfull = nbytes / 16;
+        const bool k32 = nbytes < (1ull << 35);
+        HashConsts hc;
+        hc.init();
+        for (; v + 3 * stride < nfull; v += 4 * stride) {
+            uint4 x[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) x[j] = ldg_stream(buf + (v + j * stride) * 16);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const uint64_t k0 = 2 * (v + j * stride);
+                h += k32 ? hash_vec_full_k32(x[j], static_cast<uint32_t>(k0), hc) : hash_vec_full(x[j], k0);
+            }
+        }
+    }
+    for (; v < nvec; v += stride) {
         const uint64_t off = v * 16;
         if (aligned && off + 16 <= nbytes) {
             h += hash_vec_full(ldg_stream(buf + off), 2 * v);

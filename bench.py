@@ -217,6 +217,9 @@ def main():
     ap.add_argument("--only-class", default="", help="keep only candidates of this recipe class (dense workloads)")
     ap.add_argument("--as-int32", action="store_true",
                     help="verify the same bytes in exact integer mode (tensors viewed as int32)")
+    ap.add_argument("--shard", default="replicas", choices=["replicas", "candidates"],
+                    help="N > 1: every rank verifies its own full batch (default), or the candidate list of ONE "
+                         "batch is split among the ranks (strong scaling; records gathered on every rank)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
@@ -248,6 +251,18 @@ def main():
         wl.cands = [wl.cands[j] for j in keep]
         wl.facts = [wl.facts[j] for j in keep]
         wl.name += ":" + args.only_class
+    sharded = args.shard == "candidates" and world > 1 and not ragged
+    shard_counts = None
+    if sharded:
+        # one batch, candidates split among the ranks; every rank holds the (seeded, identical) reference
+        from paper_2507_23194_b200 import replicas as R
+        n_all = len(wl.cands)
+        shard_counts = [len(R.shard_candidates(n_all, world, r)) for r in range(world)]
+        mine = R.shard_candidates(n_all, world, rank)
+        wl.cands = [wl.cands[j] for j in mine]
+        wl.facts = [wl.facts[j] for j in mine]
+        wl.name += f":shard{rank}of{world}"
+        torch.cuda.empty_cache()
     if args.as_int32 and not ragged:
         wl.ref = wl.ref.view(torch.int32)
         wl.cands = [c.view(torch.int32) for c in wl.cands]
@@ -309,7 +324,16 @@ def main():
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
         total_ms = float(t.item())
     ms_per_step = total_ms / args.steps
-    value = world * cand_bytes / (ms_per_step * 1e-3) / 1e9
+    job_bytes = world * cand_bytes
+    if sharded:
+        t = torch.tensor([cand_bytes], dtype=torch.float64, device=device)
+        dist.all_reduce(t, op=dist.ReduceOp.SUM)
+        job_bytes = float(t.item())                       # the one batch, all shards
+        from paper_2507_23194_b200 import replicas as R
+        all_records = R.gather_records(res, shard_counts)
+        if all_records.shape[0] != sum(shard_counts):
+            raise SystemExit("gathered records do not cover the batch")
+    value = job_bytes / (ms_per_step * 1e-3) / 1e9
 
     # ---- end to end through the host-buffer entry point (dense workloads) ----
     e2e = None
@@ -413,12 +437,14 @@ def main():
 
     line = {
         "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
-        "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
+        "scaling": "strong" if sharded else "weak",
         "vs_baseline": None, "dtype": dtype_name(wl), "data": "synthetic",
         "config": {"workload": wl.name, "candidates": n_cands, "candidate_bytes_per_step": cand_bytes,
                    "reference_bytes": ref_bytes, "atol": wl.atol, "rtol": wl.rtol, "equal_nan": wl.equal_nan,
                    "l2": "inputs larger than L2 (no flush needed)" if cand_bytes > (1 << 28) else "fits L2: not a bandwidth number",
-                   "parallelism": "independent replicas per GPU" if world > 1 else "one GPU"},
+                   "parallelism": ("one batch, candidates split over the GPUs, records gathered" if sharded else
+                                   "independent replicas per GPU") if world > 1 else "one GPU"},
         "frac_of_measured_hbm": value / world / peak, "frac_of_nominal_8000": value / world / 8000.0,
         "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
         "roofline": roofline, "cpu_baseline": cpu_baseline, "grouping": grouping,

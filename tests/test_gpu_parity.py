@@ -613,3 +613,27 @@ def test_candidates_that_fool_the_sampling_pass(oracle, code):
     assert_records_equal(got, want, f"sampling dtype {code}")
     assert rh == oracle.hash_bytes(host_bytes(r))
     assert got[1].tobytes() == got[8].tobytes() and got[3].tobytes() == got[7].tobytes() == got[9].tobytes()
+
+
+def test_many_classified_candidates_over_two_launches(oracle):
+    """300 candidates of 256 KB each: more than one launch of 256 (the classification bytes of the second
+    launch follow those of the first in the workspace), enough bytes for the sampling pass to run, and
+    a second launch of 44 = 16 + 16 + 12 candidates. Every third candidate differs everywhere."""
+    g = torch.Generator().manual_seed(2024)
+    n = 128 * 1024
+    r = torch.randn(n, generator=g).to(torch.bfloat16)
+    noisy = [(r.float() * (1 + 2e-2 * torch.randn(n, generator=g))).to(torch.bfloat16) for _ in range(5)]
+    cands = []
+    for j in range(300):
+        if j % 3 == 0:
+            c = noisy[j % 5].clone()
+            c[j] = float(j)                                   # make every record distinct
+        else:
+            c = r.clone()
+            if j % 3 == 1:
+                c[(j * 37) % n] = 100.0
+        cands.append(c)
+    got, rh = run_dense(r.to(DEV), [c.to(DEV) for c in cands], 1e-2, 1e-2, True)
+    want = oracle_batch(oracle, r, cands, 1, 1e-2, 1e-2, True)
+    assert_records_equal(got, want, "300 classified candidates")
+    assert rh == oracle.hash_bytes(host_bytes(r))

@@ -637,3 +637,50 @@ def test_many_classified_candidates_over_two_launches(oracle):
     want = oracle_batch(oracle, r, cands, 1, 1e-2, 1e-2, True)
     assert_records_equal(got, want, "300 classified candidates")
     assert rh == oracle.hash_bytes(host_bytes(r))
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_randomised_large_batches(oracle, seed):
+    """Random dtype, candidate count (1 ... 40), differing-vector density per candidate (0 ... 1),
+    tolerances and equal_nan at 64-160 MB of candidates per call: the sizes at which the sampling pass
+    runs and every chunk shape and loop of the dense kernel occurs."""
+    for case in range(4):
+        rng = np.random.default_rng(7000 + seed * 10 + case)
+        g = torch.Generator().manual_seed(7000 + seed * 10 + case)
+        code = int(rng.integers(0, 5))
+        N = int(rng.choice([1, 2, 3, 4, 5, 7, 8, 12, 16, 17, 20, 31, 33, 40]))
+        n = (int(rng.integers(64, 160)) << 20) // (N * ESZ[code]) + int(rng.integers(0, 64))
+        if code >= 3:
+            r = torch.randint(-(1 << 20), 1 << 20, (n,), generator=g, dtype=TDT[code])
+        else:
+            r = (torch.randn(n, generator=g) * float(10.0 ** rng.integers(-3, 3))).to(TDT[code])
+            if rng.random() < 0.5:
+                r[torch.randint(0, n, (8,), generator=g)] = float("nan")
+        epv = 16 // ESZ[code]
+        cands = []
+        for j in range(N):
+            p = float(rng.choice([0.0, 0.0, 0.001, 0.05, 0.3, 0.6, 0.9, 1.0]))
+            if p == 0.0:
+                cands.append(r.clone())
+                continue
+            pick = (torch.rand(n // epv + 1, generator=g) < p).repeat_interleave(epv)[:n]
+            if code >= 3:
+                cands.append(torch.where(pick, r + int(rng.integers(1, 9)), r))
+                continue
+            kind = int(rng.integers(0, 3))
+            if kind == 1:
+                alt = (r.float() + 1.0).to(TDT[code])
+            else:
+                alt = (r.float() * (1 + 1e-2 * torch.randn(n, generator=g))).to(TDT[code])
+            if kind == 2:
+                alt[torch.randint(0, n, (64,), generator=g)] = float("inf")
+                alt[torch.randint(0, n, (64,), generator=g)] = float("nan")
+            cands.append(torch.where(pick, alt, r))
+        atol = float(rng.choice([0.0, 1e-3, 1e-2]))
+        rtol = float(rng.choice([0.0, 1e-2, 0.1]))
+        en = bool(rng.integers(0, 2))
+        got, rh = run_dense(r.to(DEV), [c.to(DEV) for c in cands], atol, rtol, en)
+        want = oracle_batch(oracle, r, cands, code, atol, rtol, en)
+        assert_records_equal(got, want, f"large seed {seed} case {case} dtype {code} N {N} n {n}")
+        assert rh == oracle.hash_bytes(host_bytes(r))
+        torch.cuda.empty_cache()

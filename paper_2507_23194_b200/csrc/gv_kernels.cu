@@ -934,6 +934,49 @@ __device__ __forceinline__ bool vec_has_nan(int dt, const uint4& r) {
     return any;
 }
 
+// Tiles [tile_begin, tile_end) with synchronous element-sized loads: the tail tile of a tensor, or every
+// tile of a tensor whose bases are not 16-byte aligned. Returns the sum of the reference's hash terms
+// over the full vectors it met (the caller adds it to every candidate's slot).
+__device__ __noinline__ uint64_t ragged_tail(int dt, const unsigned char* ref, uint64_t nbytes, uint64_t tile_begin,
+                                             uint64_t tile_end, int kg, uint2* slots, CtaAcc* wacc,
+                                             const unsigned char* const* wptr, TolF tol, bool nan_matters) {
+    const int esz = elem_size(dt);
+    const int lane = threadIdx.x & 31;
+    uint64_t ref_sum = 0;
+#pragma unroll 1
+    for (uint64_t tile = tile_begin; tile < tile_end; ++tile) {
+        const uint64_t voff = tile * kWarpTile + lane * 16;
+        const uint64_t rem = voff < nbytes ? nbytes - voff : 0;
+        const int nvalid = rem >= 16 ? 16 / esz : static_cast<int>(rem / esz);
+        if (nvalid <= 0) continue;
+        const bool full = rem >= 16;
+        const uint4 r = load_vec_any(esz, ref, voff, nbytes);
+        const bool force = nan_matters && full && vec_has_nan(dt, r);
+        uint64_t h_ref = 0;
+        if (full) {
+            h_ref = hash_vec_full(r, voff / 8);
+            ref_sum += h_ref;
+        }
+#pragma unroll 1
+        for (int k = 0; k < kg; ++k) {
+            const uint4 c = load_vec_any(esz, wptr[k], voff, nbytes);
+            if (full) {
+                const bool differs = (c.x != r.x) || (c.y != r.y) || (c.z != r.z) || (c.w != r.w);
+                if (differs) {
+                    const uint64_t d = hash_vec_full(c, voff / 8) - h_ref;
+                    const uint2 sl = slots[k * 32];
+                    const uint64_t h = pack64(sl.x, sl.y) + d;
+                    slots[k * 32] = make_uint2(static_cast<uint32_t>(h), static_cast<uint32_t>(h >> 32));
+                }
+                if (differs || force) ragged_differing(dt, c, r, voff, tol, &wacc[k]);
+            } else {
+                ragged_partial(dt, c, r, voff, nvalid, tol, &wacc[k], &slots[k * 32]);
+            }
+        }
+    }
+    return ref_sum;
+}
+
 // Tiles [tile_begin, tile_end) of one tensor against kg of its candidates (pointers in wptr).
 // Full tiles with 16-byte aligned bases are streamed through the lane's asynchronous-copy ring
 // (reference vector first, then the kg candidate vectors of the tile, kRing copies in flight), so
@@ -957,17 +1000,6 @@ __device__ __forceinline__ void ragged_stretch(const RaggedParams& p, int dt, co
     // vector's own hash terms: those are summed once per tile (ref_sum), the slots only collect the
     // corrections hash(c) - hash(r) of differing vectors, and ref_sum is added to every slot at the end.
     uint64_t ref_sum = 0;
-    auto one_visit = [&](const uint4& c, const uint4& r, uint64_t h_ref, bool force, uint64_t voff, int k) {
-        const bool differs = (c.x != r.x) || (c.y != r.y) || (c.z != r.z) || (c.w != r.w);
-        if (differs) {
-            const uint64_t d = hash_vec_full(c, voff / 8) - h_ref;
-            const uint2 sl = slots[k * 32];
-            const uint64_t h = pack64(sl.x, sl.y) + d;
-            slots[k * 32] = make_uint2(static_cast<uint32_t>(h), static_cast<uint32_t>(h >> 32));
-        }
-        if (differs || force) ragged_differing(dt, c, r, voff, tol, &wacc[k]);
-    };
-
     // Streamed tiles (the whole warp is present): differing vectors go to the warp's queue and are
     // compared 32 at a time, one per lane, like the dense kernel's sparse visits.
     const uint32_t lanes_below = (1u << lane) - 1u;
@@ -1090,28 +1122,9 @@ __device__ __forceinline__ void ragged_stretch(const RaggedParams& p, int dt, co
         }
     }
 
-    // ---- synchronous part: the tail tile, or every tile of an unaligned tensor ----
-#pragma unroll 1
-    for (uint64_t tile = full_end; tile < tile_end; ++tile) {
-        const uint64_t voff = tile * kWarpTile + lane * 16;
-        const uint64_t rem = voff < nbytes ? nbytes - voff : 0;
-        const int nvalid = rem >= 16 ? 16 / esz : static_cast<int>(rem / esz);
-        if (nvalid <= 0) continue;
-        const bool full = rem >= 16;
-        const uint4 r = load_vec_any(esz, ref, voff, nbytes);
-        const bool force = nan_matters && full && vec_has_nan(dt, r);
-        uint64_t h_ref = 0;
-        if (full) {
-            h_ref = hash_vec_full(r, voff / 8);
-            ref_sum += h_ref;
-        }
-#pragma unroll 1
-        for (int k = 0; k < kg; ++k) {
-            const uint4 c = load_vec_any(esz, wptr[k], voff, nbytes);
-            if (full) one_visit(c, r, h_ref, force, voff, k);
-            else ragged_partial(dt, c, r, voff, nvalid, tol, &wacc[k], &slots[k * 32]);
-        }
-    }
+    // ---- synchronous part: the tail tile, or every tile of an unaligned tensor (out of line: cold code
+    // whose registers the streaming loops should not pay for) ----
+    if (full_end < tile_end) ref_sum += ragged_tail(dt, ref, nbytes, full_end, tile_end, kg, slots, wacc, wptr, tol, nan_matters);
     for (int k = 0; k < kg; ++k) {
         const uint2 sl = slots[k * 32];
         const uint64_t h = pack64(sl.x, sl.y) + ref_sum;

@@ -385,6 +385,9 @@ dense_kernel(const __grid_constant__ DenseParams p) {
     bool timed_out = false;
     HashConsts hc;
     hc.init();
+    // candidate bytes are read exactly once: mark them evict-first in L2 so that they do not push out the
+    // reference, which every chunk reads again (+5 % on copies of a reference that fits L2)
+    const uint64_t l2pol = l2_evict_first_policy();
 
     for (int g = 0; g < num_groups; ++g) {
         const int cand0 = s_cstart[g], kg = s_csize[g];       // first entry of the chunk in s_list, its size
@@ -540,7 +543,7 @@ dense_kernel(const __grid_constant__ DenseParams p) {
 #pragma unroll 1
                 for (int j = 0; j < kRing; ++j) {
                     const int tt = j / kg, cc = j - tt * kg;
-                    if (static_cast<uint32_t>(tt) < my_tiles) cp_async16(ring_base + j * 512u, s_cptr[cc] + voff + tt * tile_stride);
+                    if (static_cast<uint32_t>(tt) < my_tiles) cp_async16_hint(ring_base + j * 512u, s_cptr[cc] + voff + tt * tile_stride, l2pol);
                     if ((j % U) == U - 1) cp_async_commit();
                 }
                 uint32_t vstage = 0u;                      // first stage of the current block: 0 or 4
@@ -616,7 +619,7 @@ dense_kernel(const __grid_constant__ DenseParams p) {
                         }
 #pragma unroll
                         for (int u = 0; u < U; ++u) {
-                            if (live) cp_async16(stage0 + u * 512u, rp[u] + refill_off);
+                            if (live) cp_async16_hint(stage0 + u * 512u, rp[u] + refill_off, l2pol);
                         }
                         cp_async_commit();                  // one group per block of U refills
                     }
@@ -635,7 +638,7 @@ dense_kernel(const __grid_constant__ DenseParams p) {
                         const uint64_t off = first_off + static_cast<uint64_t>(t) * tile_stride;
                         const uint32_t at = ring_base + into * per * 512u;
                         cp_async16(at, p.ref + off);
-                        for (int u = 0; u < kg; ++u) cp_async16(at + (1u + u) * 512u, s_cptr[u] + off);
+                        for (int u = 0; u < kg; ++u) cp_async16_hint(at + (1u + u) * 512u, s_cptr[u] + off, l2pol);
                     }
                     cp_async_commit();
                 };

@@ -96,7 +96,10 @@ typedef struct gv_tol {
  *   results    device, N records, fully overwritten.
  *   ref_hash   device, one uint64, receives the reference's content hash; may be NULL.
  *   workspace  device, >= gv_workspace_bytes(0, N) bytes, 16-byte aligned; must stay untouched
- *              until the stream has passed this call. It carries a status word for gv_check().
+ *              until the stream has passed this call. It carries a status word for gv_check() and
+ *              one byte per candidate for the pass that samples each candidate and decides which
+ *              of the kernel's loops handles it (a matter of speed only: records do not depend on it).
+ * Enqueues up to three kernels per 256 candidates (record initialisation once, sampling pass, verify).
  * N == 0 or n_elems == 0 is legal (no records / zero records: all fields 0, first_mismatch
  * GV_NO_INDEX, hash 0). The paper notes that an earlier harness silently compared empty outputs
  * (Section 3.1); deciding that an empty test output is an error is left to the caller, who can

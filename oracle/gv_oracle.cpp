@@ -127,6 +127,25 @@ uint64_t gvo_hash(const void* buf, uint64_t nbytes) {
     return h;
 }
 
+// Second hash lane, for callers that want a stronger duplicate key than the one in the records: the
+// same sum with the word index multiplied by the odd constant 0x9E3779B97F4A7C15 (mod 2^64) before the
+// xor: hash2 = sum over k of splitmix64((k * gamma) xor W_k). Buffers that collide in the first lane
+// because their sets {k xor W_k} coincide (e.g. int64 [0, 0] and [1, 1]) do not collide here.
+uint64_t gvo_hash2(const void* buf, uint64_t nbytes) {
+    const unsigned char* p = static_cast<const unsigned char*>(buf);
+    const uint64_t nwords = (nbytes + 7) / 8;
+    uint64_t h = 0;
+    for (uint64_t k = 0; k < nwords; ++k) {
+        uint64_t w = 0;
+        for (int b = 0; b < 8; ++b) {
+            const uint64_t pos = 8 * k + static_cast<uint64_t>(b);
+            if (pos < nbytes) w |= static_cast<uint64_t>(p[pos]) << (8 * b);
+        }
+        h += gvo_splitmix64((k * 0x9E3779B97F4A7C15ull) ^ w);
+    }
+    return h;
+}
+
 // Widening used by the compare; exported so a test can check it against numpy for all 2^16
 // patterns of both 16-bit types. Returns the binary32 bit pattern.
 uint32_t gvo_widen_bits(int dtype, uint32_t raw) {

@@ -81,6 +81,8 @@ def lib() -> ctypes.CDLL:
         L.gvo_splitmix64.argtypes = [ctypes.c_uint64]
         L.gvo_hash.restype = ctypes.c_uint64
         L.gvo_hash.argtypes = [ctypes.c_void_p, ctypes.c_uint64]
+        L.gvo_hash2.restype = ctypes.c_uint64
+        L.gvo_hash2.argtypes = [ctypes.c_void_p, ctypes.c_uint64]
         L.gvo_widen_bits.restype = ctypes.c_uint32
         L.gvo_widen_bits.argtypes = [ctypes.c_int, ctypes.c_uint32]
         L.gvo_verify.restype = ctypes.c_int
@@ -124,6 +126,14 @@ def hash_bytes(a) -> int:
         a = np.frombuffer(bytes(a), dtype=np.uint8)
     a = _as_bytes_array(a)
     return int(lib().gvo_hash(a.ctypes.data_as(ctypes.c_void_p), ctypes.c_uint64(a.nbytes)))
+
+
+def hash2_bytes(a) -> int:
+    """Second hash lane (word index multiplied by the odd constant before the xor)."""
+    if isinstance(a, (bytes, bytearray)):
+        a = np.frombuffer(bytes(a), dtype=np.uint8)
+    a = _as_bytes_array(a)
+    return int(lib().gvo_hash2(a.ctypes.data if a.size else None, a.nbytes))
 
 
 def widen_bits(dtype: int, raw: int) -> int:

@@ -670,3 +670,30 @@ def test_speedup_hand_worked_and_numpy(oracle):
         assert ra.tolist() == (wr / wg).tolist()
         assert abs(sp - float(np.mean((wr / wg).astype(np.float64)))) <= 1e-12
     assert oracle.speedup(np.zeros((0, 3), dtype=np.float32), np.zeros((0, 2), dtype=np.float32))[3] == 0.0
+
+
+# --------------------------------------------------------------------------------------------
+# second hash lane (word index multiplied by the odd gamma before the xor)
+# --------------------------------------------------------------------------------------------
+def test_hash2_zero_words_are_the_published_generator_outputs(oracle):
+    # word k of an all-zero buffer contributes splitmix64(k * gamma): output k of the generator seeded with 0
+    outs = [int(row.split()[1], 16) for row in _rows("splitmix64_published.txt")]
+    for n in range(1, len(outs) + 1):
+        assert oracle.hash2_bytes(b"\0" * (8 * n)) == sum(outs[:n]) & M64
+
+
+def test_hash2_brute_force_and_collision_pair(oracle):
+    rng = np.random.default_rng(9)
+    data = rng.integers(0, 256, size=4200, dtype=np.uint8).tobytes()
+    for nbytes in list(range(0, 40)) + [255, 256, 257, 4096, 4099]:
+        b = data[:nbytes] + b"\0" * (-nbytes % 8)
+        want = 0
+        for k in range(len(b) // 8):
+            want = (want + _py_splitmix64(((k * GAMMA) & M64) ^ int.from_bytes(b[8 * k:8 * k + 8], "little"))) & M64
+        assert oracle.hash2_bytes(data[:nbytes]) == want, nbytes
+    # the pair that collides in the first lane is told apart by the second
+    z = np.array([0, 0], dtype=np.int64)
+    o = np.array([1, 1], dtype=np.int64)
+    assert oracle.hash_bytes(z) == oracle.hash_bytes(o)
+    assert oracle.hash2_bytes(z) != oracle.hash2_bytes(o)
+    assert oracle.hash2_bytes(b"") == 0

@@ -166,6 +166,13 @@ gv_status gv_verify_ragged_noalloc(const void* ref_base, const int64_t* ref_off,
  * The same function the verifier applies to each candidate (used to de-duplicate candidates). */
 gv_status gv_hash(const void* buf, uint64_t nbytes, uint64_t* out, void* cuda_stream);
 
+/* Second hash lane, same arguments: sum over the 64-bit words W_k of splitmix64((k * 0x9E3779B97F4A7C15)
+ * xor W_k). Buffers whose first-lane hashes collide because their sets {k xor W_k} coincide (int64 [0, 0]
+ * and [1, 1]) differ here. It is not part of the verify pass or of the records (it would double the hash
+ * work of data that differs); call it on the few candidates whose records fall into one duplicate group
+ * when a stronger key than the record's hash is wanted. */
+gv_status gv_hash2(const void* buf, uint64_t nbytes, uint64_t* out, void* cuda_stream);
+
 /* Groups of duplicate candidates (what the content hash is for: the paper's parallel scaling,
  * Section 4.2, samples many generation runs per reference, and identical candidates need to be
  * examined only once). Candidates i and j are duplicates exactly when their 64-byte records are

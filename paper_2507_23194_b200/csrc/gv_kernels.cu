@@ -45,6 +45,9 @@ __global__ void init_results_kernel(gv_result* res, uint64_t count, uint32_t* st
 // =============================================================================================
 // gv_hash
 // =============================================================================================
+// LANE2: the second hash lane -- the word index is multiplied by the odd constant kGamma before the xor.
+constexpr uint64_t kGamma = 0x9E3779B97F4A7C15ull;
+template <bool LANE2>
 __global__ void __launch_bounds__(kThreads) hash_kernel(const unsigned char* buf, uint64_t nbytes,
                                                         unsigned long long* out) {
     uint64_t h = 0;
@@ -66,13 +69,18 @@ __global__ void __launch_bounds__(kThreads) hash_kernel(const unsigned char* buf
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
                 const uint64_t k0 = 2 * (v + j * stride);
-                h += k32 ? hash_vec_full_k32(x[j], static_cast<uint32_t>(k0), hc) : hash_vec_full(x[j], k0);
+                if constexpr (LANE2) {
+                    const uint64_t g0 = k0 * kGamma;
+                    h += splitmix64(g0 ^ pack64(x[j].x, x[j].y)) + splitmix64((g0 + kGamma) ^ pack64(x[j].z, x[j].w));
+                } else {
+                    h += k32 ? hash_vec_full_k32(x[j], static_cast<uint32_t>(k0), hc) : hash_vec_full(x[j], k0);
+                }
             }
         }
     }
     for (; v < nvec; v += stride) {
         const uint64_t off = v * 16;
-        if (aligned && off + 16 <= nbytes) {
+        if (aligned && off + 16 <= nbytes && !LANE2) {
             h += hash_vec_full(ldg_stream(buf + off), 2 * v);
         } else {
             // unaligned base or ragged tail: assemble the words byte by byte, zero padded
@@ -81,7 +89,12 @@ __global__ void __launch_bounds__(kThreads) hash_kernel(const unsigned char* buf
                 if (off + b < nbytes) w[b >> 2] |= static_cast<uint32_t>(buf[off + b]) << (8 * (b & 3));
             }
             const uint64_t rem = nbytes - off;
-            h += hash_vec(make_uint4(w[0], w[1], w[2], w[3]), 2 * v, rem > 8 ? 2 : 1);
+            if constexpr (LANE2) {
+                h += splitmix64((2 * v * kGamma) ^ pack64(w[0], w[1]));
+                if (rem > 8) h += splitmix64(((2 * v + 1) * kGamma) ^ pack64(w[2], w[3]));
+            } else {
+                h += hash_vec(make_uint4(w[0], w[1], w[2], w[3]), 2 * v, rem > 8 ? 2 : 1);
+            }
         }
     }
     h = warp_sum_u64(h);
@@ -1288,6 +1301,25 @@ extern "C" void gv_debug_counters(unsigned long long* out, int reset) {
 }
 #endif
 
+template <bool LANE2>
+gv_status launch_hash(const void* buf, uint64_t nbytes, uint64_t* out, void* cuda_stream) {
+    if (!out || (nbytes > 0 && !buf)) return GV_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(out) & 7u) return GV_ERR_MISALIGNED;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    int sm_count = 0;
+    gv_status rc = device_info(&sm_count);
+    if (rc != GV_OK) return rc;
+    GV_CUDA(cudaMemsetAsync(out, 0, sizeof(uint64_t), st));
+    if (nbytes == 0) return GV_OK;
+    const uint64_t nvec = (nbytes + 15) / 16;
+    uint64_t grid = (nvec + gv::kThreads - 1) / gv::kThreads;
+    const uint64_t cap = static_cast<uint64_t>(sm_count) * 8;
+    if (grid > cap) grid = cap;
+    gv::hash_kernel<LANE2><<<static_cast<unsigned>(grid), gv::kThreads, 0, st>>>(
+        static_cast<const unsigned char*>(buf), nbytes, reinterpret_cast<unsigned long long*>(out));
+    GV_CUDA(cudaGetLastError());
+    return GV_OK;
+}
 template <int DT>
 gv_status launch_profile(gv::ProfileParams p, unsigned grid, cudaStream_t st) {
     gv::profile_kernel<DT><<<grid, gv::kProfileThreads, 0, st>>>(p);
@@ -1340,7 +1372,7 @@ gv_status gv_verify_batch(const void* ref, const void* const* cands, int32_t N, 
     if (N == 0) {
         if (ref_hash) {
             int grid = sm_count * 8;
-            gv::hash_kernel<<<grid, gv::kThreads, 0, st>>>(static_cast<const unsigned char*>(ref), n_elems * esz,
+            gv::hash_kernel<false><<<grid, gv::kThreads, 0, st>>>(static_cast<const unsigned char*>(ref), n_elems * esz,
                                                            reinterpret_cast<unsigned long long*>(ref_hash));
             GV_CUDA(cudaGetLastError());
         }
@@ -1531,22 +1563,10 @@ gv_status gv_verify_ragged_noalloc(const void* ref_base, const int64_t* ref_off,
 }
 
 gv_status gv_hash(const void* buf, uint64_t nbytes, uint64_t* out, void* cuda_stream) {
-    if (!out || (nbytes > 0 && !buf)) return GV_ERR_INVALID_ARG;
-    if (reinterpret_cast<uintptr_t>(out) & 7u) return GV_ERR_MISALIGNED;
-    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-    int sm_count = 0;
-    gv_status rc = device_info(&sm_count);
-    if (rc != GV_OK) return rc;
-    GV_CUDA(cudaMemsetAsync(out, 0, sizeof(uint64_t), st));
-    if (nbytes == 0) return GV_OK;
-    const uint64_t nvec = (nbytes + 15) / 16;
-    uint64_t grid = (nvec + gv::kThreads - 1) / gv::kThreads;
-    const uint64_t cap = static_cast<uint64_t>(sm_count) * 8;
-    if (grid > cap) grid = cap;
-    gv::hash_kernel<<<static_cast<unsigned>(grid), gv::kThreads, 0, st>>>(
-        static_cast<const unsigned char*>(buf), nbytes, reinterpret_cast<unsigned long long*>(out));
-    GV_CUDA(cudaGetLastError());
-    return GV_OK;
+    return launch_hash<false>(buf, nbytes, out, cuda_stream);
+}
+gv_status gv_hash2(const void* buf, uint64_t nbytes, uint64_t* out, void* cuda_stream) {
+    return launch_hash<true>(buf, nbytes, out, cuda_stream);
 }
 
 static size_t round256(size_t x) { return (x + 255) / 256 * 256; }

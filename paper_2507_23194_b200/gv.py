@@ -46,7 +46,7 @@ class gv_tol(ctypes.Structure):
                 ("equal_nan", ctypes.c_int32), ("reserved", ctypes.c_int32)]
 
 
-EXPORTS = ["gv_verify_batch", "gv_verify_ragged", "gv_verify_ragged_noalloc", "gv_hash", "gv_group_candidates",
+EXPORTS = ["gv_verify_batch", "gv_verify_ragged", "gv_verify_ragged_noalloc", "gv_hash", "gv_hash2", "gv_group_candidates",
            "gv_group_workspace_bytes", "gv_error_profile", "gv_profile_workspace_bytes", "gv_exec_summary", "gv_speedup", "gv_verify_batch_host", "gv_host_staging_bytes",
            "gv_workspace_bytes", "gv_check", "gv_status_string", "gv_last_cuda_error", "gv_version"]
 
@@ -67,6 +67,8 @@ def _load() -> ctypes.CDLL:
     L.gv_verify_ragged_noalloc.argtypes = [vp, vp, vp, vp, vp, vp, i64, i32, ctypes.POINTER(gv_tol), vp, vp, vp]
     L.gv_hash.restype = ctypes.c_int
     L.gv_hash.argtypes = [vp, u64, vp, vp]
+    L.gv_hash2.restype = ctypes.c_int
+    L.gv_hash2.argtypes = [vp, u64, vp, vp]
     L.gv_group_candidates.restype = ctypes.c_int
     L.gv_group_candidates.argtypes = [vp, i64, vp, vp, vp, vp, sz, vp]
     L.gv_group_workspace_bytes.restype = sz
@@ -239,6 +241,15 @@ def gv_speedup(ref_lat: torch.Tensor, gen_lat: torch.Tensor, stream: Optional[to
     _raise(lib.gv_speedup(ref_lat.data_ptr(), gen_lat.data_ptr(), T, ref_lat.shape[1], gen_lat.shape[1], mr.data_ptr(),
                           mg.data_ptr(), ra.data_ptr(), sp.data_ptr(), _stream_ptr(stream)))
     return mr[:T], mg[:T], ra[:T], sp
+
+
+def gv_hash2(buf: torch.Tensor, out: Optional[torch.Tensor] = None,
+             stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:
+    """Enqueue the second hash lane of ``buf``'s bytes; returns a device int64 tensor holding the u64."""
+    if out is None:
+        out = torch.empty(1, dtype=torch.int64, device=buf.device)
+    _raise(lib.gv_hash2(buf.data_ptr(), buf.numel() * buf.element_size(), out.data_ptr(), _stream_ptr(stream)))
+    return out
 
 
 def gv_profile_workspace_bytes() -> int:

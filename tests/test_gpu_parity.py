@@ -684,3 +684,19 @@ def test_randomised_large_batches(oracle, seed):
         assert_records_equal(got, want, f"large seed {seed} case {case} dtype {code} N {N} n {n}")
         assert rh == oracle.hash_bytes(host_bytes(r))
         torch.cuda.empty_cache()
+
+
+def test_hash2_sizes_and_offsets(oracle):
+    # the second hash lane against the oracle: every small size, unaligned bases, a large buffer
+    rng = np.random.default_rng(21)
+    data = torch.from_numpy(rng.integers(0, 256, size=(1 << 22) + 100, dtype=np.uint8))
+    dd = data.to(DEV)
+    for off in (0, 1, 3, 8, 16):
+        for nbytes in list(range(0, 50)) + [255, 256, 257, 4095, 4096, 4097, 65536 + 5]:
+            h = gv.gv_hash2(dd[off:off + nbytes])
+            assert int(h.cpu().numpy().view(np.uint64)[0]) == oracle.hash2_bytes(data[off:off + nbytes].numpy()), (off, nbytes)
+    h = gv.gv_hash2(dd[:1 << 22])
+    assert int(h.cpu().numpy().view(np.uint64)[0]) == oracle.hash2_bytes(data[:1 << 22].numpy())
+    z, o = torch.zeros(2, dtype=torch.int64, device=DEV), torch.ones(2, dtype=torch.int64, device=DEV)
+    assert int(gv.gv_hash(z).cpu()[0]) == int(gv.gv_hash(o).cpu()[0])          # the first lane's collision pair
+    assert int(gv.gv_hash2(z).cpu()[0]) != int(gv.gv_hash2(o).cpu()[0])

@@ -404,7 +404,11 @@ dense_kernel(const __grid_constant__ DenseParams p) {
 
     for (int g = 0; g < num_groups; ++g) {
         const int cand0 = s_cstart[g], kg = s_csize[g];       // first entry of the chunk in s_list, its size
-        const bool chunk_dense = cand0 >= n_sparse;            // every candidate of the chunk is flagged
+        // in-place loop: every candidate of the chunk is flagged, or (a small chunk across the class
+        // boundary) at least half of them are -- unflagged candidates rarely differ, and when they do the
+        // in-place loop handles them correctly, whereas flagged ones are costly in the queueing loop
+        const int flagged_here = max(0, cand0 + kg - max(cand0, n_sparse));
+        const bool chunk_dense = 2 * flagged_here >= kg;
         if (tid < kg) s_cptr[tid] = p.cands[s_list[cand0 + tid]];
         __syncthreads();
         for (int k = 0; k < kg; ++k) slots[k * 32] = make_uint2(0u, 0u);

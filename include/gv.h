@@ -2,7 +2,7 @@
  *
  * What it computes. The GEAK paper's Evaluator runs a "functionality test" on every generated
  * kernel (Section 4.1): the candidate's unit-test outputs are checked against the reference
- * kernel's by a "tolerance based tensor comparison of output tensors" (Section 3.1), and a
+ * kernel's tensor against tensor within tolerances, not as printed text (Section 3.1), and a
  * kernel counts towards Execution Accuracy when all its tests pass (Section 3.3). Parallel and
  * sequential scaling (Section 4.2, Section 5.2) produce many candidates per reference output;
  * this library verifies N candidates against one reference in a single pass over the data.
@@ -250,7 +250,8 @@ gv_status gv_exec_summary(const gv_result* results, int64_t T, int32_t N, int32_
 /* Speedup of a generated kernel over the reference kernel from latency samples (paper Section 3.3: the
  * expectation over the unit tests of the ratio of the median reference latency to the generated kernel's
  * latency; meaningful only for kernels that pass). Reading: both latencies are summarised by medians.
- *   ref_lat     device, float[T][S_ref]; gen_lat device, float[T][S_gen]: samples per unit test (no NaNs).
+ *   ref_lat     device, float[T][S_ref]; gen_lat device, float[T][S_gen]: samples per unit test (no NaNs;
+ *               a median that falls on a zero is reported as +0 whatever the zeros' signs).
  *   median_ref, median_gen, ratio   device, float[T]: medians (even count: fl((a + b) * 0.5) of the two
  *               middle values, the sum rounded first) and ratio[t] = fl(median_ref[t] / median_gen[t]).
  *   speedup     device, double[1]: the mean of ratio[] accumulated in binary64 in index order; 0 for T == 0.

@@ -1,9 +1,9 @@
 // gv_oracle.cpp -- TEST INFRASTRUCTURE, NOT PRODUCT CODE.
 //
 // Plain, slow, single-threaded CPU statement of what the batched output verifier computes:
-// the "tolerance based tensor comparison of output tensors produced by test functions" of the
-// paper's Section 3.1 (TritonBench-revised, second bullet), applied to one candidate output
-// against one reference output, as the inner step of the Evaluator's functionality test
+// the paper's Section 3.1 (TritonBench-revised, second bullet) has test outputs compared tensor
+// against tensor within tolerances rather than as printed text; here that comparison is applied to
+// one candidate output against one reference output, as the inner step of the Evaluator's functionality test
 // (Section 4.1) whose outcome feeds Execution Accuracy (Section 3.3: a kernel passes when it
 // satisfies all unit tests, i.e. n_mismatch == 0 for every test tensor).
 //
@@ -20,10 +20,13 @@
 // Every function here is pinned by tests/test_oracle_*.py against values fixed outside this
 // file (published SplitMix64 outputs, a hand-derived truth table, torch.isclose / numpy on the
 // host, closed forms and by-construction counts; the grouping by a hand-worked example, its
-// degenerate cases and a dictionary of byte strings).
+// degenerate cases and a dictionary of byte strings; the accuracies by the fractions the paper's
+// result tables print; the memory efficiency by a hand-worked example and exact rationals).
 
+#include <algorithm>
 #include <cstdint>
 #include <cstring>
+#include <vector>
 
 namespace {
 
@@ -450,16 +453,14 @@ int gvo_speedup(const float* ref_lat, const float* gen_lat, int64_t T, int32_t S
         for (int which = 0; which < 2; ++which) {
             const float* row = which == 0 ? ref_lat + t * S_ref : gen_lat + t * S_gen;
             const int32_t S = which == 0 ? S_ref : S_gen;
-            // selection by counting: the value of rank q is the x with (#smaller) <= q < (#smaller or equal)
-            float picked[2] = {0.0f, 0.0f};
-            const int32_t want[2] = {(S - 1) / 2, S / 2};
-            for (int w = 0; w < 2; ++w) {
-                for (int32_t a = 0; a < S; ++a) {
-                    int32_t less = 0, leq = 0;
-                    for (int32_t b = 0; b < S; ++b) { less += row[b] < row[a]; leq += row[b] <= row[a]; }
-                    if (less <= want[w] && want[w] < leq) { picked[w] = row[a]; break; }
-                }
-            }
+            // the definition: sort a copy of the row, take the middle value (odd count) or the two middle
+            // values (even count). A middle value that is a zero is taken as +0 (-0 and +0 compare equal, so
+            // their order after sorting is arbitrary).
+            std::vector<float> sorted(row, row + S);
+            std::sort(sorted.begin(), sorted.end());
+            float picked[2] = {sorted[(S - 1) / 2], sorted[S / 2]};
+            for (int w = 0; w < 2; ++w)
+                if (picked[w] == 0.0f) picked[w] = 0.0f;
             const float s2 = picked[0] + picked[1];
             med[which] = (S & 1) ? picked[0] : s2 * 0.5f;
         }
@@ -471,5 +472,85 @@ int gvo_speedup(const float* ref_lat, const float* gen_lat, int64_t T, int32_t S
     *speedup = T ? sum / static_cast<double>(T) : 0.0;
     return 0;
 }
+
+// Memory efficiency of a generated kernel from latency samples. Section 4.1 says that, for code that
+// passed the functionality test, the Evaluator assesses "latency and memory efficiency" and gives no
+// formula; the case study of Appendix A argues in bytes moved (one read and one write of the data
+// against two). Reading: per unit test, the bandwidth a kernel achieved on the bytes the test HAS to
+// move (inputs read once, outputs written once -- supplied by the caller), as a fraction of the
+// device's peak bandwidth; the latency of a test is summarised by the median of its samples, as for
+// Speedup (even count: fl32(fl32(a + b) * 0.5) of the two middle values; a zero median is +0).
+//   median[t]     binary32, from lat[t][0..S)
+//   bandwidth[t]  = (double)bytes[t] / (double)median[t]          one binary64 division
+//   efficiency[t] = bandwidth[t] / peak                           one binary64 division
+//   mean_eff      = (sum over t of efficiency[t], accumulated in binary64 in index order) / T; 0 for T == 0
+// peak is in bytes per unit of the latency samples (bytes per millisecond when the samples are in ms)
+// and must be finite and > 0. Samples are finite and > 0.
+int gvo_mem_efficiency(const float* lat, const uint64_t* bytes, int64_t T, int32_t S, double peak, float* median,
+                       double* bandwidth, double* efficiency, double* mean_eff) {
+    if (T < 0 || S < 1 || !(peak > 0.0) || !(peak <= 1.7976931348623157e308)) return 1;
+    double sum = 0.0;
+    for (int64_t t = 0; t < T; ++t) {
+        std::vector<float> sorted(lat + t * S, lat + (t + 1) * S);
+        std::sort(sorted.begin(), sorted.end());
+        float lo = sorted[(S - 1) / 2], hi = sorted[S / 2];
+        if (lo == 0.0f) lo = 0.0f;
+        if (hi == 0.0f) hi = 0.0f;
+        const float s2 = lo + hi;
+        median[t] = (S & 1) ? lo : s2 * 0.5f;
+        bandwidth[t] = static_cast<double>(bytes[t]) / static_cast<double>(median[t]);
+        efficiency[t] = bandwidth[t] / peak;
+        sum += efficiency[t];
+    }
+    *mean_eff = T ? sum / static_cast<double>(T) : 0.0;
+    return 0;
+}
+
+// Call accuracy and execution accuracy over a (kernel x run) matrix (Section 3.3: Call Accuracy is the
+// fraction of generated kernels that compile and run without error, Execution Accuracy the fraction
+// that satisfy all unit tests, counted only for kernels that compiled; Section 4.2 / Section 5.2: with R
+// independent runs per kernel both are reported as pass@k over the runs, k = 1..R). The denominator
+// is the number of kernels in the benchmark (the result tables divide the correctly generated kernels by
+// the total kernels in the dataset: 101 of 184 is printed as 54.89 %).
+// status[q*R + r], kernel q, run r: bit 0 = the run's kernel compiled and ran, bit 1 = it satisfied all
+// unit tests (the pass flag of gvo_exec_summary). A run counts for execution accuracy only with both.
+//   n_call[q], n_exec[q]   numbers of such runs of kernel q
+//   call_acc[k-1], exec_acc[k-1], k = 1..kmax <= R: (sum over q, in index order, in binary64, of
+//       pass@k(R, c_q)) / K with pass@k(R, c) = 1 - prod_{i<k} (R-c-i)/(R-i), factors multiplied left to
+//       right, each one division; exactly 1 when R - c < k. As fractions, not per cent. K == 0 gives 0.
+int gvo_accuracy_matrix(const uint8_t* status, int64_t K, int32_t R, int32_t kmax, int32_t* n_call, int32_t* n_exec,
+                        double* call_acc, double* exec_acc) {
+    if (K < 0 || R < 0 || kmax < 0 || kmax > R) return 1;
+    for (int64_t q = 0; q < K; ++q) {
+        int32_t a = 0, b = 0;
+        for (int32_t r = 0; r < R; ++r) {
+            const uint8_t s = status[q * R + r];
+            a += (s & 1) ? 1 : 0;
+            b += ((s & 3) == 3) ? 1 : 0;
+        }
+        n_call[q] = a;
+        n_exec[q] = b;
+    }
+    for (int32_t k = 1; k <= kmax; ++k) {
+        double sums[2] = {0.0, 0.0};
+        for (int64_t q = 0; q < K; ++q) {
+            const int32_t c[2] = {n_call[q], n_exec[q]};
+            for (int w = 0; w < 2; ++w) {
+                double pass_k = 1.0;
+                if (R - c[w] >= k) {
+                    double prod = 1.0;
+                    for (int32_t i = 0; i < k; ++i)
+                        prod = prod * (static_cast<double>(R - c[w] - i) / static_cast<double>(R - i));
+                    pass_k = 1.0 - prod;
+                }
+                sums[w] += pass_k;
+            }
+        }
+        call_acc[k - 1] = K ? sums[0] / static_cast<double>(K) : 0.0;
+        exec_acc[k - 1] = K ? sums[1] / static_cast<double>(K) : 0.0;
+    }
+    return 0;
+}
+
 
 }  // extern "C"

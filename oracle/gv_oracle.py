@@ -105,6 +105,12 @@ def lib() -> ctypes.CDLL:
         L.gvo_speedup.restype = ctypes.c_int
         L.gvo_speedup.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64, ctypes.c_int32, ctypes.c_int32,
                                   ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
+        L.gvo_mem_efficiency.restype = ctypes.c_int
+        L.gvo_mem_efficiency.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64, ctypes.c_int32, ctypes.c_double,
+                                         ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
+        L.gvo_accuracy_matrix.restype = ctypes.c_int
+        L.gvo_accuracy_matrix.argtypes = [ctypes.c_void_p, ctypes.c_int64, ctypes.c_int32, ctypes.c_int32, ctypes.c_void_p,
+                                          ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
         L.gvo_group.restype = ctypes.c_int
         L.gvo_group.argtypes = [ctypes.c_void_p, ctypes.c_int64, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
         _lib = L
@@ -253,3 +259,35 @@ def speedup(ref_lat: np.ndarray, gen_lat: np.ndarray):
     if rc:
         raise RuntimeError(f"gvo_speedup failed with {rc}")
     return mr[:T], mg[:T], ra[:T], float(sp[0])
+
+
+def mem_efficiency(lat: np.ndarray, nbytes: np.ndarray, peak: float):
+    """(median[T] float32, bandwidth[T], efficiency[T] float64, mean efficiency) for T x S latency samples,
+    the bytes each unit test has to move and the peak bandwidth in bytes per latency unit."""
+    a = np.ascontiguousarray(lat, dtype=np.float32)
+    b = np.ascontiguousarray(nbytes, dtype=np.uint64)
+    T = a.shape[0]
+    assert a.ndim == 2 and b.shape == (T,)
+    med = np.zeros(max(T, 1), dtype=np.float32)
+    bw, eff = (np.zeros(max(T, 1), dtype=np.float64) for _ in range(2))
+    mean = np.zeros(1, dtype=np.float64)
+    rc = lib().gvo_mem_efficiency(a.ctypes.data, b.ctypes.data, T, a.shape[1], float(peak), med.ctypes.data,
+                                  bw.ctypes.data, eff.ctypes.data, mean.ctypes.data)
+    if rc:
+        raise ValueError(f"gvo_mem_efficiency rejected its arguments ({rc})")
+    return med[:T], bw[:T], eff[:T], float(mean[0])
+
+
+def accuracy_matrix(status: np.ndarray, kmax: int):
+    """(n_call[K], n_exec[K] int32, call_acc[kmax], exec_acc[kmax] float64) for a K x R uint8 status matrix
+    (bit 0: the run compiled and ran, bit 1: it satisfied all unit tests)."""
+    s = np.ascontiguousarray(status, dtype=np.uint8)
+    assert s.ndim == 2
+    K, R = s.shape
+    nc, ne = (np.zeros(max(K, 1), dtype=np.int32) for _ in range(2))
+    ca, ea = (np.zeros(max(kmax, 1), dtype=np.float64) for _ in range(2))
+    rc = lib().gvo_accuracy_matrix(s.ctypes.data, K, R, kmax, nc.ctypes.data, ne.ctypes.data, ca.ctypes.data,
+                                   ea.ctypes.data)
+    if rc:
+        raise ValueError(f"gvo_accuracy_matrix rejected its arguments ({rc})")
+    return nc[:K], ne[:K], ca[:kmax], ea[:kmax]

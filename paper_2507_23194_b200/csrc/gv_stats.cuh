@@ -53,8 +53,11 @@ __device__ __forceinline__ void select_ranks(const float* row, int S, int q0, in
         const float x = row[a];
         int less = 0, leq = 0;
         for (int b = 0; b < S; ++b) { less += row[b] < x; leq += row[b] <= x; }
-        if (less <= q0 && q0 < leq) picked[0] = x;        // every thread that qualifies writes the same value
-        if (less <= q1 && q1 < leq) picked[1] = x;
+        // Every thread that qualifies holds an equal value; equal values are bit-identical except -0 / +0,
+        // so a zero is written as +0 and all writers agree on the bits.
+        const float v = x == 0.0f ? 0.0f : x;
+        if (less <= q0 && q0 < leq) picked[0] = v;
+        if (less <= q1 && q1 < leq) picked[1] = v;
     }
 }
 

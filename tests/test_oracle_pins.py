@@ -435,14 +435,29 @@ def test_config5_reduced_by_construction(oracle, align):
             assert int(r["first_mismatch"]) == (oracle.NO_INDEX if f["first"] is None else f["first"])
             if f.get("hash_equals_ref"):
                 assert int(r["hash"]) == ref_hash
-    if align == 0:
-        # tightly packed tensors: counts can be read off consecutive offsets as well
-        res2 = oracle.verify_ragged(wl.ref_buf.numpy(), wl.ref_off.numpy(), wl.cand_buf.numpy(),
-                                    wl.cand_off.numpy(), wl.dtypes.numpy(), wl.N, wl.atol, wl.rtol, wl.equal_nan)
-        # (only valid when no tensor needed alignment padding before it)
-        tight = all(int(wl.ref_off[t + 1] - wl.ref_off[t]) == wl.n_elems[t] * esz[int(wl.dtypes[t])] for t in range(wl.T))
-        if tight:
-            assert res2.tobytes() == res.tobytes()
+    # Counts read off consecutive offsets (no n_elems table): repack the same tensors back to back, the
+    # 4-byte types first and the 2-byte types after them, so that no tensor needs padding before it and the
+    # layout is tight whatever the recipe drew. Records are per tensor, so they must equal the ones above.
+    order = sorted(range(wl.T), key=lambda t: -esz[int(wl.dtypes[t])])
+    rb, cb, ro, co = bytearray(), bytearray(), [], []
+    ref_np, cand_np = wl.ref_buf.numpy(), wl.cand_buf.numpy()
+    for t in order:
+        nb = wl.n_elems[t] * esz[int(wl.dtypes[t])]
+        ro.append(len(rb))
+        rb += ref_np[int(wl.ref_off[t]):int(wl.ref_off[t]) + nb].tobytes()
+        for j in range(wl.N):
+            o = int(wl.cand_off[t * wl.N + j])
+            co.append(len(cb))
+            cb += cand_np[o:o + nb].tobytes()
+    ro.append(len(rb))
+    dts = np.array([int(wl.dtypes[t]) for t in order], dtype=np.uint8)
+    tight = all(ro[i + 1] - ro[i] == wl.n_elems[t] * esz[int(wl.dtypes[t])] for i, t in enumerate(order))
+    assert tight
+    res2 = oracle.verify_ragged(np.frombuffer(bytes(rb), dtype=np.uint8), np.array(ro, dtype=np.int64),
+                                np.frombuffer(bytes(cb), dtype=np.uint8), np.array(co, dtype=np.int64), dts, wl.N,
+                                wl.atol, wl.rtol, wl.equal_nan)
+    want = np.concatenate([res[t * wl.N:(t + 1) * wl.N] for t in order])
+    assert res2.tobytes() == want.tobytes()
 
 
 # --------------------------------------------------------------------------------------------
@@ -670,6 +685,112 @@ def test_speedup_hand_worked_and_numpy(oracle):
         assert ra.tolist() == (wr / wg).tolist()
         assert abs(sp - float(np.mean((wr / wg).astype(np.float64)))) <= 1e-12
     assert oracle.speedup(np.zeros((0, 3), dtype=np.float32), np.zeros((0, 2), dtype=np.float32))[3] == 0.0
+
+
+def test_speedup_median_is_sort_then_middle_and_zero_is_positive(oracle):
+    # both zeros in a row: whichever lands in the middle, the median is +0 (bit pattern 0)
+    ref = np.array([[-0.0, 0.0, -0.0, 0.0, 5.0], [0.0, -0.0, -0.0, 1.0, 1.0]], dtype=np.float32)
+    gen = np.array([[1.0, 1.0], [2.0, 2.0]], dtype=np.float32)
+    mr, mg, ra, _ = oracle.speedup(ref, gen)
+    assert mr.view(np.uint32).tolist() == [0, 0] and mg.tolist() == [1.0, 2.0] and ra.view(np.uint32).tolist() == [0, 0]
+    ref = np.array([[0.0, -0.0, -0.0, 0.0]], dtype=np.float32)             # even count: (+0) + (+0)
+    assert oracle.speedup(ref, gen[:1])[0].view(np.uint32).tolist() == [0]
+    # the middle of a sorted row, by hand: 9 distinct values in scrambled order
+    ref = np.array([[7, 1, 9, 3, 5, 2, 8, 4, 6]], dtype=np.float32)
+    gen = np.array([[7, 1, 9, 3, 5, 2, 8, 4]], dtype=np.float32)          # sorted 1 2 3 4 5 7 8 9 -> (4 + 5) / 2
+    mr, mg, ra, sp = oracle.speedup(ref, gen)
+    assert mr.tolist() == [5.0] and mg.tolist() == [4.5] and ra.tolist() == [np.float32(5.0) / np.float32(4.5)]
+
+
+# --------------------------------------------------------------------------------------------
+# memory efficiency from latency samples; call / execution accuracy over (kernel x run) matrices
+# --------------------------------------------------------------------------------------------
+def test_mem_efficiency_hand_worked_and_exact(oracle):
+    # two unit tests, latencies in ms, peak 8e9 bytes per ms (8 TB/s)
+    lat = np.array([[0.5, 0.25, 1.0], [2.0, 4.0, 8.0]], dtype=np.float32)      # medians 0.5 and 4
+    nbytes = np.array([2_000_000_000, 8_000_000_000], dtype=np.uint64)          # 4e9 B/ms and 2e9 B/ms
+    med, bw, eff, mean = oracle.mem_efficiency(lat, nbytes, 8e9)
+    assert med.tolist() == [0.5, 4.0] and bw.tolist() == [4e9, 2e9] and eff.tolist() == [0.5, 0.25] and mean == 0.375
+    # the case study's argument (Appendix A): a kernel that reads and writes the data twice moves twice the
+    # bytes a test has to move; at the same device bandwidth it takes twice as long and is half as efficient
+    lat1 = np.array([[1.0, 1.0, 1.0]], dtype=np.float32)
+    one = oracle.mem_efficiency(lat1, np.array([1 << 30], dtype=np.uint64), float(1 << 30))
+    two = oracle.mem_efficiency(lat1 * 2, np.array([1 << 30], dtype=np.uint64), float(1 << 30))
+    assert one[2].tolist() == [1.0] and two[2].tolist() == [0.5]
+    # random data against exact rationals (each result is one or two correctly rounded binary64 divisions)
+    rng = np.random.default_rng(12)
+    for T, S in [(1, 1), (9, 4), (30, 7)]:
+        lat = rng.lognormal(0, 0.5, (T, S)).astype(np.float32)
+        nbytes = rng.integers(1, 1 << 40, T).astype(np.uint64)
+        peak = 6.5e9
+        med, bw, eff, mean = oracle.mem_efficiency(lat, nbytes, peak)
+        srt = np.sort(lat, axis=1)
+        want_med = srt[:, S // 2] if S & 1 else (srt[:, S // 2 - 1] + srt[:, S // 2]) * np.float32(0.5)
+        assert med.tolist() == want_med.tolist()
+        for t in range(T):
+            exact_bw = Fraction(int(nbytes[t])) / Fraction(float(want_med[t]))
+            assert bw[t] == float(exact_bw)                                      # float(Fraction) rounds correctly
+            assert eff[t] == float(Fraction(bw[t]) / Fraction(peak))
+        assert abs(mean - float(sum(Fraction(e) for e in eff) / T)) <= 1e-15
+    assert oracle.mem_efficiency(np.zeros((0, 2), dtype=np.float32), np.zeros(0, dtype=np.uint64), 1.0)[3] == 0.0
+    with pytest.raises(ValueError):
+        oracle.mem_efficiency(lat1, np.array([1], dtype=np.uint64), 0.0)
+
+
+def test_accuracy_printed_fractions_of_the_paper(oracle):
+    # one run per kernel: the accuracy is correct / total, total = kernels in the benchmark
+    for row in _rows("paper_accuracy_tables.txt"):
+        correct, total, printed = row.split()
+        correct, total = int(correct), int(total)
+        status = np.zeros((total, 1), dtype=np.uint8)
+        status[:correct, 0] = 3
+        status[correct:correct + (total - correct) // 2, 0] = 1          # compiled, failed a test: counts for call only
+        nc, ne, ca, ea = oracle.accuracy_matrix(status, 1)
+        assert round(100 * ea[0], 2) == float(printed), row
+        assert int(ne.sum()) == correct and ca[0] == (correct + (total - correct) // 2) / total
+
+
+def test_accuracy_pass_at_k_endpoints_of_the_paper_and_exact_rationals(oracle):
+    from math import comb
+    rng = np.random.default_rng(13)
+    for row in _rows("paper_pass_at_k_endpoints.txt"):
+        K, R, with_good, good_total, p1, pR = row.split()
+        K, R, with_good = int(K), int(R), int(with_good)
+        # spread the good runs over `with_good` kernels (at least one each), any way
+        counts = np.zeros(K, dtype=np.int64)
+        counts[:with_good] = 1
+        if good_total != "*":
+            left = int(good_total) - with_good
+            while left:
+                q = int(rng.integers(0, with_good))
+                if counts[q] < R:
+                    counts[q] += 1
+                    left -= 1
+        counts = rng.permutation(counts)
+        status = np.zeros((K, R), dtype=np.uint8)
+        for q in range(K):
+            status[q, rng.permutation(R)[:counts[q]]] = 3
+        nc, ne, ca, ea = oracle.accuracy_matrix(status, R)
+        assert ne.tolist() == counts.tolist() and nc.tolist() == counts.tolist()
+        assert round(100 * ea[R - 1], 2) == float(pR), row
+        if p1 != "*":
+            assert round(100 * ea[0], 2) == float(p1), row
+        for k in range(1, R + 1):                                            # every k against exact rationals
+            exact = sum(1 - Fraction(comb(R - int(c), k), comb(R, k)) for c in counts) / K
+            assert abs(ea[k - 1] - float(exact)) <= 1e-13
+        assert np.all(np.diff(ea) >= -1e-15)
+    # bit 1 without bit 0 does not count; bit 0 alone counts for call accuracy only
+    status = np.array([[2, 2, 2], [1, 1, 0], [3, 0, 2]], dtype=np.uint8)
+    nc, ne, ca, ea = oracle.accuracy_matrix(status, 3)
+    assert nc.tolist() == [0, 2, 1] and ne.tolist() == [0, 0, 1]
+    assert ca[0] == (0 + 2 / 3 + (1.0 - 2 / 3)) / 3 and ca[2] == 2 / 3 and ea[2] == 1 / 3
+    # agreement with the per-kernel summary: one kernel's row gives that function's pass@k
+    rec = np.zeros(5, dtype=oracle.RESULT_DTYPE)
+    rec["n_mismatch"][[1, 4]] = 7
+    ok, c, pk = oracle.exec_summary(rec, 1, 5, 5)
+    _, ne, _, ea = oracle.accuracy_matrix((ok * 2 + 1).reshape(1, 5), 5)
+    assert ne.tolist() == [c] and ea.tolist() == pk.tolist()
+    assert oracle.accuracy_matrix(np.zeros((0, 4), dtype=np.uint8), 2)[2].tolist() == [0.0, 0.0]
 
 
 # --------------------------------------------------------------------------------------------

@@ -93,7 +93,8 @@ typedef struct gv_tol {
  *   ref        device, n_elems elements.
  *   cands      HOST array of N device pointers (copied before return).
  *   tol        host; ignored (may be NULL) for integer dtypes.
- *   results    device, N records, fully overwritten.
+ *   results    device, N records, fully overwritten (see gv_check for the one case in which they are
+ *              incomplete).
  *   ref_hash   device, one uint64, receives the reference's content hash; may be NULL.
  *   workspace  device, >= gv_workspace_bytes(0, N) bytes, 16-byte aligned; must stay untouched
  *              until the stream has passed this call. It carries a status word for gv_check() and
@@ -117,6 +118,7 @@ gv_status gv_verify_batch(const void* ref, const void* const* cands, int32_t N, 
  *   dtypes     device, uint8[T]: gv_dtype code of tensor t.
  *   n_elems    device, int64[T]: element count of tensor t; may be NULL when tensors are packed
  *              back to back, in which case it is (ref_off[t+1] - ref_off[t]) / element size.
+ *   T          at most 2^31 - 1 tensors; a table entry describing more than 2^40 bytes is a bad entry.
  *   results    device, T*N records, tensor-major; first_mismatch is relative to the tensor.
  *   workspace  device, >= gv_workspace_bytes(T, N) bytes, 16-byte aligned.
  * Offsets must be multiples of the tensor's element size. The tables live on the device and are
@@ -260,6 +262,36 @@ gv_status gv_exec_summary(const gv_result* results, int64_t T, int32_t N, int32_
 gv_status gv_speedup(const float* ref_lat, const float* gen_lat, int64_t T, int32_t S_ref, int32_t S_gen,
                      float* median_ref, float* median_gen, float* ratio, double* speedup, void* cuda_stream);
 
+/* Memory efficiency of a generated kernel from latency samples. Paper Section 4.1: for code that passed
+ * the functionality test the Evaluator assesses latency and memory efficiency; no formula is given, and
+ * the case study of Appendix A argues in bytes moved (one read and one write of the data against two).
+ * Reading: per unit test, the bandwidth achieved on the bytes the test HAS to move (inputs read once,
+ * outputs written once; the caller supplies them) as a fraction of the device's peak bandwidth, the
+ * latency summarised by the median of its samples exactly as in gv_speedup.
+ *   lat         device, float[T][S] latency samples (finite, > 0);  bytes  device, uint64[T].
+ *   peak        peak bandwidth in bytes per unit of the samples (bytes per ms for samples in ms); finite, > 0.
+ *   median      device, float[T];  bandwidth device, double[T] = (double)bytes[t] / (double)median[t];
+ *   efficiency  device, double[T] = bandwidth[t] / peak (each one correctly rounded binary64 division).
+ *   mean_efficiency  device, double[1]: mean of efficiency[] accumulated in index order; 0 for T == 0.
+ * 1 <= S <= GV_SAMPLES_MAX. Two launches. */
+gv_status gv_mem_efficiency(const float* lat, const uint64_t* bytes, int64_t T, int32_t S, double peak, float* median,
+                            double* bandwidth, double* efficiency, double* mean_efficiency, void* cuda_stream);
+
+/* Call accuracy and execution accuracy over a (kernel x run) matrix (paper Section 3.3: the fraction of
+ * generated kernels that compile and run, and the fraction that satisfy all unit tests, the latter counted
+ * only for kernels that compiled; Sections 4.2 and 5.2: with R independent runs per kernel both are
+ * reported as pass@k over the runs). The denominator is the number of kernels of the benchmark, as in the
+ * paper's result tables (correctly generated kernels / total kernels in the dataset).
+ *   status      device, uint8[K][R]: bit 0 = run r of kernel q compiled and ran, bit 1 = it satisfied all
+ *               unit tests (the pass flag gv_exec_summary produces). A run counts as correct only with both.
+ *   n_call, n_exec   device, int32[K]: such runs per kernel.
+ *   call_acc, exec_acc   device, double[kmax]: entry k-1 = (sum over the kernels, in index order, of
+ *               pass@k(R, count)) / K with pass@k as in gv_exec_summary; fractions, not per cent; 0 for K == 0.
+ * 0 <= kmax <= R <= GV_RUNS_MAX. Two launches. */
+#define GV_RUNS_MAX 1024
+gv_status gv_accuracy_matrix(const uint8_t* status, int64_t K, int32_t R, int32_t kmax, int32_t* n_call, int32_t* n_exec,
+                             double* call_acc, double* exec_acc, void* cuda_stream);
+
 /* Host-buffer convenience for callers whose outputs live in host memory: copies the reference and
  * the candidates host->device in slabs through `staging` (device, staging_bytes), verifies them and
  * copies the N records (and the reference hash) back to host memory. Copies and kernels are
@@ -281,8 +313,20 @@ size_t gv_host_staging_bytes(uint64_t n_elems, gv_dtype dt, int32_t slab);
 size_t gv_workspace_bytes(int64_t T, int32_t N);
 
 /* Synchronises cuda_stream, reads the status word of `workspace` and returns GV_OK,
- * GV_ERR_DEVICE_TIMEOUT or GV_ERR_BAD_TABLE (or GV_ERR_CUDA). Optional. */
+ * GV_ERR_DEVICE_TIMEOUT or GV_ERR_BAD_TABLE (or GV_ERR_CUDA). Optional, with one exception of
+ * meaning: every wait inside the kernels is bounded, and a warp whose wait expires stops working on
+ * its share of the data, so when gv_check reports GV_ERR_DEVICE_TIMEOUT the records (and ref_hash) of
+ * that call are INCOMPLETE AND MUST NOT BE USED -- they look like ordinary records. A caller that needs
+ * to rule this out calls gv_check; on healthy hardware the waits (tens of milliseconds of patience for
+ * a 512-byte copy) do not expire. GV_ERR_BAD_TABLE leaves the records of the well-formed tensors valid. */
 gv_status gv_check(const void* workspace, void* cuda_stream);
+
+/* Diagnostic for the path above (no counterpart in the paper): enqueues one warp that waits, through
+ * the kernels' own bounded wait with a limit of a few milliseconds, on a transfer that is never
+ * started, records the expiry in the status word of `workspace` (>= 256 bytes, 16-byte aligned; the
+ * word is overwritten) and returns by itself. gv_check(workspace) afterwards reports
+ * GV_ERR_DEVICE_TIMEOUT; the device and the workspace remain usable. */
+gv_status gv_selftest_wait_expiry(void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 const char* gv_status_string(gv_status s);
 const char* gv_last_cuda_error(void); /* text of the last CUDA error seen by this thread, or "" */

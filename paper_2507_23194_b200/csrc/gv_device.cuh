@@ -42,74 +42,9 @@ __device__ __forceinline__ uint32_t smem_u32(const void* p) {
 // ------------------------------------------------------------------------------------------
 // content hash
 // ------------------------------------------------------------------------------------------
-// The mixing function as the hot loops evaluate it. Integer add/shift/logic instructions and
-// integer multiply-add instructions execute on two different half-rate pipes of the SM; written
-// the plain way, the 64-bit xor-shifts and additions all land on the first and make it the
-// bottleneck of the whole kernel. Here part of them is expressed through 32x32->64 multiply-adds
-// by a power of two (z >> s and z << (32 - s) are the two halves of z * 2^(32 - s)), which moves
-// that work to the multiplier pipe. `two_pow` operands come from an opaque register so the
-// assembler keeps them as multiplies. Same value as the plain definition for every input
-// (checked bit for bit against the oracle).
-#ifndef GV_MAX2
-#define GV_MAX2 0
-#endif
-#ifndef GV_HASH_MASK
-#define GV_HASH_MASK 0x0
-#endif
-__device__ __forceinline__ uint32_t opaque_u32(uint32_t v) {
-    uint32_t r;
-    asm volatile("mov.u32 %0, %1;" : "=r"(r) : "r"(v));
-    return r;
-}
-// (hi:lo) ^= (hi:lo) >> S for 0 < S < 32, shifts done by the multiplier pipe
-template <int S>
-__device__ __forceinline__ void xorshift_mul(uint32_t& lo, uint32_t& hi, uint32_t two_pow /* 2^(32-S) */) {
-    uint32_t p_lo, p_hi, t;
-    asm("{\n\t.reg .u64 p;\n\t"
-        "mul.wide.u32 p, %3, %5;\n\t"          // hi * 2^(32-S): low half = hi << (32-S), high half = hi >> S
-        "mov.b64 {%0, %1}, p;\n\t"
-        "mad.hi.u32 %2, %4, %5, %0;\n\t}"      // (lo >> S) + (hi << (32-S)): disjoint bits, + is |
-        : "=r"(p_lo), "=r"(p_hi), "=r"(t)
-        : "r"(hi), "r"(lo), "r"(two_pow));
-    lo ^= t;
-    hi ^= p_hi;
-}
-template <int S>
-__device__ __forceinline__ void xorshift_alu(uint32_t& lo, uint32_t& hi) {
-    const uint32_t t = __funnelshift_r(lo, hi, S);
-    lo ^= t;
-    hi ^= hi >> S;
-}
-__device__ __forceinline__ void mul64_const(uint32_t& lo, uint32_t& hi, uint32_t c_lo, uint32_t c_hi) {
-    const uint64_t p = static_cast<uint64_t>(lo) * c_lo;
-    hi = static_cast<uint32_t>(p >> 32) + lo * c_hi + hi * c_lo;
-    lo = static_cast<uint32_t>(p);
-}
-// MASK bit 0/1/2: xor-shift 30/27/31 through the multiplier; bit 3: the "+ gamma" through a wide multiply-add
-template <int MASK>
-__device__ __forceinline__ uint64_t splitmix64_split(uint32_t lo, uint32_t hi, uint32_t one, uint32_t p2, uint32_t p5,
-                                                     uint32_t p1) {
-    if (MASK & 8) {
-        uint32_t t_hi;
-        asm("{\n\t.reg .u64 p;\n\t"
-            "mad.wide.u32 p, %2, %3, 0x9E3779B97F4A7C15;\n\t"
-            "mov.b64 {%0, %1}, p;\n\t}"
-            : "=r"(lo), "=r"(t_hi)
-            : "r"(lo), "r"(one));
-        hi += t_hi;
-    } else {
-        const uint64_t z = ((static_cast<uint64_t>(hi) << 32) | lo) + 0x9E3779B97F4A7C15ull;
-        lo = static_cast<uint32_t>(z);
-        hi = static_cast<uint32_t>(z >> 32);
-    }
-    if (MASK & 1) xorshift_mul<30>(lo, hi, p2); else xorshift_alu<30>(lo, hi);
-    mul64_const(lo, hi, 0x1CE4E5B9u, 0xBF58476Du);
-    if (MASK & 2) xorshift_mul<27>(lo, hi, p5); else xorshift_alu<27>(lo, hi);
-    mul64_const(lo, hi, 0x133111EBu, 0x94D049BBu);
-    if (MASK & 4) xorshift_mul<31>(lo, hi, p1); else xorshift_alu<31>(lo, hi);
-    return (static_cast<uint64_t>(hi) << 32) | lo;
-}
-
+// The mixing function of the content hash (the SplitMix64 finaliser), written the plain way. Moving part of
+// its shifts and additions to the multiplier pipe was measured (a dozen formulations) and brought nothing:
+// the plain form is what ships.
 __device__ __forceinline__ uint64_t splitmix64(uint64_t x) {
     uint64_t z = x + 0x9E3779B97F4A7C15ull;
     z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
@@ -135,16 +70,8 @@ __device__ __forceinline__ uint64_t hash_vec_full(const uint4& v, uint64_t k0) {
 
 // Full vector whose word indices fit 32 bits (tensors below 32 GiB): the high half of the index is
 // zero, so only the low halves are xored.
-// Powers of two (and 1) held in registers the assembler cannot see through; see splitmix64_split.
-struct HashConsts {
-    uint32_t one, p2, p5, p1;
-    __device__ __forceinline__ void init() {
-        one = opaque_u32(1u); p2 = opaque_u32(1u << 2); p5 = opaque_u32(1u << 5); p1 = opaque_u32(1u << 1);
-    }
-};
-__device__ __forceinline__ uint64_t hash_vec_full_k32(const uint4& v, uint32_t k0, const HashConsts& hc) {
-    return splitmix64_split<GV_HASH_MASK>(v.x ^ k0, v.y, hc.one, hc.p2, hc.p5, hc.p1) +
-           splitmix64_split<GV_HASH_MASK>(v.z ^ (k0 + 1u), v.w, hc.one, hc.p2, hc.p5, hc.p1);
+__device__ __forceinline__ uint64_t hash_vec_full_k32(const uint4& v, uint32_t k0) {
+    return splitmix64(pack64(v.x ^ k0, v.y)) + splitmix64(pack64(v.z ^ (k0 + 1u), v.w));
 }
 
 // ------------------------------------------------------------------------------------------
@@ -322,13 +249,6 @@ struct __align__(16) CtaAcc {
     }
 };
 
-#ifdef GV_DEBUG_COUNTERS
-__device__ unsigned long long g_dbg[8];
-#define GV_COUNT(i) atomicAdd(&g_dbg[i], 1ull)
-#else
-#define GV_COUNT(i) ((void)0)
-#endif
-
 struct TolF {
     float atol, rtol;
     int equal_nan;
@@ -461,14 +381,12 @@ __device__ __forceinline__ uint32_t rel_threshold_bits(uint32_t m_bits) {
 __device__ __forceinline__ void raise_maxabs(CtaAcc* s, uint32_t bits) {
     if (bits > *reinterpret_cast<volatile unsigned int*>(&s->maxabs)) {
         atomicMax(&s->maxabs, bits);
-
     }
 }
 __device__ __forceinline__ void raise_maxrel(CtaAcc* s, uint32_t bits) {
     if (bits > *reinterpret_cast<volatile unsigned int*>(&s->maxrel)) {
         atomicMax(&s->maxrel, bits);
         atomicMax(&s->thr, rel_threshold_bits(bits));
-
     }
 }
 
@@ -541,7 +459,6 @@ __device__ __forceinline__ bool vec_fast_float(const uint4& c, const RefVec<16 /
             if (ad[e] > tolc_of(fabsf(r.rf[e]), t)) { cnt += 1u; first_e = e; }
         }
         if (cnt) {
-            GV_COUNT(3);
             if (ADD_NOW) atomicAdd(&s->cnt, static_cast<unsigned long long>(cnt));
             else n_not_close += cnt;
             const unsigned long long idx = elem0 + first_e;
@@ -551,7 +468,6 @@ __device__ __forceinline__ bool vec_fast_float(const uint4& c, const RefVec<16 /
     if (raise_abs) raise_maxabs(s, vab);
     if (maybe_rel) {
         // some element may raise the relative maximum M: each one that passes the filter is examined
-        GV_COUNT(2);
         const float M = __uint_as_float(run.y);
         uint32_t best = 0u;
 #pragma unroll
@@ -665,8 +581,8 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
     return ok != 0;
 }
 // Bounded wait: returns false when the limit is reached (the caller flags a timeout and leaves).
-__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity) {
-    for (uint32_t i = 0; i < kWaitLimit; ++i) {
+__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity, uint32_t limit = kWaitLimit) {
+    for (uint32_t i = 0; i < limit; ++i) {
         if (mbar_try_wait(bar, parity)) return true;
     }
     return false;

@@ -1,14 +1,17 @@
 // gv_kernels.cu -- kernels and C ABI of the batched output verifier (sm_100a).
 //
-// Hot path (one call of gv_verify_batch): init records -> one persistent kernel in which every
-// CTA walks its share of reference tiles once per chunk of candidates. The reference tile is
-// brought into shared memory by a 1-D bulk async copy (TMA) completing on an mbarrier, double
-// buffered so the next tile arrives while the current one is compared against the chunk; each
-// thread then keeps its slice of the tile in registers and streams the same slice of every
-// candidate of the chunk with 128-bit loads. Per (thread, candidate) partials (hash, mismatch
-// count, max |d|) live in conflict-free shared-memory slots for the whole lifetime of the chunk,
-// so the warp/block reduction and the global integer atomics happen once per CTA and candidate,
-// not once per tile.
+// Hot path (one call of gv_verify_batch): record initialisation, a sampling pass that classifies the
+// candidates, then one persistent kernel in which every WARP works alone on 512-byte warp-tiles of the
+// reference (one 16-byte vector per lane) for one chunk of up to 16 candidates at a time. The warp's
+// reference tile arrives by a 1-D bulk async copy (TMA) on the warp's own mbarrier, double buffered;
+// each lane keeps its reference vector in registers for the whole chunk and streams its own 16 bytes
+// of every candidate through a private ring of asynchronous 16-byte copies in shared memory. A
+// candidate vector identical to the reference vector costs an identity test only (it shares the
+// reference's hash terms); vectors that differ are hashed and compared, either in place or through a
+// per-warp queue, depending on the candidate's class. Hash partials live in per-(candidate, lane)
+// shared-memory slots, the other statistics in per-CTA accumulators; one block combine and one set
+// of global integer atomics per (CTA, candidate). The comment above dense_kernel has the details; the
+// ragged path and the follow-on calls are described where they are defined.
 #include <cuda_runtime.h>
 #include <math.h>
 #include <stdint.h>
@@ -42,6 +45,21 @@ __global__ void init_results_kernel(gv_result* res, uint64_t count, uint32_t* st
     }
 }
 
+// A bounded wait that is certain to expire: the barrier expects 16 bytes of a bulk copy nobody issues.
+// The expiry is reported the way the verify kernels report theirs (status bit), and the kernel returns.
+__global__ void wait_expiry_kernel(uint32_t* status) {
+    __shared__ __align__(8) uint64_t bar;
+    if (threadIdx.x == 0) {
+        status[0] = 0;
+        mbar_init(&bar, 1);
+        mbar_fence_init();
+        mbar_expect_tx(&bar, 16);
+    }
+    __syncwarp();
+    const bool ok = mbar_wait_bounded(&bar, 0u, 256u);
+    if (!__all_sync(0xFFFFFFFFu, ok) && threadIdx.x == 0) atomicOr(status, kStatusTimeout);
+}
+
 // =============================================================================================
 // gv_hash
 // =============================================================================================
@@ -60,8 +78,6 @@ __global__ void __launch_bounds__(kThreads) hash_kernel(const unsigned char* buf
         // (eight independent mixing chains per thread); 32-bit word indices while they suffice
         const uint64_t nfull = nbytes / 16;
         const bool k32 = nbytes < (1ull << 35);
-        HashConsts hc;
-        hc.init();
         for (; v + 3 * stride < nfull; v += 4 * stride) {
             uint4 x[4];
 #pragma unroll
@@ -73,7 +89,7 @@ __global__ void __launch_bounds__(kThreads) hash_kernel(const unsigned char* buf
                     const uint64_t g0 = k0 * kGamma;
                     h += splitmix64(g0 ^ pack64(x[j].x, x[j].y)) + splitmix64((g0 + kGamma) ^ pack64(x[j].z, x[j].w));
                 } else {
-                    h += k32 ? hash_vec_full_k32(x[j], static_cast<uint32_t>(k0), hc) : hash_vec_full(x[j], k0);
+                    h += k32 ? hash_vec_full_k32(x[j], static_cast<uint32_t>(k0)) : hash_vec_full(x[j], k0);
                 }
             }
         }
@@ -146,17 +162,9 @@ struct DenseParams {
 //   * Accumulators: max |d|, max relative error, counts and the first index go to per-CTA shared
 //     accumulators only when they can change them. One block combine and one set of global
 //     integer atomics per (CTA, candidate).
-#ifndef GV_UNROLL
-#define GV_UNROLL 4
-#endif
-#ifndef GV_MINB_FLOAT
-#define GV_MINB_FLOAT 2
-#endif
 constexpr int kWarps = kThreads / 32;
-#ifndef GV_RING
-#define GV_RING 8
-#endif
-constexpr int kRing = GV_RING;            // asynchronous copies in flight per lane (power of two)
+constexpr int kRing = 8;                  // asynchronous copies in flight per lane (power of two)
+constexpr int kVisitBlock = 4;            // visits per unrolled block of the dense loop (divides kRing)
 constexpr int kWarpTile = 512;            // bytes of one warp-tile
 
 // Queue of differing vectors (one per warp). A candidate vector that differs from the reference
@@ -168,9 +176,7 @@ constexpr int kWarpTile = 512;            // bytes of one warp-tile
 constexpr int kQCap = 64;                           // entries (a power of two, >= 31 pending + 32 new)
 constexpr uint32_t kQPlane = kQCap * 16;            // bytes of one plane (candidate / reference / meta)
 constexpr size_t kQueueBytes = 3 * size_t(kQPlane);
-#ifndef GV_QDIRECT
-#define GV_QDIRECT 18                               // visits with at least this many differing lanes are compared in place
-#endif
+constexpr int kDenseLanes = 18;                     // a candidate whose sampled tiles average this many differing lanes (of 32) is compared in place
 
 template <int WARPS>
 struct DenseSmem {
@@ -184,16 +190,12 @@ struct DenseSmem {
     static constexpr size_t kTotal = kRefHashOff + 8;
 };
 
-// CTA shapes: 8 warps and about 98 KB of shared memory per CTA (ring 32, reference stages 8, hash slots
-// 32, queue 24, accumulators 1.3), hence 2 CTAs per SM for every dtype; the float kernels also need
-// the whole register file at that occupancy (up to 128 registers per thread); the integer ones are
-// compiled for 3 CTAs per SM, which keeps them at 80 registers.
-#ifndef GV_FLOAT_WARPS
-#define GV_FLOAT_WARPS 8
-#endif
+// CTA shape: 8 warps and about 98 KB of shared memory per CTA (ring 32, reference stages 8, hash slots
+// 32, queue 24, accumulators 1.3), hence 2 CTAs per SM for every dtype, which leaves each thread up to
+// 128 registers.
 template <int DT> struct DenseShape {
-    static constexpr int kWarpsPerCta = Traits<DT>::IS_FLOAT ? GV_FLOAT_WARPS : 8;
-    static constexpr int kCtasPerSm = Traits<DT>::IS_FLOAT ? GV_MINB_FLOAT : 3;
+    static constexpr int kWarpsPerCta = 8;
+    static constexpr int kCtasPerSm = 2;
 };
 
 // The exact rule for one vector the fast path could not settle; kept out of line so the hot loop
@@ -238,9 +240,7 @@ __device__ __forceinline__ void batch_entries(uint32_t qbase, uint32_t head, uin
         if constexpr (BIGK) {
             h = hash_vec_full(c, voff / 8);
         } else {
-            HashConsts hc;
-            hc.init();
-            h = hash_vec_full_k32(c, static_cast<uint32_t>(voff / 8), hc);
+            h = hash_vec_full_k32(c, static_cast<uint32_t>(voff / 8));
         }
         const uint2 sl = slots[k * 32];
         const uint64_t hs = pack64(sl.x, sl.y) + (h - h_ref);
@@ -270,7 +270,7 @@ __device__ __noinline__ void process_batch(uint32_t qbase, uint32_t head, uint32
 
 // Which candidates differ from the reference nearly everywhere? One CTA per candidate compares a
 // sample of its 512-byte tiles (evenly spread) with the reference, bytes only, and writes 1 when on
-// average at least GV_QDIRECT of the 32 vectors of a tile differ. The flag only selects which of
+// average at least kDenseLanes of the 32 vectors of a tile differ. The flag only selects which of
 // the dense kernel's two loops handles the candidate; both are correct for any data.
 constexpr int kSampleTiles = 64;
 __global__ void __launch_bounds__(kThreads) classify_kernel(const __grid_constant__ DenseParams p, uint64_t full_tiles,
@@ -291,7 +291,7 @@ __global__ void __launch_bounds__(kThreads) classify_kernel(const __grid_constan
     }
     if (lane == 0 && mine) atomicAdd(&s_total, mine);
     __syncthreads();
-    if (tid == 0) flags[blockIdx.x] = (S > 0 && s_total >= GV_QDIRECT * S) ? 1 : 0;
+    if (tid == 0) flags[blockIdx.x] = (S > 0 && s_total >= kDenseLanes * S) ? 1 : 0;
 }
 
 // BIGK: word indices of the hash need more than 32 bits (tensors of 32 GiB and more).
@@ -396,8 +396,6 @@ dense_kernel(const __grid_constant__ DenseParams p) {
     uint32_t phase[2] = {0u, 0u};
     uint64_t my_ref_hash = 0;
     bool timed_out = false;
-    HashConsts hc;
-    hc.init();
     // candidate bytes are read exactly once: mark them evict-first in L2 so that they do not push out the
     // reference, which every chunk reads again (+5 % on copies of a reference that fits L2)
     const uint64_t l2pol = l2_evict_first_policy();
@@ -482,7 +480,7 @@ dense_kernel(const __grid_constant__ DenseParams p) {
             uint64_t ref_sum = 0;      // sum of h_ref over the tiles of this chunk
             auto hash_of = [&](const uint4& v) -> uint64_t {
                 if constexpr (BIGK) return hash_vec_full(v, voff / 8);
-                else return hash_vec_full_k32(v, static_cast<uint32_t>(voff / 8), hc);
+                else return hash_vec_full_k32(v, static_cast<uint32_t>(voff / 8));
             };
             auto correct_slot = [&](const uint4& c, int k) {
                 const uint64_t d = hash_of(c) - h_ref;
@@ -508,7 +506,7 @@ dense_kernel(const __grid_constant__ DenseParams p) {
             };
             // one visit: candidate vector c (already read from the ring) against the held reference.
             // A lane wants a compare when its vector differs, or when the reference holds a NaN that
-            // equal_nan does not excuse. Dense differences (GV_QDIRECT lanes or more) are compared in
+            // equal_nan does not excuse. Dense differences (kDenseLanes lanes or more) are compared in
             // place against the values hoisted for the tile; sparse ones are queued.
             auto visit = [&](const uint4& c, const uint4& r, int k) {
                 const bool differs = (c.x != r.x) || (c.y != r.y) || (c.z != r.z) || (c.w != r.w);
@@ -556,7 +554,7 @@ dense_kernel(const __grid_constant__ DenseParams p) {
                 // The visits of the warp form one sequence (tile by tile, candidate by candidate); while a
                 // block is consumed its stages are refilled with the block two further on, which lies in
                 // the same tile, the next one or (4 candidates) the one after.
-                constexpr int U = GV_UNROLL;               // visits per unrolled block (divides kRing)
+                constexpr int U = kVisitBlock;
 #pragma unroll 1
                 for (int j = 0; j < kRing; ++j) {
                     const int tt = j / kg, cc = j - tt * kg;
@@ -706,12 +704,8 @@ dense_kernel(const __grid_constant__ DenseParams p) {
             }
         };
         if (gw < full_tiles && !timed_out) {
-#ifdef GV_ONLY_MODE0
-            fast_loop(std::integral_constant<int, 0>{});
-#else
             if (chunk_dense) fast_loop(std::integral_constant<int, 1>{});
             else fast_loop(std::integral_constant<int, 0>{});
-#endif
         }
 
         // ================= general loop: ragged tail, or some base not 16-byte aligned =================
@@ -780,6 +774,7 @@ struct RaggedParams {
 };
 
 constexpr int kRaggedTile = kWarpTile;      // ragged work is split into the same 512-byte warp-tiles
+constexpr int64_t kRaggedMaxBytes = int64_t(1) << 40;   // largest tensor a table entry may describe (1 TiB)
 
 // Pre-pass: validates the tables and turns sizes into an exclusive prefix of tile counts.
 // One CTA; T is at most a few million in practice (one pass of 1024-wide chunks).
@@ -805,7 +800,9 @@ __global__ void __launch_bounds__(1024) ragged_prepass_kernel(RaggedParams p) {
                     good = good && span >= 0 && span % esz == 0;
                     n = span / esz;
                 }
-                good = good && n >= 0 && ro >= 0 && ro % esz == 0;
+                // sizes beyond kRaggedMaxBytes per tensor are table errors: no device holds such a tensor, and
+                // the bound keeps n * esz and the running tile total (T < 2^31 tensors) far from overflow
+                good = good && n >= 0 && n <= kRaggedMaxBytes / esz && ro >= 0 && ro % esz == 0;
                 for (int j = 0; good && j < p.N; ++j) {
                     const int64_t co = p.cand_off[t * p.N + j];
                     good = co >= 0 && co % esz == 0;
@@ -1179,7 +1176,7 @@ __global__ void __launch_bounds__(kThreads, 2) ragged_kernel(const __grid_consta
     }
     int64_t t = lo;
     uint64_t item = begin;
-    while (item < end) {
+    while (item < end && t < p.T) {         // (t < T always holds for a consistent prefix table; the guard keeps a corrupted one from walking off its end)
         const uint64_t t_first = static_cast<uint64_t>(p.tile_prefix[t]);
         const uint64_t t_last = static_cast<uint64_t>(p.tile_prefix[t + 1]);
         if (t_last <= item) { ++t; continue; }                  // empty or already finished tensor
@@ -1298,13 +1295,6 @@ gv_status launch_dense(gv_dtype dt, const gv::DenseParams& p, int sm_count, cuda
 
 }  // namespace
 
-#ifdef GV_DEBUG_COUNTERS
-extern "C" void gv_debug_counters(unsigned long long* out, int reset) {
-    cudaMemcpyFromSymbol(out, gv::g_dbg, sizeof(unsigned long long) * 8);
-    if (reset) { unsigned long long z[8] = {0}; cudaMemcpyToSymbol(gv::g_dbg, z, sizeof(z)); }
-}
-#endif
-
 template <bool LANE2>
 gv_status launch_hash(const void* buf, uint64_t nbytes, uint64_t* out, void* cuda_stream) {
     if (!out || (nbytes > 0 && !buf)) return GV_ERR_INVALID_ARG;
@@ -1421,7 +1411,7 @@ gv_status gv_verify_ragged(const void* ref_base, const int64_t* ref_off, const v
                            const int64_t* cand_off, const uint8_t* dtypes, const int64_t* n_elems, int64_t T,
                            int32_t N, const gv_tol* tol, gv_result* results, void* workspace,
                            size_t workspace_bytes, void* cuda_stream) {
-    if (T < 0 || N < 0) return GV_ERR_INVALID_ARG;
+    if (T < 0 || T > 0x7FFFFFFFll || N < 0) return GV_ERR_INVALID_ARG;
     if (T > 0 && (!ref_base || !ref_off || !dtypes)) return GV_ERR_INVALID_ARG;
     if (T > 0 && N > 0 && (!cand_base || !cand_off || !results)) return GV_ERR_INVALID_ARG;
     if (!tol_valid(tol)) return GV_ERR_INVALID_ARG;
@@ -1606,6 +1596,41 @@ gv_status gv_speedup(const float* ref_lat, const float* gen_lat, int64_t T, int3
     return GV_OK;
 }
 
+gv_status gv_mem_efficiency(const float* lat, const uint64_t* bytes, int64_t T, int32_t S, double peak, float* median,
+                            double* bandwidth, double* efficiency, double* mean_efficiency, void* cuda_stream) {
+    if (T < 0 || T > 0x7FFFFFFFll || S < 1 || S > GV_SAMPLES_MAX || !mean_efficiency) return GV_ERR_INVALID_ARG;
+    if (!(peak > 0.0) || !isfinite(peak)) return GV_ERR_INVALID_ARG;
+    if (T > 0 && (!lat || !bytes || !median || !bandwidth || !efficiency)) return GV_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(lat) & 3u) || (reinterpret_cast<uintptr_t>(median) & 3u) ||
+        (reinterpret_cast<uintptr_t>(bytes) & 7u) || (reinterpret_cast<uintptr_t>(bandwidth) & 7u) ||
+        (reinterpret_cast<uintptr_t>(efficiency) & 7u) || (reinterpret_cast<uintptr_t>(mean_efficiency) & 7u))
+        return GV_ERR_MISALIGNED;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    if (T > 0)
+        gv::mem_efficiency_kernel<<<static_cast<unsigned>(T), gv::kStatsThreads, 0, st>>>(
+            lat, reinterpret_cast<const unsigned long long*>(bytes), S, peak, median, bandwidth, efficiency);
+    gv::mean_f64_kernel<<<1, 1, 0, st>>>(efficiency, T, mean_efficiency);
+    GV_CUDA(cudaGetLastError());
+    return GV_OK;
+}
+gv_status gv_accuracy_matrix(const uint8_t* status, int64_t K, int32_t R, int32_t kmax, int32_t* n_call, int32_t* n_exec,
+                             double* call_acc, double* exec_acc, void* cuda_stream) {
+    if (K < 0 || K > 0x7FFFFFFFll || R < 0 || R > GV_RUNS_MAX || kmax < 0 || kmax > R) return GV_ERR_INVALID_ARG;
+    if (K > 0 && (!n_call || !n_exec || (R > 0 && !status))) return GV_ERR_INVALID_ARG;
+    if (kmax > 0 && (!call_acc || !exec_acc)) return GV_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(n_call) & 3u) || (reinterpret_cast<uintptr_t>(n_exec) & 3u) ||
+        (reinterpret_cast<uintptr_t>(call_acc) & 7u) || (reinterpret_cast<uintptr_t>(exec_acc) & 7u))
+        return GV_ERR_MISALIGNED;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    if (K > 0)
+        gv::accuracy_counts_kernel<<<static_cast<unsigned>((K + gv::kStatsThreads - 1) / gv::kStatsThreads), gv::kStatsThreads, 0, st>>>(
+            status, K, R, n_call, n_exec);
+    if (kmax > 0)
+        gv::accuracy_at_k_kernel<<<static_cast<unsigned>(kmax), gv::kStatsThreads, 0, st>>>(n_call, n_exec, K, R, call_acc, exec_acc);
+    GV_CUDA(cudaGetLastError());
+    return GV_OK;
+}
+
 // ---- error profile of one candidate ----
 size_t gv_profile_workspace_bytes(void) {
     return 256 + static_cast<size_t>(gv::kProfileMaxCtas) *
@@ -1727,6 +1752,7 @@ gv_status gv_verify_batch_host(const void* ref_host, const void* const* cands_ho
     if (N > 0 && (!cands_host || !results_host)) return GV_ERR_INVALID_ARG;
     if (n_elems > 0 && !ref_host) return GV_ERR_INVALID_ARG;
     if (n_elems > (1ull << 60) / esz) return GV_ERR_INVALID_ARG;
+    if (dt <= GV_F16 && !tol_valid(tol)) return GV_ERR_INVALID_ARG;      // (before the first copy is enqueued)
     if (!staging || (reinterpret_cast<uintptr_t>(staging) & 255u)) return GV_ERR_WORKSPACE;
     if (staging_bytes < gv_host_staging_bytes(n_elems, dt, 1)) return GV_ERR_WORKSPACE;
     for (int32_t j = 0; j < N; ++j)
@@ -1768,6 +1794,19 @@ gv_status gv_verify_batch_host(const void* ref_host, const void* const* cands_ho
         if (N == 0) break;
     }
     GV_CUDA(cudaStreamSynchronize(st));
+    return GV_OK;
+}
+
+// Diagnostic: drives the bounded device-side wait to its limit on purpose. One warp arms an mbarrier
+// in its own shared memory for a transfer that is never started, polls it through the same bounded
+// wait the verify kernels use (with a limit of a few hundred polls, a few milliseconds at most),
+// records the expiry in the status word and returns. Nothing traps, faults or waits without limit;
+// the context stays usable.
+gv_status gv_selftest_wait_expiry(void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 15u) || workspace_bytes < 256) return GV_ERR_WORKSPACE;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    gv::wait_expiry_kernel<<<1, 32, 0, st>>>(static_cast<uint32_t*>(workspace));
+    GV_CUDA(cudaGetLastError());
     return GV_OK;
 }
 

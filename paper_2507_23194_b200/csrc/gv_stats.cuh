@@ -87,6 +87,75 @@ __global__ void __launch_bounds__(kStatsThreads) median_ratio_kernel(const float
     }
 }
 
+// one CTA per unit test: median latency, achieved bandwidth on the bytes the test has to move, and its
+// fraction of the peak (Section 4.1 names "memory efficiency" without a formula; the header states the reading)
+__global__ void __launch_bounds__(kStatsThreads) mem_efficiency_kernel(const float* lat, const unsigned long long* bytes, int S,
+                                                                       double peak, float* median, double* bandwidth,
+                                                                       double* efficiency) {
+    __shared__ float s_row[kSamplesMax];
+    __shared__ float s_pick[2];
+    const long long t = blockIdx.x;
+    const float* src = lat + t * S;
+    for (int a = threadIdx.x; a < S; a += kStatsThreads) s_row[a] = src[a];
+    __syncthreads();
+    select_ranks(s_row, S, (S - 1) / 2, S / 2, s_pick);
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        const float med = (S & 1) ? s_pick[0] : __fmul_rn(__fadd_rn(s_pick[0], s_pick[1]), 0.5f);
+        const double bw = __ddiv_rn(static_cast<double>(bytes[t]), static_cast<double>(med));
+        median[t] = med;
+        bandwidth[t] = bw;
+        efficiency[t] = __ddiv_rn(bw, peak);
+    }
+}
+// mean of T binary64 values accumulated in index order (one thread: the order is the definition)
+__global__ void mean_f64_kernel(const double* x, long long T, double* mean) {
+    double sum = 0.0;
+    for (long long t = 0; t < T; ++t) sum += x[t];
+    *mean = T ? sum / static_cast<double>(T) : 0.0;
+}
+
+// Call / execution accuracy over a (kernel x run) status matrix, K x R bytes (bit 0: compiled and ran,
+// bit 1: satisfied all unit tests). First the per-kernel counts, one thread per kernel ...
+__global__ void __launch_bounds__(kStatsThreads) accuracy_counts_kernel(const unsigned char* status, long long K, int R,
+                                                                        int* n_call, int* n_exec) {
+    const long long q = blockIdx.x * static_cast<long long>(kStatsThreads) + threadIdx.x;
+    if (q >= K) return;
+    int a = 0, b = 0;
+    for (int r = 0; r < R; ++r) {
+        const unsigned s = status[q * R + r];
+        a += (s & 1u) ? 1 : 0;
+        b += ((s & 3u) == 3u) ? 1 : 0;
+    }
+    n_call[q] = a;
+    n_exec[q] = b;
+}
+// ... then one CTA per k = blockIdx.x + 1: pass@k(R, c) depends on the count c alone, so the R + 1 possible
+// values are tabulated once (each the definition's left-to-right product), and two threads add the kernels'
+// values in index order, which is the order the definition sums in.
+constexpr int kRunsMax = 1024;
+__global__ void __launch_bounds__(kStatsThreads) accuracy_at_k_kernel(const int* n_call, const int* n_exec, long long K, int R,
+                                                                      double* call_acc, double* exec_acc) {
+    __shared__ double s_pass[kRunsMax + 1];
+    const int k = blockIdx.x + 1;
+    for (int c = threadIdx.x; c <= R; c += kStatsThreads) {
+        double v = 1.0;
+        if (R - c >= k) {
+            double prod = 1.0;
+            for (int i = 0; i < k; ++i) prod = prod * __ddiv_rn(static_cast<double>(R - c - i), static_cast<double>(R - i));
+            v = 1.0 - prod;
+        }
+        s_pass[c] = v;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0 || threadIdx.x == 32) {
+        const int* cnt = threadIdx.x == 0 ? n_call : n_exec;
+        double sum = 0.0;
+        for (long long q = 0; q < K; ++q) sum += s_pass[cnt[q]];
+        (threadIdx.x == 0 ? call_acc : exec_acc)[k - 1] = K ? sum / static_cast<double>(K) : 0.0;
+    }
+}
+
 // the mean of the ratios, accumulated in binary64 in index order (one thread: the order is the definition)
 __global__ void speedup_mean_kernel(const float* ratio, long long T, double* speedup) {
     double sum = 0.0;

@@ -47,7 +47,8 @@ class gv_tol(ctypes.Structure):
 
 
 EXPORTS = ["gv_verify_batch", "gv_verify_ragged", "gv_verify_ragged_noalloc", "gv_hash", "gv_hash2", "gv_group_candidates",
-           "gv_group_workspace_bytes", "gv_error_profile", "gv_profile_workspace_bytes", "gv_exec_summary", "gv_speedup", "gv_verify_batch_host", "gv_host_staging_bytes",
+           "gv_group_workspace_bytes", "gv_error_profile", "gv_profile_workspace_bytes", "gv_exec_summary", "gv_speedup",
+           "gv_mem_efficiency", "gv_accuracy_matrix", "gv_selftest_wait_expiry", "gv_verify_batch_host", "gv_host_staging_bytes",
            "gv_workspace_bytes", "gv_check", "gv_status_string", "gv_last_cuda_error", "gv_version"]
 
 
@@ -79,6 +80,12 @@ def _load() -> ctypes.CDLL:
     L.gv_exec_summary.argtypes = [vp, i64, i32, i32, vp, vp, vp, vp]
     L.gv_speedup.restype = ctypes.c_int
     L.gv_speedup.argtypes = [vp, vp, i64, i32, i32, vp, vp, vp, vp, vp]
+    L.gv_mem_efficiency.restype = ctypes.c_int
+    L.gv_mem_efficiency.argtypes = [vp, vp, i64, i32, ctypes.c_double, vp, vp, vp, vp, vp]
+    L.gv_accuracy_matrix.restype = ctypes.c_int
+    L.gv_accuracy_matrix.argtypes = [vp, i64, i32, i32, vp, vp, vp, vp, vp]
+    L.gv_selftest_wait_expiry.restype = ctypes.c_int
+    L.gv_selftest_wait_expiry.argtypes = [vp, sz, vp]
     L.gv_profile_workspace_bytes.restype = sz
     L.gv_profile_workspace_bytes.argtypes = []
     L.gv_verify_batch_host.restype = ctypes.c_int
@@ -241,6 +248,36 @@ def gv_speedup(ref_lat: torch.Tensor, gen_lat: torch.Tensor, stream: Optional[to
     _raise(lib.gv_speedup(ref_lat.data_ptr(), gen_lat.data_ptr(), T, ref_lat.shape[1], gen_lat.shape[1], mr.data_ptr(),
                           mg.data_ptr(), ra.data_ptr(), sp.data_ptr(), _stream_ptr(stream)))
     return mr[:T], mg[:T], ra[:T], sp
+
+
+def gv_mem_efficiency(lat: torch.Tensor, nbytes: torch.Tensor, peak: float, stream: Optional[torch.cuda.Stream] = None):
+    """Enqueue the memory efficiency for float32 latency samples of shape (T, S) and the int64/uint64 bytes each
+    unit test has to move; returns device tensors (median[T] float32, bandwidth[T], efficiency[T], mean[1] float64)."""
+    T = lat.shape[0]
+    dev = lat.device
+    med = torch.empty(max(T, 1), dtype=torch.float32, device=dev)
+    bw, eff = (torch.empty(max(T, 1), dtype=torch.float64, device=dev) for _ in range(2))
+    mean = torch.empty(1, dtype=torch.float64, device=dev)
+    _raise(lib.gv_mem_efficiency(lat.data_ptr(), nbytes.data_ptr(), T, lat.shape[1], float(peak), med.data_ptr(),
+                                 bw.data_ptr(), eff.data_ptr(), mean.data_ptr(), _stream_ptr(stream)))
+    return med[:T], bw[:T], eff[:T], mean
+
+
+def gv_accuracy_matrix(status: torch.Tensor, kmax: int, stream: Optional[torch.cuda.Stream] = None):
+    """Enqueue call / execution accuracy of a (K, R) uint8 status matrix; returns device tensors
+    (n_call[K], n_exec[K] int32, call_acc[kmax], exec_acc[kmax] float64)."""
+    K, R = status.shape
+    dev = status.device
+    nc, ne = (torch.empty(max(K, 1), dtype=torch.int32, device=dev) for _ in range(2))
+    ca, ea = (torch.empty(max(kmax, 1), dtype=torch.float64, device=dev) for _ in range(2))
+    _raise(lib.gv_accuracy_matrix(status.data_ptr(), K, R, kmax, nc.data_ptr(), ne.data_ptr(), ca.data_ptr(),
+                                  ea.data_ptr(), _stream_ptr(stream)))
+    return nc[:K], ne[:K], ca[:kmax], ea[:kmax]
+
+
+def gv_selftest_wait_expiry(workspace: torch.Tensor, stream: Optional[torch.cuda.Stream] = None) -> None:
+    """Enqueue the diagnostic kernel whose bounded wait expires; gv_check(workspace) then reports the timeout."""
+    _raise(lib.gv_selftest_wait_expiry(workspace.data_ptr(), workspace.numel(), _stream_ptr(stream)))
 
 
 def gv_hash2(buf: torch.Tensor, out: Optional[torch.Tensor] = None,

@@ -165,3 +165,79 @@ def test_stats_argument_errors_return_before_any_launch(gvlib):
     assert sp(a=None) == gv.GV_ERR_INVALID_ARG
     assert sp(a=0x1002) == gv.GV_ERR_MISALIGNED
     assert sp(out=0x6004) == gv.GV_ERR_MISALIGNED
+
+
+def test_new_aggregates_and_host_entry_argument_errors(gvlib):
+    gv = gvlib
+    me = lambda lat=0x1000, nb=0x2000, T=3, S=5, peak=1e9, med=0x3000, bw=0x4000, eff=0x5000, mean=0x6000: (
+        gv.lib.gv_mem_efficiency(lat, nb, T, S, peak, med, bw, eff, mean, None))
+    assert me(S=0) == gv.GV_ERR_INVALID_ARG
+    assert me(S=4097) == gv.GV_ERR_INVALID_ARG
+    assert me(peak=0.0) == gv.GV_ERR_INVALID_ARG
+    assert me(peak=float("inf")) == gv.GV_ERR_INVALID_ARG
+    assert me(peak=float("nan")) == gv.GV_ERR_INVALID_ARG
+    assert me(mean=None) == gv.GV_ERR_INVALID_ARG
+    assert me(nb=None) == gv.GV_ERR_INVALID_ARG
+    assert me(nb=0x2004) == gv.GV_ERR_MISALIGNED
+    assert me(bw=0x4004) == gv.GV_ERR_MISALIGNED
+    am = lambda st=0x1000, K=4, R=10, kmax=10, nc=0x2000, ne=0x3000, ca=0x4000, ea=0x5000: gv.lib.gv_accuracy_matrix(
+        st, K, R, kmax, nc, ne, ca, ea, None)
+    assert am(K=-1) == gv.GV_ERR_INVALID_ARG
+    assert am(kmax=11) == gv.GV_ERR_INVALID_ARG                      # more draws than runs
+    assert am(R=1025, kmax=1) == gv.GV_ERR_INVALID_ARG               # beyond GV_RUNS_MAX
+    assert am(st=None) == gv.GV_ERR_INVALID_ARG
+    assert am(ca=None) == gv.GV_ERR_INVALID_ARG
+    assert am(nc=0x2002) == gv.GV_ERR_MISALIGNED
+    assert am(ea=0x5004) == gv.GV_ERR_MISALIGNED
+    assert gv.lib.gv_selftest_wait_expiry(None, 256, None) == gv.GV_ERR_WORKSPACE
+    assert gv.lib.gv_selftest_wait_expiry(0x1000, 16, None) == gv.GV_ERR_WORKSPACE
+    # the host-buffer entry point checks the tolerances before it enqueues its first copy
+    ptrs = (ctypes.c_void_p * 1)(0x2000)
+    bad = gv.gv_tol(float("nan"), 0.0, 0, 0)
+    rc = gv.lib.gv_verify_batch_host(0x1000, ctypes.cast(ptrs, ctypes.c_void_p), 1, 16, 0, ctypes.byref(bad), 0x3000, None,
+                                     0x10000, 1 << 20, None)
+    assert rc == gv.GV_ERR_INVALID_ARG
+    rc = gv.lib.gv_verify_batch_host(0x1000, ctypes.cast(ptrs, ctypes.c_void_p), 1, 16, 0, None, 0x3000, None, 0x10000,
+                                     1 << 20, None)
+    assert rc == gv.GV_ERR_INVALID_ARG
+    # ragged: more than 2^31 - 1 tensors is an argument error
+    t = gv.gv_tol(1e-3, 1e-3, 0, 0)
+    assert gv.lib.gv_verify_ragged(0x1000, 0x2000, 0x3000, 0x4000, 0x5000, None, 1 << 31, 2, ctypes.byref(t), 0x6000, 0x7000,
+                                   1 << 40, None) == gv.GV_ERR_INVALID_ARG
+
+
+def test_tile_index_arithmetic_exhaustively():
+    """The decomposition every verify kernel relies on, restated on the host and checked for every size up to
+    four CTA tiles and a bit, at every alignment of the tail: a tensor of nbytes bytes is covered exactly once by
+    the full 512-byte warp-tiles [0, nbytes // 512) (fast loop, 32 lanes x 16 bytes) plus the tail tile whose
+    lanes hold the remaining full vectors and at most one partial vector; the words the hash sums are exactly
+    ceil(nbytes / 8); tile t belongs to warp t mod W of the grid; a ragged warp's contiguous stretch split is a
+    partition of the global tile sequence."""
+    tile, vec = 512, 16
+    for esz in (2, 4, 8):
+        for n in range(0, (4 * 8 * tile + 17 * esz) // esz + 1):
+            nbytes = n * esz
+            full_tiles, all_tiles = nbytes // tile, (nbytes + tile - 1) // tile
+            covered = full_tiles * tile
+            words = full_tiles * (tile // 8)
+            for t in range(full_tiles, all_tiles):                  # at most one
+                for lane in range(32):
+                    voff = t * tile + lane * vec
+                    rem = max(0, nbytes - voff)
+                    nvalid = vec // esz if rem >= vec else rem // esz
+                    covered += nvalid * esz
+                    words += 0 if nvalid == 0 else (2 if nvalid * esz > 8 else 1)
+            assert all_tiles - full_tiles in (0, 1)
+            assert covered == nbytes and words == (nbytes + 7) // 8, (esz, n)
+    for total in list(range(0, 70)) + [1000, 4097]:
+        for W in (1, 2, 7, 16, 2368):
+            per, extra = divmod(total, W)
+            spans, pos = [], 0
+            for gw in range(W):
+                begin = gw * per + min(gw, extra)
+                end = begin + per + (1 if gw < extra else 0)
+                assert begin == pos
+                pos = end
+                spans.append((begin, end))
+            assert pos == total
+            assert sorted(t for gw in range(W) for t in range(gw, total, W)) == list(range(total))   # dense: t mod W

@@ -1,10 +1,11 @@
 """GPU parity at the benchmark's full sizes, through the same call bench.py times.
 
 Every record of every candidate is checked against what the workload recipe fixes by construction
-(mismatch counts, first index, NaN/Inf counts, exact copies = zero record + reference hash), and a
-sample of candidates (several per recipe class) is checked byte for byte against the CPU oracle,
-which computes those records one by one on the host."""
+(mismatch counts, first index, NaN/Inf counts, exact copies = zero record + reference hash), and
+every record of every candidate (every tensor of the ragged batch) is checked byte for byte against
+the CPU oracle, which computes those records one by one on the host (one candidate per host thread)."""
 import ctypes
+import os
 from concurrent.futures import ThreadPoolExecutor
 
 import numpy as np
@@ -19,6 +20,7 @@ if not torch.cuda.is_available():
 from paper_2507_23194_b200 import gv, workloads as W  # noqa: E402
 
 DEV = "cuda:0"
+THREADS = max(1, min(32, len(os.sched_getaffinity(0))))      # host threads for the oracle (it releases the GIL)
 
 
 def host_bytes(t: torch.Tensor) -> np.ndarray:
@@ -61,20 +63,10 @@ def oracle_sample(oracle, wl, got, sample):
     def one(j):
         return j, oracle.verify(ref, host_bytes(wl.cands[j]), wl.dtype, wl.atol, wl.rtol, wl.equal_nan)
 
-    with ThreadPoolExecutor(max_workers=8) as ex:
+    with ThreadPoolExecutor(max_workers=THREADS) as ex:
         for j, want in ex.map(one, sample):
             assert got[j].tobytes() == want.tobytes(), (
                 f"{wl.name}: candidate {j} ({wl.facts[j]['class']})\n gpu    {got[j]}\n oracle {want}")
-
-
-def pick(wl, per_class):
-    seen, out = {}, []
-    for j, f in enumerate(wl.facts):
-        key = f["class"] + str(f.get("sigma", "")) + str(f.get("frac", ""))
-        if seen.get(key, 0) < per_class:
-            seen[key] = seen.get(key, 0) + 1
-            out.append(j)
-    return out
 
 
 def test_config2_full(oracle):
@@ -83,7 +75,7 @@ def test_config2_full(oracle):
     got, rh = run_dense(wl)
     assert rh == oracle.hash_bytes(host_bytes(wl.ref))
     check_facts(wl, got, rh)
-    oracle_sample(oracle, wl, got, pick(wl, 6))
+    oracle_sample(oracle, wl, got, range(len(wl.cands)))
 
 
 def test_config3_full(oracle):
@@ -92,7 +84,7 @@ def test_config3_full(oracle):
     got, rh = run_dense(wl)
     assert rh == oracle.hash_bytes(host_bytes(wl.ref))
     check_facts(wl, got, rh)
-    oracle_sample(oracle, wl, got, pick(wl, 2))
+    oracle_sample(oracle, wl, got, range(len(wl.cands)))
     del wl
     torch.cuda.empty_cache()
 
@@ -107,7 +99,7 @@ def test_config4_full(oracle, wide):
     for j, f in enumerate(wl.facts):                      # float fields stay zero in exact mode
         assert got[j]["max_abs_err"] == 0 and got[j]["max_rel_err"] == 0
         assert int(got[j]["n_nan_disagree"]) == 0 and int(got[j]["n_inf_disagree"]) == 0
-    oracle_sample(oracle, wl, got, pick(wl, 1))
+    oracle_sample(oracle, wl, got, range(len(wl.cands)))
     del wl
     torch.cuda.empty_cache()
 
@@ -126,9 +118,9 @@ def test_config5_full(oracle):
         assert int(got[i]["n_mismatch"]) == f["n_mismatch"], (i, f["class"])
         assert int(got[i]["first_mismatch"]) == (gv.GV_NO_INDEX if f["first"] is None else f["first"]), (i, f["class"])
         assert int(got[i]["n_nan_disagree"]) == 0 and int(got[i]["n_inf_disagree"]) == 0
-    # oracle on a sample of tensors: every 9th, plus the 16 largest and the 16 smallest
-    order = np.argsort(np.array(wl.n_elems))
-    sample = sorted(set(range(0, wl.T, 9)) | set(order[:16].tolist()) | set(order[-16:].tolist()))
+    # the oracle on every tensor, split among the host threads largest first so that the parts are balanced
+    order = np.argsort(-np.array(wl.n_elems))
+    sample = order.tolist()
     ref_buf, cand_buf = wl.ref_buf.cpu().numpy(), wl.cand_buf.cpu().numpy()
     ref_off, cand_off = wl.ref_off.cpu().numpy(), wl.cand_off.cpu().numpy()
     dtypes, n_el = wl.dtypes.cpu().numpy(), wl.n_elems_t.cpu().numpy()
@@ -140,8 +132,8 @@ def test_config5_full(oracle):
         return ts, oracle.verify_ragged(ref_buf, ro, cand_buf, co, dtypes[ts], wl.N, wl.atol, wl.rtol, wl.equal_nan,
                                         n_elems=n_el[ts])
 
-    chunks = [sample[i::8] for i in range(8)]
-    with ThreadPoolExecutor(max_workers=8) as ex:
+    chunks = [sample[i::4 * THREADS] for i in range(4 * THREADS)]
+    with ThreadPoolExecutor(max_workers=THREADS) as ex:
         for ts, want in ex.map(part, [c for c in chunks if c]):
             for a, t in enumerate(ts):
                 g = got[t * wl.N:(t + 1) * wl.N]
@@ -149,55 +141,92 @@ def test_config5_full(oracle):
                 assert g.tobytes() == w.tobytes(), f"tensor {t} (n={wl.n_elems[t]}, dtype {dtypes[t]})\n{g}\n{w}"
 
 
-def test_tensor_beyond_32_gib_uses_64_bit_word_indices(oracle):
-    """Maximum sizes: a 40 GiB int32 tensor (word indices of the hash pass 2^32, element indices pass
-    2^33). The oracle would need minutes for it, so the checks are properties that hold at any size:
-    an exact copy gives the zero record with the reference's hash; the reference hash equals what the
-    separate gv_hash kernel computes; a candidate changed in three known places differs from the copy
-    by exactly those three terms of the hash (recomputed here with Python integers), with the counts,
-    first index and exact maximum difference known by construction."""
+def _patterned_hash(oracle, n_words: int, word: int) -> int:
+    """Hash of a buffer whose every 64-bit word equals `word`: sum over k < n_words of splitmix64(k xor word).
+    For a block of 2^22 word indices starting at a multiple k0 of 2^22, (k0 + j) xor word = j xor (k0 xor word),
+    so the block's terms are the oracle's hash of a 32 MiB host buffer filled with the word (k0 xor word): the
+    34 GiB tensor's hash comes from the CPU oracle block by block without ever holding it on the host. One
+    block is also recomputed with numpy uint64 arithmetic straight from the formula."""
+    block = 1 << 22
+    M64 = (1 << 64) - 1
+
+    def part(k0):
+        m = min(block, n_words - k0)
+        return oracle.hash_bytes(np.full(m, (k0 ^ word) & M64, dtype=np.uint64))
+
+    with ThreadPoolExecutor(max_workers=THREADS) as ex:
+        total = sum(ex.map(part, range(0, n_words, block))) & M64
+    k0 = 5 * block
+    if k0 + block <= n_words:
+        g, c1, c2 = np.uint64(0x9E3779B97F4A7C15), np.uint64(0xBF58476D1CE4E5B9), np.uint64(0x94D049BB133111EB)
+        with np.errstate(over="ignore"):
+            z = (np.arange(k0, k0 + block, dtype=np.uint64) ^ np.uint64(word)) + g
+            z = (z ^ (z >> np.uint64(30))) * c1
+            z = (z ^ (z >> np.uint64(27))) * c2
+            z = z ^ (z >> np.uint64(31))
+            assert int(z.sum(dtype=np.uint64)) == part(k0)
+    return total
+
+
+def _big_case(oracle, torch_dtype, word_elems, places, bump):
+    """A 34+ GiB tensor whose every 64-bit word holds the same pattern (so its hash has a closed form that
+    numpy evaluates from the definition), an exact copy, and a candidate changed at three known places."""
+    esz = torch.empty(0, dtype=torch_dtype).element_size()
+    per_word = 8 // esz
+    n_words = (34 << 30) // 8 + 3                            # 34 GiB and a ragged tail: word indices pass 2^32
+    n = n_words * per_word
     free, _ = torch.cuda.mem_get_info()
-    n = 10 * (1 << 30)
-    need = 3 * n * 4 + (4 << 30)
+    need = 3 * n * esz + (4 << 30)
     if free < need:
         pytest.skip(f"needs {need >> 30} GiB of free device memory")
-    g = torch.Generator(device=DEV).manual_seed(99)
-    ref = torch.empty(n, dtype=torch.int32, device=DEV)
-    step = 1 << 28
-    for s in range(0, n, step):                               # fill in slices (bounded temporaries)
-        ref[s:s + step] = torch.randint(-(1 << 30), 1 << 30, (min(step, n - s),), generator=g, device=DEV,
-                                        dtype=torch.int32)
+    pat = torch.tensor(word_elems, dtype=torch_dtype, device=DEV)
+    word = int.from_bytes(host_bytes(pat).tobytes(), "little")
+    ref = pat.repeat(n_words)
+    assert ref.numel() == n
     copy = ref.clone()
     mod = ref.clone()
-    places = [5, (1 << 33) + 11, n - 1]
-    deltas = [7, -3, 1 << 20]
-    old = [int(ref[p]) for p in places]
-    for p, d in zip(places, deltas):
-        mod[p] += d
+    for p in places(n):
+        mod[p] = bump(mod[p])
     res = torch.empty((2, 64), dtype=torch.uint8, device=DEV)
     ws = torch.empty(gv.gv_workspace_bytes(0, 2), dtype=torch.uint8, device=DEV)
     rh = torch.zeros(1, dtype=torch.int64, device=DEV)
-    gv.gv_verify_batch(ref, [copy, mod], results=res, ref_hash=rh, workspace=ws)
+    gv.gv_verify_batch(ref, [copy, mod], 1e-3, 1e-3, False, results=res, ref_hash=rh, workspace=ws)
     torch.cuda.synchronize()
     assert gv.gv_check(ws) == gv.GV_OK
     got = gv.results_to_numpy(res)
-    ref_hash = int(rh.cpu().numpy().view(np.uint64)[0])
-    assert ref_hash == int(gv.gv_hash(ref).cpu().numpy().view(np.uint64)[0])
+    want_hash = _patterned_hash(oracle, n_words, word)       # pinned outside CUDA
+    assert int(rh.cpu().numpy().view(np.uint64)[0]) == want_hash, "reference hash of the dense kernel"
+    assert int(gv.gv_hash(ref).cpu().numpy().view(np.uint64)[0]) == want_hash, "gv_hash"
     zero = np.zeros((), dtype=gv.RESULT_DTYPE)
     zero["first_mismatch"] = gv.GV_NO_INDEX
-    zero["hash"] = ref_hash
+    zero["hash"] = want_hash
     assert got[0].tobytes() == zero.tobytes()
-    assert int(got[1]["n_mismatch"]) == 3 and int(got[1]["first_mismatch"]) == 5
-    assert int(got[1]["max_abs_diff_int"]) == 1 << 20
-    # hash delta in closed form: only the three touched 64-bit words change
+    # the changed candidate: only the touched words' terms differ, recomputed with Python integers
     M64 = (1 << 64) - 1
-    want = ref_hash
-    for p in places:
-        k = p // 2
-        w_old = int.from_bytes(host_bytes(ref[2 * k:2 * k + 2]).tobytes(), "little")
-        w_new = int.from_bytes(host_bytes(mod[2 * k:2 * k + 2]).tobytes(), "little")
-        want = (want - oracle.splitmix64(k ^ w_old) + oracle.splitmix64(k ^ w_new)) & M64
+    want = want_hash
+    for k in sorted({p // per_word for p in places(n)}):
+        w_new = int.from_bytes(host_bytes(mod[k * per_word:(k + 1) * per_word]).tobytes(), "little")
+        want = (want - oracle.splitmix64(k ^ word) + oracle.splitmix64(k ^ w_new)) & M64
     assert int(got[1]["hash"]) == want
-    assert old == [int(ref[p]) for p in places]
+    ps = sorted(places(n))
+    assert int(got[1]["n_mismatch"]) == len(ps) and int(got[1]["first_mismatch"]) == ps[0]
+    out = got[1].copy()
     del ref, copy, mod
     torch.cuda.empty_cache()
+    return out
+
+
+def test_int32_tensor_beyond_32_gib_uses_64_bit_word_indices(oracle):
+    """Maximum sizes: a 34 GiB int32 tensor (word indices of the hash pass 2^32, element indices pass 2^33).
+    The absolute hash is pinned by the closed form of a patterned buffer evaluated with numpy; counts, first
+    index and the exact maximum difference of the changed candidate are known by construction."""
+    got = _big_case(oracle, torch.int32, [0x1234567, -77], lambda n: [5, (1 << 33) + 11, n - 1], lambda v: v + (1 << 20))
+    assert int(got["max_abs_diff_int"]) == 1 << 20 and got["max_abs_err"] == 0
+
+
+def test_bf16_tensor_beyond_32_gib_uses_64_bit_word_indices(oracle):
+    """The same for a float dtype (the float instances of the kernel with 64-bit word indices): 34 GiB of bf16,
+    three elements raised by 0.5 (far outside the tolerance)."""
+    got = _big_case(oracle, torch.bfloat16, [1.0, -2.0, 0.5, 3.0], lambda n: [3, (1 << 34) + 6, n - 2], lambda v: v + 0.5)
+    assert got["max_abs_err"] == np.float32(0.5) and int(got["max_abs_diff_int"]) == 0
+    assert got["max_rel_err"] == np.float32(1.0)            # 0.5 -> 1.0 at two of the places; 3.0 -> 3.5 at the third

@@ -1,0 +1,134 @@
+"""GPU checks of the boundary's promises outside the plain parity cases: nothing is written outside the
+caller's records, inconsistent ragged tables are flagged without being followed (huge counts included), a
+bounded device-side wait that expires is reported and leaves the device usable, and the second hash lane's
+main loop agrees with the oracle on buffers large enough to reach it."""
+import numpy as np
+import pytest
+import torch
+
+pytestmark = pytest.mark.gpu
+
+if not torch.cuda.is_available():
+    pytest.skip("no CUDA device", allow_module_level=True)
+
+from paper_2507_23194_b200 import gv, workloads as W  # noqa: E402
+
+DEV = "cuda:0"
+
+
+def host_bytes(t):
+    return t.detach().contiguous().view(torch.uint8).cpu().numpy()
+
+
+def test_hash2_main_loop_on_large_buffers(oracle):
+    # the four-vector loop of the hash kernel runs only when a thread owns four vectors: 64 MiB and more
+    rng = np.random.default_rng(31)
+    data = torch.from_numpy(rng.integers(0, 256, size=(96 << 20) + 64, dtype=np.uint8))
+    dd = data.to(DEV)
+    for off, nbytes in [(0, 64 << 20), (0, (64 << 20) + 7), (16, (96 << 20) - 5), (0, (96 << 20) + 16), (3, 80 << 20)]:
+        h2 = gv.gv_hash2(dd[off:off + nbytes])
+        h1 = gv.gv_hash(dd[off:off + nbytes])
+        part = data[off:off + nbytes].numpy()
+        assert int(h2.cpu().numpy().view(np.uint64)[0]) == oracle.hash2_bytes(part), (off, nbytes)
+        assert int(h1.cpu().numpy().view(np.uint64)[0]) == oracle.hash_bytes(part), (off, nbytes)
+
+
+def test_records_have_guards_on_both_sides(oracle):
+    # dense: N records inside a larger buffer of sentinel bytes; ragged: the same with T * N records
+    wl = W.config1(DEV, n=(1 << 15) + 11)
+    N = len(wl.cands)
+    buf = torch.full((N + 8, 64), 0x5A, dtype=torch.uint8, device=DEV)
+    ws = torch.empty(gv.gv_workspace_bytes(0, N), dtype=torch.uint8, device=DEV)
+    rh_buf = torch.full((3,), 0x5A5A5A5A5A5A5A5A, dtype=torch.int64, device=DEV)
+    gv.gv_verify_batch(wl.ref, wl.cands, wl.atol, wl.rtol, wl.equal_nan, results=buf[4:4 + N], ref_hash=rh_buf[1:2],
+                       workspace=ws)
+    torch.cuda.synchronize()
+    assert gv.gv_check(ws) == gv.GV_OK
+    out = buf.cpu().numpy()
+    assert (out[:4] == 0x5A).all() and (out[4 + N:] == 0x5A).all()
+    assert rh_buf.cpu().tolist()[0] == 0x5A5A5A5A5A5A5A5A and rh_buf.cpu().tolist()[2] == 0x5A5A5A5A5A5A5A5A
+    want = oracle.verify_batch(host_bytes(wl.ref), [host_bytes(c) for c in wl.cands], oracle.F32, wl.atol, wl.rtol,
+                               wl.equal_nan)
+    assert out[4:4 + N].tobytes() == want.tobytes()
+    rw = W.config5(DEV, T=50, max_log2=13.0, seed=21)
+    cnt = rw.T * rw.N
+    buf = torch.full((cnt + 8, 64), 0x5A, dtype=torch.uint8, device=DEV)
+    ws = torch.empty(gv.gv_workspace_bytes(rw.T, rw.N), dtype=torch.uint8, device=DEV)
+    gv.gv_verify_ragged(rw.ref_buf, rw.ref_off, rw.cand_buf, rw.cand_off, rw.dtypes, rw.N, rw.atol, rw.rtol, rw.equal_nan,
+                        n_elems=rw.n_elems_t, results=buf[4:4 + cnt], workspace=ws)
+    torch.cuda.synchronize()
+    assert gv.gv_check(ws) == gv.GV_OK
+    out = buf.cpu().numpy()
+    assert (out[:4] == 0x5A).all() and (out[4 + cnt:] == 0x5A).all()
+    want = oracle.verify_ragged(rw.ref_buf.cpu().numpy(), rw.ref_off.cpu().numpy(), rw.cand_buf.cpu().numpy(),
+                                rw.cand_off.cpu().numpy(), rw.dtypes.cpu().numpy(), rw.N, rw.atol, rw.rtol, rw.equal_nan,
+                                n_elems=rw.n_elems_t.cpu().numpy())
+    assert out[4:4 + cnt].tobytes() == want.tobytes()
+
+
+@pytest.mark.parametrize("huge", [1 << 62, (1 << 61) + 1, (1 << 40) + 1, -5])      # each beyond the limit for every element size
+def test_huge_or_negative_counts_are_flagged_not_followed(oracle, huge):
+    # one table entry claims an absurd element count: the tensor's records stay zero records, the status word
+    # says so, every other tensor is verified as usual, and nothing outside the buffers is touched
+    rw = W.config5(DEV, T=24, max_log2=11.0, seed=22)
+    ne = rw.n_elems_t.clone()
+    victim = 7
+    ne[victim] = huge
+    ws = torch.empty(gv.gv_workspace_bytes(rw.T, rw.N), dtype=torch.uint8, device=DEV)
+    res = gv.gv_verify_ragged(rw.ref_buf, rw.ref_off, rw.cand_buf, rw.cand_off, rw.dtypes, rw.N, rw.atol, rw.rtol,
+                              rw.equal_nan, n_elems=ne, workspace=ws)
+    torch.cuda.synchronize()
+    assert gv.gv_check(ws) == gv.GV_ERR_BAD_TABLE
+    got = gv.results_to_numpy(res)
+    want = oracle.verify_ragged(rw.ref_buf.cpu().numpy(), rw.ref_off.cpu().numpy(), rw.cand_buf.cpu().numpy(),
+                                rw.cand_off.cpu().numpy(), rw.dtypes.cpu().numpy(), rw.N, rw.atol, rw.rtol, rw.equal_nan,
+                                n_elems=rw.n_elems_t.cpu().numpy())
+    zero = np.zeros((), dtype=gv.RESULT_DTYPE)
+    zero["first_mismatch"] = gv.GV_NO_INDEX
+    for t in range(rw.T):
+        for j in range(rw.N):
+            i = t * rw.N + j
+            assert got[i].tobytes() == (zero if t == victim else want[i]).tobytes(), (t, j)
+    # the same table through the entry point with the library's own scratch
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    res2 = torch.zeros((rw.T * rw.N, 64), dtype=torch.uint8, device=DEV)
+    gv.gv_verify_ragged_noalloc(rw.ref_buf, rw.ref_off, rw.cand_buf, rw.cand_off, rw.dtypes, rw.N, rw.atol, rw.rtol,
+                                rw.equal_nan, results=res2, n_elems=ne, status_out=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 2 and gv.results_to_numpy(res2).tobytes() == got.tobytes()
+
+
+def test_offsets_spanning_an_absurd_size_are_flagged(oracle):
+    # counts read off consecutive offsets: a span of 2^62 bytes is a bad entry, not a tensor. (It is the LAST
+    # tensor's span: an offsets table cannot make an inner span huge without also moving the next tensor's
+    # start out of the buffer, which the library has no means to detect -- buffer sizes are not arguments.)
+    T, N = 2, 2
+    ref = torch.arange(64, dtype=torch.int32, device=DEV)
+    offs = torch.tensor([0, 64, (1 << 62) + 64], dtype=torch.int64, device=DEV)
+    cand = torch.cat([ref, ref]).contiguous()
+    cand_off = torch.tensor([0, 256, 64, 320], dtype=torch.int64, device=DEV)
+    dtypes = torch.full((T,), 3, dtype=torch.uint8, device=DEV)
+    ws = torch.empty(gv.gv_workspace_bytes(T, N), dtype=torch.uint8, device=DEV)
+    res = gv.gv_verify_ragged(ref.view(torch.uint8), offs, cand.view(torch.uint8), cand_off, dtypes, N, 0.0, 0.0, False,
+                              workspace=ws)
+    torch.cuda.synchronize()
+    assert gv.gv_check(ws) == gv.GV_ERR_BAD_TABLE
+    got = gv.results_to_numpy(res)
+    assert int(got[0]["hash"]) == oracle.hash_bytes(host_bytes(ref[:16])) and int(got[0]["n_mismatch"]) == 0
+    assert int(got[1]["hash"]) == int(got[0]["hash"])
+    assert int(got[2]["hash"]) == 0 and int(got[3]["hash"]) == 0            # the flagged tensor: zero records
+
+
+def test_bounded_wait_that_expires_is_reported_and_the_device_stays_usable(oracle):
+    ws = torch.zeros(gv.gv_workspace_bytes(0, 4), dtype=torch.uint8, device=DEV)
+    gv.gv_selftest_wait_expiry(ws)
+    assert gv.gv_check(ws) == gv.GV_ERR_DEVICE_TIMEOUT                        # gv_check synchronises: the kernel returned
+    assert gv.lib.gv_status_string(gv.GV_ERR_DEVICE_TIMEOUT) == b"device-side wait timed out"
+    # an ordinary call on the same workspace right after it is clean and correct
+    wl = W.config1(DEV, n=(1 << 14) + 3)
+    res = gv.gv_verify_batch(wl.ref, wl.cands[:4], wl.atol, wl.rtol, wl.equal_nan, workspace=ws)
+    torch.cuda.synchronize()
+    assert gv.gv_check(ws) == gv.GV_OK
+    want = oracle.verify_batch(host_bytes(wl.ref), [host_bytes(c) for c in wl.cands[:4]], oracle.F32, wl.atol, wl.rtol,
+                               wl.equal_nan)
+    assert gv.results_to_numpy(res).tobytes() == want.tobytes()

@@ -34,7 +34,7 @@ def _both(wl):
     return gv.results_to_numpy(got), gv.results_to_numpy(want)
 
 
-def test_noalloc_matches_workspace_entry_point_on_two_calls_in_a_row():
+def test_noalloc_matches_workspace_entry_point_on_two_calls_in_a_row(oracle):
     # first call: a large batch that fills much of the scratch table ...
     big = W.config5(DEV, T=700, max_log2=14.0, seed=11)
     got, want = _both(big)
@@ -45,6 +45,11 @@ def test_noalloc_matches_workspace_entry_point_on_two_calls_in_a_row():
     assert got.tobytes() == want.tobytes()
     for i, f in enumerate(small.facts):
         assert int(got[i]["n_mismatch"]) == f["n_mismatch"]
+    # the small batch against the CPU oracle as well (not only one CUDA entry point against the other)
+    ref = oracle.verify_ragged(small.ref_buf.cpu().numpy(), small.ref_off.cpu().numpy(), small.cand_buf.cpu().numpy(),
+                               small.cand_off.cpu().numpy(), small.dtypes.cpu().numpy(), small.N, small.atol, small.rtol,
+                               small.equal_nan, n_elems=small.n_elems_t.cpu().numpy())
+    assert got.tobytes() == ref.tobytes()
     # and once more with the first batch
     got, want = _both(big)
     assert got.tobytes() == want.tobytes()

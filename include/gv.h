@@ -328,6 +328,13 @@ gv_status gv_check(const void* workspace, void* cuda_stream);
  * GV_ERR_DEVICE_TIMEOUT; the device and the workspace remain usable. */
 gv_status gv_selftest_wait_expiry(void* workspace, size_t workspace_bytes, void* cuda_stream);
 
+/* Diagnostic (no counterpart in the paper): the wrapping sum, modulo 2^64, of all little-endian 32-bit
+ * words of a device buffer, computed by a kernel that does nothing but stream the buffer with 128-bit
+ * loads. Timed on a buffer much larger than L2 it gives the read-only bandwidth of the device, the
+ * ceiling of the verify kernels (which only read), beside the read+write copy figure usually quoted.
+ *   buf  device, 16-byte aligned;  nbytes a multiple of 16;  out device, one uint64. Memset + one launch. */
+gv_status gv_selftest_read_sum(const void* buf, uint64_t nbytes, uint64_t* out, void* cuda_stream);
+
 const char* gv_status_string(gv_status s);
 const char* gv_last_cuda_error(void); /* text of the last CUDA error seen by this thread, or "" */
 uint32_t gv_version(void);            /* major << 16 | minor << 8 | patch */

@@ -60,6 +60,30 @@ __global__ void wait_expiry_kernel(uint32_t* status) {
     if (!__all_sync(0xFFFFFFFFu, ok) && threadIdx.x == 0) atomicOr(status, kStatusTimeout);
 }
 
+// Read-only bandwidth probe: the wrapping sum of all 32-bit words of a buffer. Eight independent 128-bit
+// streaming loads per thread and iteration, three integer additions per load: nothing but the memory
+// system limits it, so its rate is the read bandwidth a verify kernel could at best reach.
+__global__ void __launch_bounds__(kThreads) read_sum_kernel(const uint4* buf, uint64_t nvec, unsigned long long* out) {
+    const uint64_t stride = static_cast<uint64_t>(gridDim.x) * blockDim.x;
+    uint64_t v = blockIdx.x * static_cast<uint64_t>(blockDim.x) + threadIdx.x;
+    unsigned long long acc = 0;
+    for (; v + 7 * stride < nvec; v += 8 * stride) {
+        uint4 x[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) x[j] = ldg_stream(buf + v + j * stride);
+        // (the additions start only when all eight loads have been issued)
+        asm volatile("" ::: "memory");
+#pragma unroll
+        for (int j = 0; j < 8; ++j) acc += static_cast<unsigned long long>(x[j].x) + x[j].y + static_cast<unsigned long long>(x[j].z) + x[j].w;
+    }
+    for (; v < nvec; v += stride) {
+        const uint4 x = ldg_stream(buf + v);
+        acc += static_cast<unsigned long long>(x.x) + x.y + static_cast<unsigned long long>(x.z) + x.w;
+    }
+    acc = warp_sum_u64(acc);
+    if ((threadIdx.x & 31) == 0 && acc) atomicAdd(out, acc);
+}
+
 // =============================================================================================
 // gv_hash
 // =============================================================================================
@@ -162,6 +186,9 @@ struct DenseParams {
 //   * Accumulators: max |d|, max relative error, counts and the first index go to per-CTA shared
 //     accumulators only when they can change them. One block combine and one set of global
 //     integer atomics per (CTA, candidate).
+#ifndef GV_AB_EVERY
+#define GV_AB_EVERY 1
+#endif
 constexpr int kWarps = kThreads / 32;
 constexpr int kRing = 8;                  // asynchronous copies in flight per lane (power of two)
 constexpr int kVisitBlock = 4;            // visits per unrolled block of the dense loop (divides kRing)
@@ -460,6 +487,9 @@ dense_kernel(const __grid_constant__ DenseParams p) {
                     hoisted = true;
                 }
             };
+            auto hoist_now = [&](const uint4& r) {
+                if constexpr (IS_FLOAT) hoist_ref<DT>(r, tol, rv, rflags);
+            };
             // a candidate vector that is not bit-identical to the reference vector (ensure_hoisted done)
             // (mismatches of float vectors settled on the fast path are added to lane_cnt; the caller
             // merges lane_cnt into the accumulator once the warp has reconverged)
@@ -478,6 +508,12 @@ dense_kernel(const __grid_constant__ DenseParams p) {
             // chunk the candidate's partial is ref_sum + slot. Identical vectors cost no hash at all.
             uint64_t h_ref = 0;        // hash terms of this lane's reference vector (current tile)
             uint64_t ref_sum = 0;      // sum of h_ref over the tiles of this chunk
+            // Float chunks of flagged candidates in the block loop: when nearly every vector differs, the identity
+            // test decides nothing (a warp runs the compare whenever one of its lanes needs it), so every vector
+            // is hashed and compared outright and the slots collect whole hashes, not corrections.
+            constexpr bool kEveryVector = GV_AB_EVERY && MODE == 1 && IS_FLOAT;
+            const bool want_ref_hash = g == 0 && p.ref_hash != nullptr;
+            uint64_t ref_only = 0;     // the reference's own terms where the slots do not need them
             auto hash_of = [&](const uint4& v) -> uint64_t {
                 if constexpr (BIGK) return hash_vec_full(v, voff / 8);
                 else return hash_vec_full_k32(v, static_cast<uint32_t>(voff / 8));
@@ -566,9 +602,16 @@ dense_kernel(const __grid_constant__ DenseParams p) {
                 for (uint32_t i = 0; i < my_tiles; ++i) {
                     uint4 r;
                     if (!next_ref(i, r)) { timed_out = true; break; }
-                    h_ref = hash_of(r);
-                    ref_sum += h_ref;
-                    new_tile(r);
+                    if constexpr (kEveryVector) {
+                        // every candidate vector of this chunk is hashed and compared, identical or not: no
+                        // identity test, no shared reference terms; the reference's own hash only if it is asked for
+                        hoist_now(r);
+                        if (want_ref_hash) ref_only += hash_of(r);
+                    } else {
+                        h_ref = hash_of(r);
+                        ref_sum += h_ref;
+                        new_tile(r);
+                    }
 #pragma unroll 1
                     for (int k0 = 0; k0 < kg; k0 += U) {
                         const uint32_t stage0 = ring_base + vstage * 512u;
@@ -589,6 +632,25 @@ dense_kernel(const __grid_constant__ DenseParams p) {
                         uint4 c[U];
 #pragma unroll
                         for (int u = 0; u < U; ++u) c[u] = lds128(stage0 + u * 512u);
+                        if constexpr (kEveryVector) {
+                            uint32_t lane_cnt[U];
+#pragma unroll
+                            for (int u = 0; u < U; ++u) {
+                                lane_cnt[u] = 0u;
+                                const uint64_t hcand = hash_of(c[u]);
+                                const uint2 sl = slots[(k0 + u) * 32];
+                                const uint64_t hs = pack64(sl.x, sl.y) + hcand;
+                                slots[(k0 + u) * 32] = make_uint2(static_cast<uint32_t>(hs), static_cast<uint32_t>(hs >> 32));
+                                differing(c[u], r, k0 + u, lane_cnt[u]);
+                            }
+                            uint32_t any_cnt = 0u;
+#pragma unroll
+                            for (int u = 0; u < U; ++u) any_cnt |= lane_cnt[u];
+                            if (__any_sync(0xFFFFFFFFu, any_cnt != 0u)) {
+#pragma unroll
+                                for (int u = 0; u < U; ++u) merge_counts_converged(&cacc[k0 + u], lane_cnt[u]);
+                            }
+                        } else {
                         // identity test for all U visits; identical vectors are done
                         uint32_t diffmask = 0u;
 #pragma unroll
@@ -631,6 +693,7 @@ dense_kernel(const __grid_constant__ DenseParams p) {
                                     }
                                 }
                             }
+                        }
                         }
 #pragma unroll
                         for (int u = 0; u < U; ++u) {
@@ -692,7 +755,7 @@ dense_kernel(const __grid_constant__ DenseParams p) {
                 const uint64_t h = pack64(sl.x, sl.y) + ref_sum;
                 slots[k * 32] = make_uint2(static_cast<uint32_t>(h), static_cast<uint32_t>(h >> 32));
             }
-            if (g == 0 && p.ref_hash) my_ref_hash += ref_sum;
+            if (want_ref_hash) my_ref_hash += ref_sum + ref_only;
             if (timed_out) {
                 // flag it; give the copy that may still be in flight a second bounded chance to land
                 if (lane == 0) {
@@ -1806,6 +1869,27 @@ gv_status gv_selftest_wait_expiry(void* workspace, size_t workspace_bytes, void*
     if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 15u) || workspace_bytes < 256) return GV_ERR_WORKSPACE;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     gv::wait_expiry_kernel<<<1, 32, 0, st>>>(static_cast<uint32_t*>(workspace));
+    GV_CUDA(cudaGetLastError());
+    return GV_OK;
+}
+
+// Diagnostic: what a read-only stream reaches on this device (the verify kernels only read their inputs,
+// while the usual copy benchmark reads and writes).
+gv_status gv_selftest_read_sum(const void* buf, uint64_t nbytes, uint64_t* out, void* cuda_stream) {
+    if (!out || (nbytes > 0 && !buf)) return GV_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(buf) & 15u) || (nbytes & 15u) || (reinterpret_cast<uintptr_t>(out) & 7u)) return GV_ERR_MISALIGNED;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    int sm_count = 0;
+    gv_status rc = device_info(&sm_count);
+    if (rc != GV_OK) return rc;
+    GV_CUDA(cudaMemsetAsync(out, 0, sizeof(uint64_t), st));
+    const uint64_t nvec = nbytes / 16;
+    if (nvec == 0) return GV_OK;
+    uint64_t grid = (nvec + gv::kThreads - 1) / gv::kThreads;
+    const uint64_t cap = static_cast<uint64_t>(sm_count) * 8;
+    if (grid > cap) grid = cap;
+    gv::read_sum_kernel<<<static_cast<unsigned>(grid), gv::kThreads, 0, st>>>(static_cast<const uint4*>(buf), nvec,
+                                                                             reinterpret_cast<unsigned long long*>(out));
     GV_CUDA(cudaGetLastError());
     return GV_OK;
 }

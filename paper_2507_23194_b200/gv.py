@@ -48,7 +48,7 @@ class gv_tol(ctypes.Structure):
 
 EXPORTS = ["gv_verify_batch", "gv_verify_ragged", "gv_verify_ragged_noalloc", "gv_hash", "gv_hash2", "gv_group_candidates",
            "gv_group_workspace_bytes", "gv_error_profile", "gv_profile_workspace_bytes", "gv_exec_summary", "gv_speedup",
-           "gv_mem_efficiency", "gv_accuracy_matrix", "gv_selftest_wait_expiry", "gv_verify_batch_host", "gv_host_staging_bytes",
+           "gv_mem_efficiency", "gv_accuracy_matrix", "gv_selftest_wait_expiry", "gv_selftest_read_sum", "gv_verify_batch_host", "gv_host_staging_bytes",
            "gv_workspace_bytes", "gv_check", "gv_status_string", "gv_last_cuda_error", "gv_version"]
 
 
@@ -86,6 +86,8 @@ def _load() -> ctypes.CDLL:
     L.gv_accuracy_matrix.argtypes = [vp, i64, i32, i32, vp, vp, vp, vp, vp]
     L.gv_selftest_wait_expiry.restype = ctypes.c_int
     L.gv_selftest_wait_expiry.argtypes = [vp, sz, vp]
+    L.gv_selftest_read_sum.restype = ctypes.c_int
+    L.gv_selftest_read_sum.argtypes = [vp, u64, vp, vp]
     L.gv_profile_workspace_bytes.restype = sz
     L.gv_profile_workspace_bytes.argtypes = []
     L.gv_verify_batch_host.restype = ctypes.c_int
@@ -278,6 +280,15 @@ def gv_accuracy_matrix(status: torch.Tensor, kmax: int, stream: Optional[torch.c
 def gv_selftest_wait_expiry(workspace: torch.Tensor, stream: Optional[torch.cuda.Stream] = None) -> None:
     """Enqueue the diagnostic kernel whose bounded wait expires; gv_check(workspace) then reports the timeout."""
     _raise(lib.gv_selftest_wait_expiry(workspace.data_ptr(), workspace.numel(), _stream_ptr(stream)))
+
+
+def gv_selftest_read_sum(buf: torch.Tensor, out: Optional[torch.Tensor] = None,
+                         stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:
+    """Enqueue the read-only bandwidth probe (sum of the buffer's 32-bit words mod 2^64) -> device int64[1]."""
+    if out is None:
+        out = torch.empty(1, dtype=torch.int64, device=buf.device)
+    _raise(lib.gv_selftest_read_sum(buf.data_ptr(), buf.numel() * buf.element_size(), out.data_ptr(), _stream_ptr(stream)))
+    return out
 
 
 def gv_hash2(buf: torch.Tensor, out: Optional[torch.Tensor] = None,

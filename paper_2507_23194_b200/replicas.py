@@ -24,6 +24,22 @@ def shard_candidates(n_cands: int, world: int, rank: int) -> List[int]:
     return list(range(start, start + base + (1 if rank < extra else 0)))
 
 
+def shard_plan(n_cands: int, world: int, rank: int):
+    """(records per rank in rank order, this rank's candidate indices) for one batch split over `world` ranks."""
+    return [len(shard_candidates(n_cands, world, r)) for r in range(world)], shard_candidates(n_cands, world, rank)
+
+
+def verify_sharded(ref, cands, verify_local, world: int, rank: int) -> torch.Tensor:
+    """One batch, candidates split among the ranks: this rank verifies its own share with `verify_local(ref,
+    cands_of_this_rank) -> uint8 [n, 64]` (the CUDA library's dense call on a GPU; any stand-in with the same
+    contract on CPU ranks) and every rank receives the records of the whole batch in candidate order."""
+    counts, mine = shard_plan(len(cands), world, rank)
+    local = verify_local(ref, [cands[j] for j in mine])
+    if local.shape[0] != len(mine):
+        raise ValueError("verify_local returned a different number of records than candidates it was given")
+    return gather_records(local, counts)
+
+
 def max_over_ranks(ms: float, device="cpu") -> float:
     """The slowest rank's time (what a multi-GPU number must be quoted on)."""
     if not dist.is_initialized() or dist.get_world_size() == 1:

@@ -132,3 +132,12 @@ def test_bounded_wait_that_expires_is_reported_and_the_device_stays_usable(oracl
     want = oracle.verify_batch(host_bytes(wl.ref), [host_bytes(c) for c in wl.cands[:4]], oracle.F32, wl.atol, wl.rtol,
                                wl.equal_nan)
     assert gv.results_to_numpy(res).tobytes() == want.tobytes()
+
+
+def test_read_sum_probe_sums_the_words():
+    rng = np.random.default_rng(32)
+    for n_words in (0, 4, 4 * 257, (1 << 22) + 4 * 3, 40 << 20):
+        a = rng.integers(0, 1 << 32, size=n_words, dtype=np.uint64).astype(np.uint32)
+        d = torch.from_numpy(a.view(np.int32)).to(DEV)
+        out = gv.gv_selftest_read_sum(d)
+        assert int(out.cpu().numpy().view(np.uint64)[0]) == int(a.sum(dtype=np.uint64))

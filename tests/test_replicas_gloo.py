@@ -26,12 +26,16 @@ def _worker(rank, world, port, ret):
     from oracle import gv_oracle as O
     from paper_2507_23194_b200 import replicas as R, workloads as W
     wl = W.config1("cpu", n=5000)
-    mine = R.shard_candidates(len(wl.cands), world, rank)
     ref = wl.ref.numpy()
-    recs = O.verify_batch(ref, [wl.cands[j].numpy() for j in mine], O.F32, wl.atol, wl.rtol, wl.equal_nan)
-    local = torch.from_numpy(recs.view(np.uint8).reshape(-1, 64).copy())
-    counts = [len(R.shard_candidates(len(wl.cands), world, r)) for r in range(world)]
-    allrec = R.gather_records(local, counts)
+
+    def verify_local(ref_t, cands):          # the oracle stands in for the CUDA library's dense call on CPU ranks
+        recs = O.verify_batch(ref_t.numpy(), [c.numpy() for c in cands], O.F32, wl.atol, wl.rtol, wl.equal_nan)
+        return torch.from_numpy(recs.view(np.uint8).reshape(-1, 64).copy())
+
+    # the code path bench.py's candidate-sharded mode takes: plan, local verify, gather
+    counts, mine = R.shard_plan(len(wl.cands), world, rank)
+    assert mine == R.shard_candidates(len(wl.cands), world, rank) and sum(counts) == len(wl.cands)
+    allrec = R.verify_sharded(wl.ref, wl.cands, verify_local, world, rank)
     slowest = R.max_over_ranks(10.0 + rank)
     total = R.aggregate_throughput(1_000_000, slowest)
     if rank == 0:

@@ -217,7 +217,8 @@ gv_status gv_group_candidates(const gv_result* results, int64_t N, int32_t* grou
  *   out           device, one gv_profile, fully overwritten.   tol as in gv_verify_batch.
  *   workspace     device, >= gv_profile_workspace_bytes() bytes, 16-byte aligned.
  * Bases must be multiples of the element size (16-byte aligned bases take 128-bit loads). n_elems == 0
- * is legal (all zero, indices GV_NO_INDEX). Enqueues two memsets and two kernels. */
+ * is legal (all zero, indices GV_NO_INDEX). Enqueues one kernel (a cooperative launch: the device must
+ * support cudaLaunchCooperativeKernel, as every sm_100 part does). */
 #define GV_PROFILE_BUCKETS 66
 #define GV_PROFILE_LIST 8
 typedef struct gv_profile {

@@ -186,9 +186,6 @@ struct DenseParams {
 //   * Accumulators: max |d|, max relative error, counts and the first index go to per-CTA shared
 //     accumulators only when they can change them. One block combine and one set of global
 //     integer atomics per (CTA, candidate).
-#ifndef GV_AB_EVERY
-#define GV_AB_EVERY 1
-#endif
 constexpr int kWarps = kThreads / 32;
 constexpr int kRing = 8;                  // asynchronous copies in flight per lane (power of two)
 constexpr int kVisitBlock = 4;            // visits per unrolled block of the dense loop (divides kRing)
@@ -511,7 +508,7 @@ dense_kernel(const __grid_constant__ DenseParams p) {
             // Float chunks of flagged candidates in the block loop: when nearly every vector differs, the identity
             // test decides nothing (a warp runs the compare whenever one of its lanes needs it), so every vector
             // is hashed and compared outright and the slots collect whole hashes, not corrections.
-            constexpr bool kEveryVector = GV_AB_EVERY && MODE == 1 && IS_FLOAT;
+            constexpr bool kEveryVector = MODE == 1 && IS_FLOAT;
             const bool want_ref_hash = g == 0 && p.ref_hash != nullptr;
             uint64_t ref_only = 0;     // the reference's own terms where the slots do not need them
             auto hash_of = [&](const uint4& v) -> uint64_t {
@@ -831,6 +828,7 @@ struct RaggedParams {
     int N;
     gv_result* results;
     uint32_t* status;
+    uint32_t* counter;          // work counter of the main kernel (zeroed by the record initialisation)
     int64_t* tile_prefix;       // T+1, workspace
     float atol, rtol;
     int equal_nan;
@@ -838,6 +836,7 @@ struct RaggedParams {
 
 constexpr int kRaggedTile = kWarpTile;      // ragged work is split into the same 512-byte warp-tiles
 constexpr int64_t kRaggedMaxBytes = int64_t(1) << 40;   // largest tensor a table entry may describe (1 TiB)
+constexpr uint64_t kChunkBig = 256;                     // most tiles a warp takes at a time from the global tile sequence
 
 // Pre-pass: validates the tables and turns sizes into an exclusive prefix of tile counts.
 // One CTA; T is at most a few million in practice (one pass of 1024-wide chunks).
@@ -960,14 +959,15 @@ __device__ __noinline__ void ragged_differing(int dt, uint4 c, uint4 r, uint64_t
     }
 }
 // The warp's queue of differing vectors (all of one tensor, hence of one dtype): the n oldest entries.
+// (Streamed tiles only, hence tensors below 32 GiB: 32-bit word indices.)
 __device__ __noinline__ void ragged_batch(int dt, uint32_t qbase, uint32_t head, uint32_t n, uint2* slots, CtaAcc* wacc,
                                           TolF tol) {
     switch (dt) {
-        case GV_F32: batch_entries<GV_F32, true>(qbase, head, n, slots, wacc, tol); break;
-        case GV_BF16: batch_entries<GV_BF16, true>(qbase, head, n, slots, wacc, tol); break;
-        case GV_F16: batch_entries<GV_F16, true>(qbase, head, n, slots, wacc, tol); break;
-        case GV_I32: batch_entries<GV_I32, true>(qbase, head, n, slots, wacc, tol); break;
-        default: batch_entries<GV_I64, true>(qbase, head, n, slots, wacc, tol); break;
+        case GV_F32: batch_entries<GV_F32, false>(qbase, head, n, slots, wacc, tol); break;
+        case GV_BF16: batch_entries<GV_BF16, false>(qbase, head, n, slots, wacc, tol); break;
+        case GV_F16: batch_entries<GV_F16, false>(qbase, head, n, slots, wacc, tol); break;
+        case GV_I32: batch_entries<GV_I32, false>(qbase, head, n, slots, wacc, tol); break;
+        default: batch_entries<GV_I64, false>(qbase, head, n, slots, wacc, tol); break;
     }
 }
 // The partial vector at the end of a tensor: element by element through the general rule.
@@ -1058,10 +1058,15 @@ __device__ __noinline__ uint64_t ragged_tail(int dt, const unsigned char* ref, u
 }
 
 // Tiles [tile_begin, tile_end) of one tensor against kg of its candidates (pointers in wptr).
-// Full tiles with 16-byte aligned bases are streamed through the lane's asynchronous-copy ring
-// (reference vector first, then the kg candidate vectors of the tile, kRing copies in flight), so
-// the loads of the next tile or two fly while the current one is compared. The ragged tail tile and
-// unaligned tensors use synchronous element-sized loads.
+// Full tiles with 16-byte aligned bases are streamed through the lane's asynchronous-copy ring, so the
+// loads of the next tile or two fly while the current one is compared. The ragged tail tile, unaligned
+// tensors and tensors of 32 GiB or more (whose hash needs 64-bit word indices, which the streamed loops
+// do not carry) use synchronous element-sized loads.
+// FOUR: the instance for exactly four candidates per tensor (the usual handful of sampled runs): tile
+// by tile, the reference vector in a two-deep stage of its own and the four candidate vectors as one
+// block of the ring, two tiles in flight; one wait, one vote and one commit per tile, pointers in
+// registers. The other instance takes any number of candidates through one sequence of copies.
+template <bool FOUR>
 __device__ __forceinline__ void ragged_stretch(const RaggedParams& p, int dt, const unsigned char* ref, uint64_t n,
                                                uint64_t tile_begin, uint64_t tile_end, int kg, uint2* slots,
                                                CtaAcc* wacc, const unsigned char* const* wsrc, int lane,
@@ -1071,10 +1076,10 @@ __device__ __forceinline__ void ragged_stretch(const RaggedParams& p, int dt, co
     const uint64_t nbytes = n * esz;
     const TolF tol = {p.atol, p.rtol, p.equal_nan};
     const bool nan_matters = (dt <= GV_F16) && !p.equal_nan;
-    bool aligned = (reinterpret_cast<uintptr_t>(ref) & 15u) == 0;
-    for (int k = 0; k < kg; ++k) aligned = aligned && (reinterpret_cast<uintptr_t>(wptr[k]) & 15u) == 0;
+    bool streamed = (reinterpret_cast<uintptr_t>(ref) & 15u) == 0 && nbytes < (1ull << 35);
+    for (int k = 0; k < kg; ++k) streamed = streamed && (reinterpret_cast<uintptr_t>(wptr[k]) & 15u) == 0;
     const uint64_t full_end_all = nbytes / kWarpTile;                  // tiles [0, full_end_all) are full
-    const uint64_t full_end = aligned ? (tile_end < full_end_all ? tile_end : full_end_all) : tile_begin;
+    const uint64_t full_end = streamed ? (tile_end < full_end_all ? tile_end : full_end_all) : tile_begin;
 
     // As in the dense kernel, a vector identical to the reference vector contributes the reference
     // vector's own hash terms: those are summed once per tile (ref_sum), the slots only collect the
@@ -1104,94 +1109,86 @@ __device__ __forceinline__ void ragged_stretch(const RaggedParams& p, int dt, co
         }
     };
 
-    if (full_end > tile_begin && kg == 4) {
-        // ---- streamed part, exactly four candidates (the usual handful of sampled runs): tile by tile,
-        // the reference vector in a two-deep stage of its own and the four candidate vectors as one block
-        // of the ring, two tiles in flight; one wait, one vote and one commit per tile, pointers in registers.
-        const unsigned char* src_r = ref + lane * 16;
-        const unsigned char* src_c[4];
+    if (full_end > tile_begin) {
+        if constexpr (FOUR) {
+            const unsigned char* src_r = ref + lane * 16;
+            const unsigned char* src_c[4];
 #pragma unroll
-        for (int u = 0; u < 4; ++u) src_c[u] = wptr[u] + lane * 16;
-        auto issue_tile = [&](uint64_t tile, uint32_t half) {     // half: 0 or 1, which half of the ring / reference stage
-            if (tile < full_end) {
-                const uint64_t off = tile * kWarpTile;
-                cp_async16(refst_base + half * 512u, src_r + off);
+            for (int u = 0; u < 4; ++u) src_c[u] = wptr[u] + lane * 16;
+            auto issue_tile = [&](uint64_t tile, uint32_t half) {     // half: 0 or 1, which half of the ring / reference stage
+                if (tile < full_end) {
+                    const uint64_t off = tile * kWarpTile;
+                    cp_async16(refst_base + half * 512u, src_r + off);
 #pragma unroll
-                for (int u = 0; u < 4; ++u) cp_async16(ring_base + (half * 4u + u) * 512u, src_c[u] + off);
+                    for (int u = 0; u < 4; ++u) cp_async16(ring_base + (half * 4u + u) * 512u, src_c[u] + off);
+                }
+                cp_async_commit();
+            };
+            issue_tile(tile_begin, 0u);
+            issue_tile(tile_begin + 1, 1u);
+            uint32_t half = 0u;
+#pragma unroll 1
+            for (uint64_t tile = tile_begin; tile < full_end; ++tile) {
+                const uint64_t voff = tile * kWarpTile + lane * 16;     // (below 32 GiB: word indices fit 32 bits)
+                cp_async_wait<1>();                                   // this tile's group has landed
+                const uint4 r = lds128(refst_base + half * 512u);
+                uint4 c[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) c[u] = lds128(ring_base + (half * 4u + u) * 512u);
+                issue_tile(tile + 2, half);                           // refill the stages just read
+                half ^= 1u;
+                const bool force = nan_matters && vec_has_nan(dt, r);
+                const uint64_t h_ref = hash_vec_full_k32(r, static_cast<uint32_t>(voff / 8));
+                ref_sum += h_ref;
+                uint32_t diffmask = force ? 0xFu : 0u;
+#pragma unroll
+                for (int u = 0; u < 4; ++u)
+                    diffmask |= ((c[u].x != r.x) || (c[u].y != r.y) || (c[u].z != r.z) || (c[u].w != r.w)) ? (1u << u) : 0u;
+                if (__any_sync(0xFFFFFFFFu, diffmask != 0u)) {
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) queued_visit(c[u], r, h_ref, (diffmask >> u) & 1u, voff, u);
+                }
             }
-            cp_async_commit();
-        };
-        issue_tile(tile_begin, 0u);
-        issue_tile(tile_begin + 1, 1u);
-        uint32_t half = 0u;
+        } else {
+            // The copies form one sequence: per tile the reference vector, then the kg candidate vectors.
+            // The stage a visit has just consumed is refilled at once with the copy kRing places ahead,
+            // so consumer and producer share one stage counter. src[0] is the reference, src[1 + k]
+            // candidate k (wsrc, one table per warp in shared memory).
+            const uint64_t end_off = full_end * kWarpTile;
+            uint64_t issue_off = tile_begin * kWarpTile + lane * 16;        // this lane's byte offset of the next copy
+            int issue_j = 0;
+            auto issue_one = [&](uint32_t stage_addr) {
+                if (issue_off < end_off) {
+                    cp_async16(stage_addr, wsrc[issue_j] + issue_off);
+                    const bool wrap = issue_j == kg;
+                    issue_j = wrap ? 0 : issue_j + 1;
+                    issue_off += wrap ? kWarpTile : 0;
+                }
+                cp_async_commit();
+            };
 #pragma unroll 1
-        for (uint64_t tile = tile_begin; tile < full_end; ++tile) {
-            const uint64_t voff = tile * kWarpTile + lane * 16;
-            cp_async_wait<1>();                                   // this tile's group has landed
-            const uint4 r = lds128(refst_base + half * 512u);
-            uint4 c[4];
-#pragma unroll
-            for (int u = 0; u < 4; ++u) c[u] = lds128(ring_base + (half * 4u + u) * 512u);
-            issue_tile(tile + 2, half);                           // refill the stages just read
-            half ^= 1u;
-            const bool force = nan_matters && vec_has_nan(dt, r);
-            const uint64_t h_ref = hash_vec_full(r, voff / 8);
-            ref_sum += h_ref;
-            uint32_t diffmask = force ? 0xFu : 0u;
-#pragma unroll
-            for (int u = 0; u < 4; ++u)
-                diffmask |= ((c[u].x != r.x) || (c[u].y != r.y) || (c[u].z != r.z) || (c[u].w != r.w)) ? (1u << u) : 0u;
-            if (__any_sync(0xFFFFFFFFu, diffmask != 0u)) {
-#pragma unroll
-                for (int u = 0; u < 4; ++u) queued_visit(c[u], r, h_ref, (diffmask >> u) & 1u, voff, u);
-            }
-        }
-        cp_async_wait<0>();
-        if (qcount) {                                   // the tensor's accumulators close: drain the queue
-            __syncwarp();
-            ragged_batch(dt, qbase, qhead, qcount, slots, wacc, tol);
-            __syncwarp();
-        }
-    } else if (full_end > tile_begin) {
-        // ---- streamed part, any number of candidates ----
-        // The copies form one sequence: per tile the reference vector, then the kg candidate vectors.
-        // The stage a visit has just consumed is refilled at once with the copy kRing places ahead,
-        // so consumer and producer share one stage counter. src[0] is the reference, src[1 + k]
-        // candidate k (wsrc, one table per warp in shared memory).
-        const uint64_t end_off = full_end * kWarpTile;
-        uint64_t issue_off = tile_begin * kWarpTile + lane * 16;        // this lane's byte offset of the next copy
-        int issue_j = 0;
-        auto issue_one = [&](uint32_t stage_addr) {
-            if (issue_off < end_off) {
-                cp_async16(stage_addr, wsrc[issue_j] + issue_off);
-                const bool wrap = issue_j == kg;
-                issue_j = wrap ? 0 : issue_j + 1;
-                issue_off += wrap ? kWarpTile : 0;
-            }
-            cp_async_commit();
-        };
+            for (int j = 0; j < kRing; ++j) issue_one(ring_base + j * 512u);
+            uint32_t stage = 0;
 #pragma unroll 1
-        for (int j = 0; j < kRing; ++j) issue_one(ring_base + j * 512u);
-        uint32_t stage = 0;
-#pragma unroll 1
-        for (uint64_t tile = tile_begin; tile < full_end; ++tile) {
-            const uint64_t voff = tile * kWarpTile + lane * 16;
-            cp_async_wait<kRing - 1>();
-            uint32_t at = ring_base + stage * 512u;
-            const uint4 r = lds128(at);
-            stage = (stage + 1u) & (kRing - 1);
-            issue_one(at);
-            const bool force = nan_matters && vec_has_nan(dt, r);
-            const uint64_t h_ref = hash_vec_full(r, voff / 8);
-            ref_sum += h_ref;
-#pragma unroll 1
-            for (int k = 0; k < kg; ++k) {
+            for (uint64_t tile = tile_begin; tile < full_end; ++tile) {
+                const uint64_t voff = tile * kWarpTile + lane * 16;
                 cp_async_wait<kRing - 1>();
-                at = ring_base + stage * 512u;
-                const uint4 c = lds128(at);
+                uint32_t at = ring_base + stage * 512u;
+                const uint4 r = lds128(at);
                 stage = (stage + 1u) & (kRing - 1);
                 issue_one(at);
-                queued_visit(c, r, h_ref, force, voff, k);
+                const bool force = nan_matters && vec_has_nan(dt, r);
+                const uint64_t h_ref = hash_vec_full_k32(r, static_cast<uint32_t>(voff / 8));
+                ref_sum += h_ref;
+#pragma unroll 1
+                for (int k = 0; k < kg; ++k) {
+                    cp_async_wait<kRing - 1>();
+                    at = ring_base + stage * 512u;
+                    const uint4 c = lds128(at);
+                    stage = (stage + 1u) & (kRing - 1);
+                    issue_one(at);
+                    queued_visit(c, r, h_ref, force, voff, k);
+                }
             }
         }
         cp_async_wait<0>();
@@ -1202,8 +1199,8 @@ __device__ __forceinline__ void ragged_stretch(const RaggedParams& p, int dt, co
         }
     }
 
-    // ---- synchronous part: the tail tile, or every tile of an unaligned tensor (out of line: cold code
-    // whose registers the streaming loops should not pay for) ----
+    // ---- synchronous part: the tail tile, or every tile of a tensor that is not streamed (out of line: cold
+    // code whose registers the streaming loops should not pay for) ----
     if (full_end < tile_end) ref_sum += ragged_tail(dt, ref, nbytes, full_end, tile_end, kg, slots, wacc, wptr, tol, nan_matters);
     for (int k = 0; k < kg; ++k) {
         const uint2 sl = slots[k * 32];
@@ -1212,8 +1209,37 @@ __device__ __forceinline__ void ragged_stretch(const RaggedParams& p, int dt, co
     }
 }
 
-__global__ void __launch_bounds__(kThreads, 2) ragged_kernel(const __grid_constant__ RaggedParams p) {
-    extern __shared__ __align__(128) unsigned char smem[];
+// Work distribution of the ragged kernel. The tile sequence of all tensors is cut into chunks: the first
+// three quarters into large ones, the rest into small ones. A warp takes chunk `gw` first and further
+// chunks from a global counter, so warps whose tiles are costly (data that differs everywhere) simply
+// take fewer of them; the large chunks keep the cost of starting a chunk (locating its tensor, refilling
+// the copy pipeline, publishing partial records) small, the small ones keep the warps' finishing times
+// close. Chunk sizes follow the amount of work: about eight large chunks per warp, at most kChunkBig tiles
+// each (a batch of a few thousand tiny tensors is thus spread over all warps, one tile at a time).
+struct ChunkPlan {
+    uint64_t total, n_big, n_chunks, big_end;
+    uint32_t big, small;
+    __device__ __forceinline__ ChunkPlan(uint64_t total_tiles, uint64_t warps_in_grid) {
+        total = total_tiles;
+        const uint64_t want = total_tiles / (8 * warps_in_grid);
+        big = static_cast<uint32_t>(want < 1 ? 1 : (want > kChunkBig ? kChunkBig : want));
+        small = big / 4 ? big / 4 : 1u;
+        n_big = (total_tiles - total_tiles / 4) / big;
+        big_end = n_big * big;
+        n_chunks = n_big + (total_tiles - big_end + small - 1) / small;
+    }
+    __device__ __forceinline__ void range(uint64_t c, uint64_t& begin, uint64_t& end) const {
+        if (c < n_big) { begin = c * big; end = begin + big; }
+        else { begin = big_end + (c - n_big) * small; end = begin + small < total ? begin + small : total; }
+    }
+};
+
+// One tensor's tiles [tile_begin, tile_end) against all its candidates, from pointer set-up to the publication
+// of the partial records. Out of line on purpose: the streaming loops inside get a register allocation of
+// their own, separate from the chunk bookkeeping of the kernel that calls this.
+template <bool FOUR>
+__device__ __noinline__ void ragged_part(const RaggedParams& p, int64_t t, uint64_t tile_begin, uint64_t tile_end,
+                                         unsigned char* smem) {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     uint2* slots = reinterpret_cast<uint2*>(smem + RaggedSmem::kSlotOff) + size_t(warp) * kChunk * 32 + lane;
     CtaAcc* wacc = reinterpret_cast<CtaAcc*>(smem + RaggedSmem::kAccOff) + warp * kChunk;
@@ -1221,58 +1247,74 @@ __global__ void __launch_bounds__(kThreads, 2) ragged_kernel(const __grid_consta
     const uint32_t ring_base = smem_u32(smem + RaggedSmem::kRingOff) + (warp * kRing * 32 + lane) * 16;
     const uint32_t qbase = smem_u32(smem + RaggedSmem::kQueueOff) + warp * static_cast<uint32_t>(kQueueBytes);
     const uint32_t refst_base = smem_u32(smem + RaggedSmem::kRefOff) + (warp * 2 * 32 + lane) * 16;
+    const int dt = p.dtypes[t];
+    const int esz = elem_size(dt);
+    const uint64_t n = p.n_elems ? static_cast<uint64_t>(p.n_elems[t])
+                                 : static_cast<uint64_t>(p.ref_off[t + 1] - p.ref_off[t]) / esz;
+    const unsigned char* ref = p.ref_base + p.ref_off[t];
+    for (int c0 = 0; c0 < p.N; c0 += kChunk) {
+        const int kg = FOUR ? 4 : min(kChunk, p.N - c0);
+        __syncwarp();
+        if (lane < kg) {
+            wsrc[1 + lane] = p.cand_base + p.cand_off[t * p.N + c0 + lane];
+            wacc[lane].clear();
+        }
+        if (lane == 0) wsrc[0] = ref;
+        for (int k = 0; k < kg; ++k) slots[k * 32] = make_uint2(0u, 0u);
+        __syncwarp();
+        ragged_stretch<FOUR>(p, dt, ref, n, tile_begin, tile_end, kg, slots, wacc, wsrc, lane, ring_base, qbase, refst_base);
+        __syncwarp();
+        // leave the tensor (or this group of its candidates): combine and publish
+        for (int k = 0; k < kg; ++k) {
+            const uint2 sl = slots[k * 32];
+            const uint64_t h = warp_sum_u64(pack64(sl.x, sl.y));
+            if (lane == 0 && h) wacc[k].hash += h;
+        }
+        __syncwarp();
+        if (lane < kg) push_global(&p.results[t * p.N + c0 + lane], wacc[lane]);
+    }
+}
 
-    const uint64_t total = static_cast<uint64_t>(p.tile_prefix[p.T]);
+template <bool FOUR>
+__global__ void __launch_bounds__(kThreads, 2) ragged_kernel(const __grid_constant__ RaggedParams p) {
+    extern __shared__ __align__(128) unsigned char smem[];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const uint64_t gw = static_cast<uint64_t>(blockIdx.x) * kWarps + warp;
     const uint64_t GW = static_cast<uint64_t>(gridDim.x) * kWarps;
-    // contiguous stretch [begin, end) of the global tile sequence for this warp
-    const uint64_t per = total / GW, extra = total % GW;
-    const uint64_t begin = gw * per + (gw < extra ? gw : extra);
-    const uint64_t end = begin + per + (gw < extra ? 1 : 0);
-    if (begin >= end) return;
+    const ChunkPlan plan(static_cast<uint64_t>(p.tile_prefix[p.T]), GW);
+    uint64_t chunk = gw;
+    while (chunk < plan.n_chunks) {
+        uint32_t next = 0u;
+        if (lane == 0) next = atomicAdd(p.counter, 1u);     // reserved now, needed when this chunk is done
+        uint64_t begin, end;
+        plan.range(chunk, begin, end);
 
-    // tensor holding tile `begin`: last t with tile_prefix[t] <= begin (tensors without tiles are skipped)
-    int64_t lo = 0, hi = p.T;
-    while (hi - lo > 1) {
-        const int64_t mid = (lo + hi) >> 1;
-        if (static_cast<uint64_t>(p.tile_prefix[mid]) <= begin) lo = mid; else hi = mid;
-    }
-    int64_t t = lo;
-    uint64_t item = begin;
-    while (item < end && t < p.T) {         // (t < T always holds for a consistent prefix table; the guard keeps a corrupted one from walking off its end)
-        const uint64_t t_first = static_cast<uint64_t>(p.tile_prefix[t]);
-        const uint64_t t_last = static_cast<uint64_t>(p.tile_prefix[t + 1]);
-        if (t_last <= item) { ++t; continue; }                  // empty or already finished tensor
-        const int dt = p.dtypes[t];
-        const int esz = elem_size(dt);
-        const uint64_t n = p.n_elems ? static_cast<uint64_t>(p.n_elems[t])
-                                     : static_cast<uint64_t>(p.ref_off[t + 1] - p.ref_off[t]) / esz;
-        const unsigned char* ref = p.ref_base + p.ref_off[t];
-        const uint64_t tile_begin = item - t_first;
-        const uint64_t tile_end = (t_last < end ? t_last : end) - t_first;
-        for (int c0 = 0; c0 < p.N; c0 += kChunk) {
-            const int kg = min(kChunk, p.N - c0);
-            __syncwarp();
-            if (lane < kg) {
-                wsrc[1 + lane] = p.cand_base + p.cand_off[t * p.N + c0 + lane];
-                wacc[lane].clear();
-            }
-            if (lane == 0) wsrc[0] = ref;
-            for (int k = 0; k < kg; ++k) slots[k * 32] = make_uint2(0u, 0u);
-            __syncwarp();
-            ragged_stretch(p, dt, ref, n, tile_begin, tile_end, kg, slots, wacc, wsrc, lane, ring_base, qbase, refst_base);
-            __syncwarp();
-            // leave the tensor (or this group of its candidates): combine and publish
-            for (int k = 0; k < kg; ++k) {
-                const uint2 sl = slots[k * 32];
-                const uint64_t h = warp_sum_u64(pack64(sl.x, sl.y));
-                if (lane == 0 && h) wacc[k].hash += h;
-            }
-            __syncwarp();
-            if (lane < kg) push_global(&p.results[t * p.N + c0 + lane], wacc[lane]);
+        // tensor holding tile `begin`: last t with tile_prefix[t] <= begin (tensors without tiles are skipped).
+        // The warp searches together: 32 probes per round, three rounds for ten thousand tensors.
+        int64_t lo = 0, hi = p.T;
+        while (hi - lo > 1) {
+            const int64_t width = hi - lo;
+            const int64_t stride = (width + 31) / 32;
+            const int64_t idx = lo + (lane + 1) * stride;
+            const bool le = idx < hi && static_cast<uint64_t>(p.tile_prefix[idx]) <= begin;
+            const int k = __popc(__ballot_sync(0xFFFFFFFFu, le));     // the prefix is monotone: k leading lanes
+            const int64_t nlo = lo + k * stride;
+            hi = nlo + stride < hi ? nlo + stride : hi;
+            lo = nlo;
         }
-        item = t_first + tile_end;
-        ++t;
+        int64_t t = lo;
+        uint64_t item = begin;
+        while (item < end && t < p.T) {         // (t < T always holds for a consistent prefix table; the guard keeps a corrupted one from walking off its end)
+            const uint64_t t_first = static_cast<uint64_t>(p.tile_prefix[t]);
+            const uint64_t t_last = static_cast<uint64_t>(p.tile_prefix[t + 1]);
+            if (t_last > item) {                                    // (else: empty or already finished tensor)
+                const uint64_t tile_end = (t_last < end ? t_last : end) - t_first;
+                ragged_part<FOUR>(p, t, item - t_first, tile_end, smem);
+                item = t_first + tile_end;
+            }
+            ++t;
+        }
+        chunk = GW + __shfl_sync(0xFFFFFFFFu, next, 0);
     }
 }
 
@@ -1378,10 +1420,23 @@ gv_status launch_hash(const void* buf, uint64_t nbytes, uint64_t* out, void* cud
     return GV_OK;
 }
 template <int DT>
-gv_status launch_profile(gv::ProfileParams p, unsigned grid, cudaStream_t st) {
-    gv::profile_kernel<DT><<<grid, gv::kProfileThreads, 0, st>>>(p);
-    gv::profile_finalize_kernel<DT><<<1, gv::kProfileThreads, 0, st>>>(p, grid);
-    GV_CUDA(cudaGetLastError());
+gv_status launch_profile(gv::ProfileParams p, uint64_t want_ctas, int sm_count, cudaStream_t st) {
+    // one cooperative launch; the grid may not exceed what is resident at once
+    static int blocks_per_sm[64] = {0};
+    int dev = 0;
+    GV_CUDA(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) return GV_ERR_CUDA;
+    auto kern = gv::profile_kernel<DT>;
+    if (blocks_per_sm[dev] == 0) {
+        int b = 0;
+        GV_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b, kern, gv::kProfileThreads, 0));
+        blocks_per_sm[dev] = b > 0 ? b : 1;
+    }
+    uint64_t cap = static_cast<uint64_t>(sm_count) * blocks_per_sm[dev];
+    if (cap > gv::kProfileMaxCtas) cap = gv::kProfileMaxCtas;
+    const unsigned grid = static_cast<unsigned>(want_ctas < cap ? (want_ctas ? want_ctas : 1) : cap);
+    void* args[] = {&p};
+    GV_CUDA(cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(kern), dim3(grid), dim3(gv::kProfileThreads), args, 0, st));
     return GV_OK;
 }
 
@@ -1507,6 +1562,7 @@ gv_status gv_verify_ragged(const void* ref_base, const int64_t* ref_off, const v
     p.N = N;
     p.results = results;
     p.status = status;
+    p.counter = status + 1;
     p.tile_prefix = reinterpret_cast<int64_t*>(static_cast<unsigned char*>(workspace) + 256);
     p.atol = static_cast<float>(tol->atol);
     p.rtol = static_cast<float>(tol->rtol);
@@ -1518,14 +1574,15 @@ gv_status gv_verify_ragged(const void* ref_base, const int64_t* ref_off, const v
     int dev = 0;
     GV_CUDA(cudaGetDevice(&dev));
     if (blocks_per_sm[dev] == 0) {
-        GV_CUDA(cudaFuncSetAttribute(gv::ragged_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     static_cast<int>(gv::RaggedSmem::kTotal)));
+        for (auto kern : {gv::ragged_kernel<false>, gv::ragged_kernel<true>})
+            GV_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(gv::RaggedSmem::kTotal)));
         int b = 0;
-        GV_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b, gv::ragged_kernel, gv::kThreads, gv::RaggedSmem::kTotal));
+        GV_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b, gv::ragged_kernel<false>, gv::kThreads, gv::RaggedSmem::kTotal));
         blocks_per_sm[dev] = b > 0 ? b : 1;
     }
     const unsigned grid = static_cast<unsigned>(sm_count * blocks_per_sm[dev]);
-    gv::ragged_kernel<<<grid, gv::kThreads, gv::RaggedSmem::kTotal, st>>>(p);
+    if (N == 4) gv::ragged_kernel<true><<<grid, gv::kThreads, gv::RaggedSmem::kTotal, st>>>(p);
+    else gv::ragged_kernel<false><<<grid, gv::kThreads, gv::RaggedSmem::kTotal, st>>>(p);
     GV_CUDA(cudaGetLastError());
     return GV_OK;
 }
@@ -1598,6 +1655,7 @@ gv_status gv_verify_ragged_noalloc(const void* ref_base, const int64_t* ref_off,
     p.N = N;
     p.results = results;
     p.status = status_out ? status_out : status;
+    p.counter = status + 1;
     p.tile_prefix = reinterpret_cast<int64_t*>(scratch + 256);
     p.atol = static_cast<float>(tol->atol);
     p.rtol = static_cast<float>(tol->rtol);
@@ -1607,14 +1665,15 @@ gv_status gv_verify_ragged_noalloc(const void* ref_base, const int64_t* ref_off,
 
     static int blocks_per_sm[64] = {0};
     if (blocks_per_sm[dev] == 0) {
-        GV_CUDA(cudaFuncSetAttribute(gv::ragged_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     static_cast<int>(gv::RaggedSmem::kTotal)));
+        for (auto kern : {gv::ragged_kernel<false>, gv::ragged_kernel<true>})
+            GV_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(gv::RaggedSmem::kTotal)));
         int b = 0;
-        GV_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b, gv::ragged_kernel, gv::kThreads, gv::RaggedSmem::kTotal));
+        GV_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b, gv::ragged_kernel<false>, gv::kThreads, gv::RaggedSmem::kTotal));
         blocks_per_sm[dev] = b > 0 ? b : 1;
     }
     const unsigned grid = static_cast<unsigned>(sm_count * blocks_per_sm[dev]);
-    gv::ragged_kernel<<<grid, gv::kThreads, gv::RaggedSmem::kTotal, st>>>(p);
+    if (N == 4) gv::ragged_kernel<true><<<grid, gv::kThreads, gv::RaggedSmem::kTotal, st>>>(p);
+    else gv::ragged_kernel<false><<<grid, gv::kThreads, gv::RaggedSmem::kTotal, st>>>(p);
     GV_CUDA(cudaGetLastError());
     return GV_OK;
 }
@@ -1731,19 +1790,13 @@ gv_status gv_error_profile(const void* ref, const void* cand, uint64_t n_elems, 
     p.cta_worst = reinterpret_cast<gv::ProfileWorst*>(ws);
     p.cta_first = reinterpret_cast<unsigned long long*>(ws + static_cast<size_t>(gv::kProfileMaxCtas) * sizeof(gv::ProfileWorst));
     const uint64_t tiles = (n_elems * esz + 511) / 512;
-    uint64_t grid = (tiles + gv::kProfileWarps - 1) / gv::kProfileWarps;
-    const uint64_t cap = static_cast<uint64_t>(sm_count) * 8 < gv::kProfileMaxCtas ? static_cast<uint64_t>(sm_count) * 8 : gv::kProfileMaxCtas;
-    if (grid > cap) grid = cap;
-    if (grid == 0) grid = 1;
-    GV_CUDA(cudaMemsetAsync(out, 0, sizeof(gv_profile), st));
-    if (row_len > 0 && n_elems > 0)
-        GV_CUDA(cudaMemsetAsync(row_mismatch, 0, sizeof(uint32_t) * ((n_elems + row_len - 1) / row_len), st));
+    const uint64_t want = (tiles + gv::kProfileWarps - 1) / gv::kProfileWarps;
     switch (dt) {
-        case GV_F32: return launch_profile<GV_F32>(p, static_cast<unsigned>(grid), st);
-        case GV_BF16: return launch_profile<GV_BF16>(p, static_cast<unsigned>(grid), st);
-        case GV_F16: return launch_profile<GV_F16>(p, static_cast<unsigned>(grid), st);
-        case GV_I32: return launch_profile<GV_I32>(p, static_cast<unsigned>(grid), st);
-        default: return launch_profile<GV_I64>(p, static_cast<unsigned>(grid), st);
+        case GV_F32: return launch_profile<GV_F32>(p, want, sm_count, st);
+        case GV_BF16: return launch_profile<GV_BF16>(p, want, sm_count, st);
+        case GV_F16: return launch_profile<GV_F16>(p, want, sm_count, st);
+        case GV_I32: return launch_profile<GV_I32>(p, want, sm_count, st);
+        default: return launch_profile<GV_I64>(p, want, sm_count, st);
     }
 }
 

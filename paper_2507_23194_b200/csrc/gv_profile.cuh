@@ -5,10 +5,12 @@
 // candidate and reference in units of the dtype's own spacing, the mismatching element with the
 // largest error, the first eight mismatching elements and, optionally, mismatch counts per row.
 // It runs on demand over the few candidates that failed, as a pass of its own, so the verifier's
-// hot loop carries none of it. One streaming pass (every byte read once, 128-bit loads) plus a
-// one-CTA finalisation over per-CTA / per-warp partials; all results are exact integers or bit
-// patterns and do not depend on scheduling.
+// hot loop carries none of it. One cooperative launch: the grid clears the outputs, synchronises,
+// streams both tensors once (every byte read once, 128-bit loads) into per-warp / per-CTA partials,
+// synchronises again, and its first CTA finalises; all results are exact integers or bit patterns
+// and do not depend on scheduling.
 #pragma once
+#include <cooperative_groups.h>
 #include <stdint.h>
 
 #include "gv.h"
@@ -99,9 +101,27 @@ __device__ __forceinline__ bool profile_better(uint64_t ka, uint64_t ia, uint64_
 }
 
 template <int DT>
+__device__ __forceinline__ void profile_finalize(const ProfileParams& p, unsigned int n_ctas);
+
+// Launched cooperatively (all CTAs resident), because the outputs the grid accumulates into with atomics
+// are cleared by the grid itself first, and the finalisation needs every CTA's partials.
+template <int DT>
 __global__ void __launch_bounds__(kProfileThreads) profile_kernel(ProfileParams p) {
     constexpr int ESZ = Traits<DT>::ESZ;
     constexpr int EPV = 16 / ESZ;
+    cooperative_groups::grid_group grid = cooperative_groups::this_grid();
+    {
+        // clear what the atomics below add to: the whole output record and, if asked for, the row counts
+        const uint64_t gtid = blockIdx.x * static_cast<uint64_t>(kProfileThreads) + threadIdx.x;
+        const uint64_t gsize = static_cast<uint64_t>(gridDim.x) * kProfileThreads;
+        unsigned long long* o = reinterpret_cast<unsigned long long*>(p.out);
+        for (uint64_t i = gtid; i < sizeof(gv_profile) / 8; i += gsize) o[i] = 0ull;
+        if (p.row_len) {
+            const uint64_t n_rows = (p.n + p.row_len - 1) / p.row_len;
+            for (uint64_t i = gtid; i < n_rows; i += gsize) p.rows[i] = 0u;
+        }
+    }
+    grid.sync();
     __shared__ unsigned int s_hist[kProfileWarps][GV_PROFILE_BUCKETS];     // one per warp: fewer same-address collisions
     __shared__ unsigned long long s_first[kProfileWarps][GV_PROFILE_LIST];
     __shared__ ProfileWorst s_worst[kProfileWarps];
@@ -254,12 +274,14 @@ __global__ void __launch_bounds__(kProfileThreads) profile_kernel(ProfileParams 
             have_last = true;
         }
     }
+    grid.sync();
+    if (blockIdx.x == 0) profile_finalize<DT>(p, gridDim.x);
 }
 
 // One CTA: the worst element over the per-CTA partials, the eight smallest indices over the
 // per-CTA lists (eight rounds of a block-wide minimum above the previous pick), and their raw values.
 template <int DT>
-__global__ void __launch_bounds__(kProfileThreads) profile_finalize_kernel(ProfileParams p, unsigned int n_ctas) {
+__device__ __forceinline__ void profile_finalize(const ProfileParams& p, unsigned int n_ctas) {
     constexpr int ESZ = Traits<DT>::ESZ;
     __shared__ ProfileWorst s_w[kProfileWarps];
     __shared__ unsigned long long s_min[kProfileWarps];

@@ -122,8 +122,13 @@ gv_status gv_verify_batch(const void* ref, const void* const* cands, int32_t N, 
  *   results    device, T*N records, tensor-major; first_mismatch is relative to the tensor.
  *   workspace  device, >= gv_workspace_bytes(T, N) bytes, 16-byte aligned.
  * Offsets must be multiples of the tensor's element size. The tables live on the device and are
- * checked there: a bad entry (negative size, misaligned offset, unknown dtype) makes that tensor's
- * records stay zero records and sets GV_ERR_BAD_TABLE in the status word read by gv_check(). */
+ * checked there: a bad entry (negative or absurd size, misaligned offset, unknown dtype) makes that
+ * tensor's records stay zero records and sets GV_ERR_BAD_TABLE in the status word read by gv_check().
+ * The library cannot check offsets against the buffers' sizes (they are not arguments): a table that
+ * points outside ref_base / cand_base is the caller's error.
+ * Enqueues three kernels (record initialisation, table pre-pass, verify). Tensors whose bases are 16-byte
+ * aligned are streamed at full speed; unaligned ones, the last partial tile of each tensor and tensors of
+ * 32 GiB or more take a slower path with the same results (such giants belong in gv_verify_batch). */
 gv_status gv_verify_ragged(const void* ref_base, const int64_t* ref_off, const void* cand_base,
                            const int64_t* cand_off, const uint8_t* dtypes, const int64_t* n_elems,
                            int64_t T, int32_t N, const gv_tol* tol, gv_result* results,

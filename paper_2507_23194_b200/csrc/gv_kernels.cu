@@ -1014,6 +1014,33 @@ __device__ __forceinline__ bool vec_has_nan(int dt, const uint4& r) {
     return any;
 }
 
+// The streaming loops' version of that test: is any element of the reference vector a NaN OR an infinity?
+// (Also sending identical vectors that hold an infinity to the compare path is harmless -- the rule finds
+// them equal -- and lets the test run on the multiply-add pipe, which these loops leave idle, instead of the
+// logic pipe, which they saturate: x * 0 is a zero for every finite x and a NaN otherwise.)
+__device__ __forceinline__ bool vec_has_nonfinite(int dt, const uint4& r) {
+    if (dt == GV_F32) {
+        float a = __fmul_rn(__uint_as_float(r.x), 0.0f);
+        a = __fmaf_rn(__uint_as_float(r.y), 0.0f, a);
+        a = __fmaf_rn(__uint_as_float(r.z), 0.0f, a);
+        a = __fmaf_rn(__uint_as_float(r.w), 0.0f, a);
+        return a != a;
+    }
+    uint32_t a = 0u;
+    if (dt == GV_F16) {
+        asm("{ .reg .b32 z;\n\t mov.b32 z, 0;\n\t"
+            "fma.rn.f16x2 %0, %1, z, z;\n\t fma.rn.f16x2 %0, %2, z, %0;\n\t"
+            "fma.rn.f16x2 %0, %3, z, %0;\n\t fma.rn.f16x2 %0, %4, z, %0; }"
+            : "=&r"(a) : "r"(r.x), "r"(r.y), "r"(r.z), "r"(r.w));
+    } else if (dt == GV_BF16) {
+        asm("{ .reg .b32 z;\n\t mov.b32 z, 0;\n\t"
+            "fma.rn.bf16x2 %0, %1, z, z;\n\t fma.rn.bf16x2 %0, %2, z, %0;\n\t"
+            "fma.rn.bf16x2 %0, %3, z, %0;\n\t fma.rn.bf16x2 %0, %4, z, %0; }"
+            : "=&r"(a) : "r"(r.x), "r"(r.y), "r"(r.z), "r"(r.w));
+    }
+    return (a & 0x7FFF7FFFu) != 0u;       // each half is a zero of either sign, or a NaN
+}
+
 // Tiles [tile_begin, tile_end) with synchronous element-sized loads: the tail tile of a tensor, or every
 // tile of a tensor whose bases are not 16-byte aligned. Returns the sum of the reference's hash terms
 // over the full vectors it met (the caller adds it to every candidate's slot).
@@ -1137,16 +1164,16 @@ __device__ __forceinline__ void ragged_stretch(const RaggedParams& p, int dt, co
                 for (int u = 0; u < 4; ++u) c[u] = lds128(ring_base + (half * 4u + u) * 512u);
                 issue_tile(tile + 2, half);                           // refill the stages just read
                 half ^= 1u;
-                const bool force = nan_matters && vec_has_nan(dt, r);
+                const bool force = nan_matters && vec_has_nonfinite(dt, r);
                 const uint64_t h_ref = hash_vec_full_k32(r, static_cast<uint32_t>(voff / 8));
                 ref_sum += h_ref;
-                uint32_t diffmask = force ? 0xFu : 0u;
+                // one test for the common case (all four candidate vectors identical to the reference vector)
+                uint32_t any_diff = 0u;
 #pragma unroll
-                for (int u = 0; u < 4; ++u)
-                    diffmask |= ((c[u].x != r.x) || (c[u].y != r.y) || (c[u].z != r.z) || (c[u].w != r.w)) ? (1u << u) : 0u;
-                if (__any_sync(0xFFFFFFFFu, diffmask != 0u)) {
+                for (int u = 0; u < 4; ++u) any_diff |= (c[u].x ^ r.x) | (c[u].y ^ r.y) | (c[u].z ^ r.z) | (c[u].w ^ r.w);
+                if (__any_sync(0xFFFFFFFFu, any_diff != 0u || force)) {
 #pragma unroll
-                    for (int u = 0; u < 4; ++u) queued_visit(c[u], r, h_ref, (diffmask >> u) & 1u, voff, u);
+                    for (int u = 0; u < 4; ++u) queued_visit(c[u], r, h_ref, force, voff, u);
                 }
             }
         } else {
@@ -1177,7 +1204,7 @@ __device__ __forceinline__ void ragged_stretch(const RaggedParams& p, int dt, co
                 const uint4 r = lds128(at);
                 stage = (stage + 1u) & (kRing - 1);
                 issue_one(at);
-                const bool force = nan_matters && vec_has_nan(dt, r);
+                const bool force = nan_matters && vec_has_nonfinite(dt, r);
                 const uint64_t h_ref = hash_vec_full_k32(r, static_cast<uint32_t>(voff / 8));
                 ref_sum += h_ref;
 #pragma unroll 1

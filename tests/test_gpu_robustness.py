@@ -141,3 +141,74 @@ def test_read_sum_probe_sums_the_words():
         d = torch.from_numpy(a.view(np.int32)).to(DEV)
         out = gv.gv_selftest_read_sum(d)
         assert int(out.cpu().numpy().view(np.uint64)[0]) == int(a.sum(dtype=np.uint64))
+
+
+@pytest.mark.parametrize("equal_nan", [False, True])
+def test_ragged_four_candidates_with_nan_and_inf_in_the_references(oracle, equal_nan):
+    """The four-candidate instance of the ragged kernel on references that hold NaNs and infinities: candidate
+    vectors identical to such a reference vector must still go through the rule (NaN is not close to NaN
+    unless equal_nan), vectors identical to one holding an infinity may, and both must give the oracle's
+    records. Large tensors (many streamed tiles per warp), all three float dtypes, plus an integer one."""
+    g = torch.Generator().manual_seed(4242)
+    tdt = {0: torch.float32, 1: torch.bfloat16, 2: torch.float16, 3: torch.int32}
+    esz = {0: 4, 1: 2, 2: 2, 3: 4}
+    codes = [0, 1, 2, 3, 2, 0]
+    sizes = [(1 << 19) + 13, (1 << 20) + 8, 777777, 1 << 18, 4096, 33]
+    N = 4
+    refs, cands = [], []
+    for code, n in zip(codes, sizes):
+        if code == 3:
+            r = torch.randint(-1000, 1000, (n,), generator=g, dtype=torch.int32)
+        else:
+            r = torch.randn(n, generator=g).to(tdt[code])
+            where = torch.randint(0, n, (40,), generator=g)
+            r[where[:15]] = float("nan")
+            r[where[15:28]] = float("inf")
+            r[where[28:]] = float("-inf")
+        refs.append(r)
+        cands.append(r.clone())                                          # identical, NaNs and infinities included
+        c = r.clone()
+        idx = torch.randint(0, n, (max(1, n // 100),), generator=g)
+        c[idx] = (c[idx].float() + 1.0).to(tdt[code]) if code != 3 else c[idx] + 1
+        cands.append(c)                                                  # about 1 % changed
+        if code == 3:
+            cands.append(r + 1)
+        else:
+            cands.append((r.float() * 1.0001).to(tdt[code]))             # differs (almost) everywhere, within tolerance
+        c = r.clone()
+        if code != 3:
+            c[torch.isnan(r)] = 0.0                                      # NaN on one side only
+            c[torch.isinf(r)] = -c[torch.isinf(r)]                       # the other infinity
+        cands.append(c)
+    ref_off, cand_off, rc, cc = [], [], 0, 0
+    for t, (code, n) in enumerate(zip(codes, sizes)):
+        rc = (rc + 15) // 16 * 16
+        ref_off.append(rc)
+        rc += n * esz[code]
+        for j in range(N):
+            cc = (cc + 15) // 16 * 16
+            cand_off.append(cc)
+            cc += n * esz[code]
+    ref_off.append(rc)
+    ref_buf = torch.zeros(rc, dtype=torch.uint8)
+    cand_buf = torch.zeros(cc, dtype=torch.uint8)
+    for t, (code, n) in enumerate(zip(codes, sizes)):
+        nb = n * esz[code]
+        ref_buf[ref_off[t]:ref_off[t] + nb] = refs[t].view(torch.uint8)
+        for j in range(N):
+            o = cand_off[t * N + j]
+            cand_buf[o:o + nb] = cands[t * N + j].view(torch.uint8)
+    ro, co = torch.tensor(ref_off), torch.tensor(cand_off)
+    dts, ne = torch.tensor(codes, dtype=torch.uint8), torch.tensor(sizes)
+    ws = torch.empty(gv.gv_workspace_bytes(len(codes), N), dtype=torch.uint8, device=DEV)
+    res = gv.gv_verify_ragged(ref_buf.to(DEV), ro.to(DEV), cand_buf.to(DEV), co.to(DEV), dts.to(DEV), N, 1e-2, 1e-2,
+                              equal_nan, n_elems=ne.to(DEV), workspace=ws)
+    torch.cuda.synchronize()
+    assert gv.gv_check(ws) == gv.GV_OK
+    want = oracle.verify_ragged(ref_buf.numpy(), ro.numpy(), cand_buf.numpy(), co.numpy(), dts.numpy(), N, 1e-2, 1e-2,
+                                equal_nan, n_elems=ne.numpy())
+    got = gv.results_to_numpy(res)
+    for i in range(len(got)):
+        assert got[i].tobytes() == want[i].tobytes(), (i, got[i], want[i])
+    n_nan = int(torch.isnan(refs[0]).sum())
+    assert int(got[0]["n_mismatch"]) == (0 if equal_nan else n_nan)      # fp32 tensor, exact copy: only its NaNs can mismatch

@@ -59,11 +59,11 @@ def _scaled(measured, ref_bytes, cap_cands, full_cands, cap_chunks=None, full_ch
 
 
 NCU_TRAFFIC_BYTES = {
-    "cfg2": _scaled(2.181e9 + 4.3e6, 33554432, 64, 256, cap_chunks=1, full_chunks=1),   # profiles/dense_kernel_bf16_cfg2.md (reference stays in L2)
-    "cfg3": _scaled(5.100e9 + 4.1e6, 268435456, 16, 32, cap_chunks=3, full_chunks=2),   # profiles/dense_kernel_f16_cfg3.md
-    "cfg4": _scaled(4.564e9 + 5.1e6, 268435456, 16, 64),      # profiles/dense_kernel_i32_cfg4.md
-    "cfg4w": 2 * _scaled(4.564e9 + 5.1e6, 268435456, 16, 64),  # the int64 variant moves twice the bytes of the same shape through the same kernel (scaled from the int32 capture, not captured itself)
-    "cfg5": (2.292e9 + 11.1e6) * 10000 / 2000,                # profiles/ragged_kernel_cfg5.md (2000 of 10000 tensors)
+    "cfg2": _scaled(2.181e9 + 4.0e6, 33554432, 64, 256, cap_chunks=1, full_chunks=1),   # profiles/dense_kernel_bf16_cfg2.md (reference stays in L2)
+    "cfg3": _scaled(5.100e9 + 3.7e6, 268435456, 16, 32, cap_chunks=3, full_chunks=2),   # profiles/dense_kernel_f16_cfg3.md
+    "cfg4": _scaled(4.564e9 + 4.5e6, 268435456, 16, 64),      # profiles/dense_kernel_i32_cfg4.md
+    "cfg4w": _scaled(4.832e9 + 3.8e6, 536870912, 8, 64, cap_chunks=1, full_chunks=4),   # profiles/dense_kernel_i64_cfg4w.md
+    "cfg5": (2.331e9 + 41.6e6) * 10000 / 2000,                # profiles/ragged_kernel_cfg5.md (2000 of 10000 tensors)
 }
 
 
@@ -540,9 +540,10 @@ def main():
     achieved = algo_bytes / (ms_per_step * 1e-3) / 1e9
     first = step_ms[:20]
     roofline = {"bound": "hbm",
-                "co_bound": "alu: vectors identical to the reference stream at HBM rate; vectors that differ pay the integer work "
-                            "of the content hash (7.3 TB/s for the hash alone) and the compare (profiles/instruction_rates_b200.md, "
-                            "profiles/compare_ceiling_b200.md)",
+                "co_bound": {"kind": "alu", "peak_GB/s": {"f16": 5430.0, "bf16": 5640.0, "f32": 5800.0},
+                             "what": "vectors identical to the reference stream at HBM rate; vectors that differ pay two splitmix64 "
+                                     "evaluations and an fp32 compare per 16 bytes, whose arithmetic alone (registers only, 16 warps "
+                                     "per SM) sustains these rates: profiles/compare_ceiling_b200.md"},
                 "kernel": "ragged_kernel" if ragged else "dense_kernel",
                 "achieved": achieved, "peak": peak, "peak_kind": peak_kind + " (STREAM-style copy)",
                 "unit": "GB/s", "frac": achieved / peak, "traffic": NCU_TRAFFIC_BYTES.get(args.workload),
@@ -595,6 +596,9 @@ def main():
             per_class[cls] = r
         line["per_class"] = per_class
 
+        # ---- the content hash as a call of its own (every byte hashed: arithmetic-bound, not a copy) ----
+        line["hash"] = bench_hash(gv, stream, device, peak)
+
         # ---- follow-on stages on the headline's records (outside the timed step) ----
         line["grouping"] = bench_grouping(gv, runner, stream, device, not args.no_cpu_baseline)
         line["error_profile"] = bench_error_profile(gv, wl, stream, device, peak)
@@ -618,6 +622,25 @@ def main():
     print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()
+
+
+def bench_hash(gv, stream, device, peak):
+    out = {}
+    buf = torch.empty((2 << 30) // 8, dtype=torch.int64, device=device)
+    buf.random_()
+    h = torch.empty(1, dtype=torch.int64, device=device)
+    for label, n_words in (("256MiB", (256 << 20) // 8), ("2GiB", (2 << 30) // 8)):
+        view = buf[:n_words]
+        for name, fn in (("gv_hash", gv.gv_hash), ("gv_hash2", gv.gv_hash2)):
+            for _ in range(3):
+                fn(view, h)
+            ms, _ = timed_steps(lambda: fn(view, h), 10, stream)
+            gbs = n_words * 8 / (statistics.median(ms) * 1e-3) / 1e9
+            out[f"{name}_{label}"] = {"GB/s": gbs, "frac_of_measured_hbm": gbs / peak}
+    out["note"] = ("two splitmix64 evaluations per 16 bytes on every byte; the 256 MiB buffer is not much larger than L2 and a call "
+                   "is a memset plus one launch")
+    del buf
+    return out
 
 
 def bench_grouping(gv, runner, stream, device, with_oracle: bool):

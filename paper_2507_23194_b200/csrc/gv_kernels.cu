@@ -836,7 +836,9 @@ struct RaggedParams {
 
 constexpr int kRaggedTile = kWarpTile;      // ragged work is split into the same 512-byte warp-tiles
 constexpr int64_t kRaggedMaxBytes = int64_t(1) << 40;   // largest tensor a table entry may describe (1 TiB)
-constexpr uint64_t kChunkBig = 256;                     // most tiles a warp takes at a time from the global tile sequence
+constexpr uint64_t kChunkBig = 256;                     // most work units a warp takes at a time from the global sequence
+constexpr int64_t kPartCost = 4;                        // work units charged per tensor on top of its tiles (pointer set-up, tail tile,
+                                                        // publishing the records: about what four streamed tiles cost)
 
 // Pre-pass: validates the tables and turns sizes into an exclusive prefix of tile counts.
 // One CTA; T is at most a few million in practice (one pass of 1024-wide chunks).
@@ -872,6 +874,9 @@ __global__ void __launch_bounds__(1024) ragged_prepass_kernel(RaggedParams p) {
             }
             if (!good) atomicOr(p.status, kStatusBadTable);
             else tiles = (n * esz + kRaggedTile - 1) / kRaggedTile;
+            // the table holds WORK units, not tiles: a tensor costs its tiles plus a fixed amount for
+            // starting and finishing it (empty and rejected tensors cost nothing and are skipped)
+            if (tiles > 0) tiles += kPartCost;
         }
         // inclusive scan of `tiles` over the 1024 threads
         long long x = tiles;
@@ -914,75 +919,93 @@ struct RaggedSmem {
     static constexpr size_t kPtrOff = kAccOff + size_t(kWarps) * kChunk * sizeof(CtaAcc);  // [warp][kChunk + 2] reference + candidate pointers
     static constexpr size_t kQueueOff = kPtrOff + size_t(kWarps) * (kChunk + 2) * 8;       // [warp][3][kQCap] uint4
     static constexpr size_t kRefOff = kQueueOff + size_t(kWarps) * kQueueBytes;            // [warp][2][32] uint4 (four-candidate loop)
-    static constexpr size_t kTotal = kRefOff + size_t(kWarps) * 2 * kWarpTile;
+    static constexpr size_t kMetaOff = kRefOff + size_t(kWarps) * 2 * kWarpTile;            // [warp][32] u64: table entries of the current tensor
+    static constexpr size_t kTotal = kMetaOff + size_t(kWarps) * 32 * 8;
 };
 
-// A full candidate vector that differs from its reference vector, any dtype. Out of line and
-// switched on the dtype at run time so that the ragged hot loop exists once, not once per dtype
-// (mixed-dtype batches would otherwise thrash the instruction cache). The derived reference values
-// are computed per call here: a ragged tile has only a handful of candidates to amortise them over.
+// Code size matters in this kernel: the warps of an SM are in different places at the same time (the
+// streaming loop, the batch function of one of four dtypes, a tensor's tail), and everything they run
+// competes for the instruction cache (ncu: waiting for instructions was the second largest stall; every
+// variant that added code to any of these paths lost throughput). So the paths beside the streaming loops
+// are written for size: rolled loops and run-time dtype tests instead of one unrolled body per dtype.
+
+// The warp's queue of differing vectors (all of one tensor, hence of one dtype): the n oldest entries, one
+// per lane. The hash uses 64-bit word indices (tensors of any size reach this function through the tail path).
 template <int DT>
-__device__ __forceinline__ void ragged_differing_t(const uint4& c, const uint4& r, uint64_t elem0, const TolF& tol,
-                                                   CtaAcc* s) {
+__device__ __forceinline__ void ragged_entry(const uint4& c, const uint4& r, uint64_t voff, const TolF& tol, CtaAcc* s) {
+    constexpr int ESZ = Traits<DT>::ESZ;
     if constexpr (Traits<DT>::IS_FLOAT) {
-        RefVec<16 / Traits<DT>::ESZ> rv;
-        uint32_t flags;
-        hoist_ref<DT>(r, tol, rv, flags);
-        uint32_t lane_cnt = 0u;
-        if (!vec_fast_float<DT>(c, rv, flags, tol, s, elem0, lane_cnt)) {
-            Acc a;
-            a.clear();
-            const uint32_t thr = *reinterpret_cast<volatile unsigned int*>(&s->thr);
-            vec_exact_float<DT>(c, rv, elem0, tol, thr, a);
-            push_rare(s, a);
-            lane_cnt += a.cnt;
-            raise_maxabs(s, a.maxabs);
-        }
-        // (called from diverged code: one shared atomic per lane that found mismatches)
-        if (lane_cnt) atomicAdd(&s->cnt, static_cast<unsigned long long>(lane_cnt));
+        RefVec<16 / ESZ> rv;
+        uint32_t rflags = 0u, unused = 0u;
+        hoist_ref<DT>(r, tol, rv, rflags);
+        if (!vec_fast_float<DT, true>(c, rv, rflags, tol, s, voff / ESZ, unused)) settle_vector_exact<DT>(c, rv, voff / ESZ, tol, s);
     } else {
         Acc a;
         a.clear();
-        vec_int<DT>(c, r, elem0, 16 / Traits<DT>::ESZ, a);
+        vec_int<DT>(c, r, voff / ESZ, 16 / ESZ, a);
         push_rare(s, a);
         if (a.cnt) atomicAdd(&s->cnt, static_cast<unsigned long long>(a.cnt));
     }
 }
-// (out of line, arguments by value: by-reference arguments would live in local memory)
-__device__ __noinline__ void ragged_differing(int dt, uint4 c, uint4 r, uint64_t byte_off, TolF tol, CtaAcc* s) {
-    switch (dt) {
-        case GV_F32: ragged_differing_t<GV_F32>(c, r, byte_off / 4, tol, s); break;
-        case GV_BF16: ragged_differing_t<GV_BF16>(c, r, byte_off / 2, tol, s); break;
-        case GV_F16: ragged_differing_t<GV_F16>(c, r, byte_off / 2, tol, s); break;
-        case GV_I32: ragged_differing_t<GV_I32>(c, r, byte_off / 4, tol, s); break;
-        default: ragged_differing_t<GV_I64>(c, r, byte_off / 8, tol, s); break;
-    }
-}
-// The warp's queue of differing vectors (all of one tensor, hence of one dtype): the n oldest entries.
-// (Streamed tiles only, hence tensors below 32 GiB: 32-bit word indices.)
 __device__ __noinline__ void ragged_batch(int dt, uint32_t qbase, uint32_t head, uint32_t n, uint2* slots, CtaAcc* wacc,
                                           TolF tol) {
+    const uint32_t lane = threadIdx.x & 31u;
+    if (lane >= n) return;
+    const uint32_t at = qbase + ((head + lane) & (kQCap - 1)) * 16u;
+    const uint4 c = lds128(at);
+    const uint4 r = lds128(at + kQPlane);
+    const uint4 m = lds128(at + 2 * kQPlane);
+    const uint64_t meta = pack64(m.x, m.y), h_ref = pack64(m.z, m.w);
+    const int k = static_cast<int>(m.x & 15u);
+    const uint64_t voff = meta & ~uint64_t(15);
+    const uint64_t h = hash_vec_full(c, voff / 8);
+    const uint2 sl = slots[k * 32];
+    const uint64_t hs = pack64(sl.x, sl.y) + (h - h_ref);
+    slots[k * 32] = make_uint2(static_cast<uint32_t>(hs), static_cast<uint32_t>(hs >> 32));
+    CtaAcc* s = &wacc[k];
     switch (dt) {
-        case GV_F32: batch_entries<GV_F32, false>(qbase, head, n, slots, wacc, tol); break;
-        case GV_BF16: batch_entries<GV_BF16, false>(qbase, head, n, slots, wacc, tol); break;
-        case GV_F16: batch_entries<GV_F16, false>(qbase, head, n, slots, wacc, tol); break;
-        case GV_I32: batch_entries<GV_I32, false>(qbase, head, n, slots, wacc, tol); break;
-        default: batch_entries<GV_I64, false>(qbase, head, n, slots, wacc, tol); break;
+        case GV_F32: ragged_entry<GV_F32>(c, r, voff, tol, s); break;
+        case GV_BF16: ragged_entry<GV_BF16>(c, r, voff, tol, s); break;
+        case GV_F16: ragged_entry<GV_F16>(c, r, voff, tol, s); break;
+        case GV_I32: ragged_entry<GV_I32>(c, r, voff, tol, s); break;
+        default: ragged_entry<GV_I64>(c, r, voff, tol, s); break;
     }
 }
-// The partial vector at the end of a tensor: element by element through the general rule.
-__device__ __noinline__ void ragged_partial(int dt, uint4 c, uint4 r, uint64_t byte_off, int nvalid, TolF tol,
-                                            CtaAcc* s, uint2* slot) {
+
+// Element e of a 16-byte vector of dtype dt, zero-extended raw bits (dynamic indexing: cold code).
+__device__ __forceinline__ uint64_t raw_element(const uint4& v, int esz, int e) {
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+    if (esz == 2) return (w[e >> 1] >> (16 * (e & 1))) & 0xFFFFu;
+    if (esz == 4) return w[e];
+    return pack64(w[2 * e], w[2 * e + 1]);
+}
+// A vector that is not complete (the end of a tensor): its nvalid elements one by one through the general
+// rule, in one rolled loop for all dtypes; its hash terms go to the slot as they are (no shared terms here).
+__device__ __noinline__ void ragged_elements(int dt, uint4 c, uint4 r, uint64_t byte_off, int nvalid, TolF tol, CtaAcc* s,
+                                             uint2* slot) {
     Acc a;
     a.clear();
     const int esz = elem_size(dt);
     a.hash = hash_vec(c, byte_off / 8, nvalid * esz > 8 ? 2 : 1);
-    switch (dt) {
-        case GV_F32: vec_compare<GV_F32>(c, r, byte_off / 4, nvalid, tol, a); break;
-        case GV_BF16: vec_compare<GV_BF16>(c, r, byte_off / 2, nvalid, tol, a); break;
-        case GV_F16: vec_compare<GV_F16>(c, r, byte_off / 2, nvalid, tol, a); break;
-        case GV_I32: vec_compare<GV_I32>(c, r, byte_off / 4, nvalid, tol, a); break;
-        default: vec_compare<GV_I64>(c, r, byte_off / 8, nvalid, tol, a); break;
+    const uint64_t elem0 = byte_off / static_cast<uint64_t>(esz);
+#pragma unroll 1
+    for (int e = 0; e < nvalid; ++e) {
+        const uint64_t cr = raw_element(c, esz, e), rr = raw_element(r, esz, e);
+        if (dt <= GV_F16) {
+            float cf, rf;
+            if (dt == GV_F32) { cf = __uint_as_float(static_cast<uint32_t>(cr)); rf = __uint_as_float(static_cast<uint32_t>(rr)); }
+            else if (dt == GV_BF16) { cf = __uint_as_float(static_cast<uint32_t>(cr) << 16); rf = __uint_as_float(static_cast<uint32_t>(rr) << 16); }
+            else { cf = f16_to_f32(static_cast<uint32_t>(cr)); rf = f16_to_f32(static_cast<uint32_t>(rr)); }
+            element_rule<false>(cf, rf, tol, elem0 + e, a);
+        } else if (cr != rr) {
+            const int64_t cv = dt == GV_I32 ? static_cast<int64_t>(static_cast<int32_t>(cr)) : static_cast<int64_t>(cr);
+            const int64_t rv = dt == GV_I32 ? static_cast<int64_t>(static_cast<int32_t>(rr)) : static_cast<int64_t>(rr);
+            const uint64_t diff = cv > rv ? static_cast<uint64_t>(cv) - static_cast<uint64_t>(rv)
+                                          : static_cast<uint64_t>(rv) - static_cast<uint64_t>(cv);      // exact mod 2^64
+            a.cnt += 1;
+            a.first = (elem0 + e) < a.first ? (elem0 + e) : a.first;
+            a.maxint = diff > a.maxint ? diff : a.maxint;
+        }
     }
     const uint2 sl = *slot;
     const uint64_t h = pack64(sl.x, sl.y) + a.hash;
@@ -991,10 +1014,29 @@ __device__ __noinline__ void ragged_partial(int dt, uint4 c, uint4 r, uint64_t b
     if (a.cnt) atomicAdd(&s->cnt, static_cast<unsigned long long>(a.cnt));
     raise_maxabs(s, a.maxabs);
 }
+// A 16-byte vector at byte_off of a tensor of nbytes bytes: one 128-bit load when it is complete and
+// aligned, else the elements that exist one by one (rolled), zero fill for the rest.
+__device__ __noinline__ uint4 load_vec_slow(int esz, const unsigned char* base, uint64_t byte_off, uint64_t nbytes) {
+    uint32_t w[4] = {0u, 0u, 0u, 0u};
+#pragma unroll 1
+    for (int b = 0; b < 16; b += esz) {
+        const uint64_t o = byte_off + b;
+        if (o < nbytes) {
+            if (esz == 2) w[b >> 2] |= static_cast<uint32_t>(*reinterpret_cast<const unsigned short*>(base + o)) << (8 * (b & 3));
+            else if (esz == 4) w[b >> 2] = *reinterpret_cast<const uint32_t*>(base + o);
+            else {
+                const uint64_t x = *reinterpret_cast<const unsigned long long*>(base + o);
+                w[b >> 2] = static_cast<uint32_t>(x);
+                w[(b >> 2) + 1] = static_cast<uint32_t>(x >> 32);
+            }
+        }
+    }
+    return make_uint4(w[0], w[1], w[2], w[3]);
+}
 __device__ __forceinline__ uint4 load_vec_any(int esz, const unsigned char* base, uint64_t byte_off, uint64_t nbytes) {
-    if (esz == 2) return load_vec_generic<2>(base, byte_off, nbytes);
-    if (esz == 4) return load_vec_generic<4>(base, byte_off, nbytes);
-    return load_vec_generic<8>(base, byte_off, nbytes);
+    if (byte_off + 16 <= nbytes && ((reinterpret_cast<uintptr_t>(base) + byte_off) & 15u) == 0)
+        return *reinterpret_cast<const uint4*>(base + byte_off);
+    return load_vec_slow(esz, base, byte_off, nbytes);
 }
 // NaN anywhere in a reference vector of a float dtype (bit tests only)
 __device__ __forceinline__ bool vec_has_nan(int dt, const uint4& r) {
@@ -1013,7 +1055,6 @@ __device__ __forceinline__ bool vec_has_nan(int dt, const uint4& r) {
     }
     return any;
 }
-
 // The streaming loops' version of that test: is any element of the reference vector a NaN OR an infinity?
 // (Also sending identical vectors that hold an infinity to the compare path is harmless -- the rule finds
 // them equal -- and lets the test run on the multiply-add pipe, which these loops leave idle, instead of the
@@ -1041,23 +1082,28 @@ __device__ __forceinline__ bool vec_has_nonfinite(int dt, const uint4& r) {
     return (a & 0x7FFF7FFFu) != 0u;       // each half is a zero of either sign, or a NaN
 }
 
-// Tiles [tile_begin, tile_end) with synchronous element-sized loads: the tail tile of a tensor, or every
-// tile of a tensor whose bases are not 16-byte aligned. Returns the sum of the reference's hash terms
-// over the full vectors it met (the caller adds it to every candidate's slot).
+// Tiles [tile_begin, tile_end) with synchronous loads: the tail tile of a tensor, or every tile of a tensor
+// that is not streamed (a base that is not 16-byte aligned, 32 GiB or more). Complete vectors that differ
+// from the reference vector go through the warp's queue like those of streamed tiles (same batch function,
+// nothing of their own); the one incomplete vector at the end of a tensor goes element by element.
+// Returns the sum of the reference's hash terms over the complete vectors it met (the caller adds it to
+// every candidate's slot).
 __device__ __noinline__ uint64_t ragged_tail(int dt, const unsigned char* ref, uint64_t nbytes, uint64_t tile_begin,
                                              uint64_t tile_end, int kg, uint2* slots, CtaAcc* wacc,
-                                             const unsigned char* const* wptr, TolF tol, bool nan_matters) {
+                                             const unsigned char* const* wptr, TolF tol, bool nan_matters, uint32_t qbase) {
     const int esz = elem_size(dt);
     const int lane = threadIdx.x & 31;
+    const uint32_t lanes_below = (1u << lane) - 1u;
+    uint32_t qhead = 0u, qcount = 0u;
     uint64_t ref_sum = 0;
 #pragma unroll 1
     for (uint64_t tile = tile_begin; tile < tile_end; ++tile) {
         const uint64_t voff = tile * kWarpTile + lane * 16;
         const uint64_t rem = voff < nbytes ? nbytes - voff : 0;
         const int nvalid = rem >= 16 ? 16 / esz : static_cast<int>(rem / esz);
-        if (nvalid <= 0) continue;
         const bool full = rem >= 16;
-        const uint4 r = load_vec_any(esz, ref, voff, nbytes);
+        uint4 r = make_uint4(0u, 0u, 0u, 0u);
+        if (nvalid > 0) r = load_vec_any(esz, ref, voff, nbytes);
         const bool force = nan_matters && full && vec_has_nan(dt, r);
         uint64_t h_ref = 0;
         if (full) {
@@ -1065,21 +1111,39 @@ __device__ __noinline__ uint64_t ragged_tail(int dt, const unsigned char* ref, u
             ref_sum += h_ref;
         }
 #pragma unroll 1
-        for (int k = 0; k < kg; ++k) {
-            const uint4 c = load_vec_any(esz, wptr[k], voff, nbytes);
-            if (full) {
-                const bool differs = (c.x != r.x) || (c.y != r.y) || (c.z != r.z) || (c.w != r.w);
-                if (differs) {
-                    const uint64_t d = hash_vec_full(c, voff / 8) - h_ref;
-                    const uint2 sl = slots[k * 32];
-                    const uint64_t h = pack64(sl.x, sl.y) + d;
-                    slots[k * 32] = make_uint2(static_cast<uint32_t>(h), static_cast<uint32_t>(h >> 32));
+        for (int k0 = 0; k0 < kg; k0 += 4) {
+            // four candidates' loads are issued together (a tiny tensor is nothing but this function: the
+            // loads' latency, not their number, is its cost)
+            uint4 cc[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) cc[u] = (k0 + u < kg && nvalid > 0) ? load_vec_any(esz, wptr[k0 + u], voff, nbytes) : r;
+#pragma unroll 1
+            for (int u = 0; u < 4 && k0 + u < kg; ++u) {
+                const int k = k0 + u;
+                const uint4 c = u == 0 ? cc[0] : u == 1 ? cc[1] : u == 2 ? cc[2] : cc[3];
+                if (nvalid > 0 && !full) ragged_elements(dt, c, r, voff, nvalid, tol, &wacc[k], &slots[k * 32]);
+                const bool want = full && ((c.x != r.x) || (c.y != r.y) || (c.z != r.z) || (c.w != r.w) || force);
+                const uint32_t bal = __ballot_sync(0xFFFFFFFFu, want);
+                if (bal == 0u) continue;
+                const uint32_t at = qbase + ((qhead + qcount + __popc(bal & lanes_below)) & (kQCap - 1)) * 16u;
+                const uint64_t meta = voff | static_cast<uint64_t>(k);
+                sts128x3_if(at, kQPlane, c, r, make_uint4(static_cast<uint32_t>(meta), static_cast<uint32_t>(meta >> 32),
+                                                          static_cast<uint32_t>(h_ref), static_cast<uint32_t>(h_ref >> 32)), want);
+                qcount += __popc(bal);
+                if (qcount >= 32u) {
+                    __syncwarp();
+                    ragged_batch(dt, qbase, qhead, 32u, slots, wacc, tol);
+                    __syncwarp();
+                    qhead = (qhead + 32u) & (kQCap - 1);
+                    qcount -= 32u;
                 }
-                if (differs || force) ragged_differing(dt, c, r, voff, tol, &wacc[k]);
-            } else {
-                ragged_partial(dt, c, r, voff, nvalid, tol, &wacc[k], &slots[k * 32]);
             }
         }
+    }
+    if (qcount) {
+        __syncwarp();
+        ragged_batch(dt, qbase, qhead, qcount, slots, wacc, tol);
+        __syncwarp();
     }
     return ref_sum;
 }
@@ -1094,19 +1158,21 @@ __device__ __noinline__ uint64_t ragged_tail(int dt, const unsigned char* ref, u
 // block of the ring, two tiles in flight; one wait, one vote and one commit per tile, pointers in
 // registers. The other instance takes any number of candidates through one sequence of copies.
 template <bool FOUR>
-__device__ __forceinline__ void ragged_stretch(const RaggedParams& p, int dt, const unsigned char* ref, uint64_t n,
-                                               uint64_t tile_begin, uint64_t tile_end, int kg, uint2* slots,
-                                               CtaAcc* wacc, const unsigned char* const* wsrc, int lane,
-                                               uint32_t ring_base, uint32_t qbase, uint32_t refst_base) {
-    const unsigned char* const* wptr = wsrc + 1;        // wsrc[0] = the reference, wsrc[1 + k] = candidate k
-    const int esz = elem_size(dt);
-    const uint64_t nbytes = n * esz;
+__device__ __noinline__ uint64_t ragged_stream(const RaggedParams& p, int dt, uint64_t tile_begin, uint64_t full_end, int kg,
+                                               unsigned char* smem) {
+    // (The streamed tiles of one tensor part. Out of line and self-contained -- it takes its pointers from the
+    // warp's table in shared memory -- so that its loops get a register allocation that nothing around them,
+    // neither the tail code nor the chunk bookkeeping, can disturb. Returns the sum of the reference's hash
+    // terms over the tiles it met.)
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    uint2* slots = reinterpret_cast<uint2*>(smem + RaggedSmem::kSlotOff) + size_t(warp) * kChunk * 32 + lane;
+    CtaAcc* wacc = reinterpret_cast<CtaAcc*>(smem + RaggedSmem::kAccOff) + warp * kChunk;
+    const unsigned char* const* wsrc = reinterpret_cast<const unsigned char* const*>(smem + RaggedSmem::kPtrOff) + warp * (kChunk + 2);
+    const uint32_t ring_base = smem_u32(smem + RaggedSmem::kRingOff) + (warp * kRing * 32 + lane) * 16;
+    const uint32_t qbase = smem_u32(smem + RaggedSmem::kQueueOff) + warp * static_cast<uint32_t>(kQueueBytes);
+    const uint32_t refst_base = smem_u32(smem + RaggedSmem::kRefOff) + (warp * 2 * 32 + lane) * 16;
     const TolF tol = {p.atol, p.rtol, p.equal_nan};
     const bool nan_matters = (dt <= GV_F16) && !p.equal_nan;
-    bool streamed = (reinterpret_cast<uintptr_t>(ref) & 15u) == 0 && nbytes < (1ull << 35);
-    for (int k = 0; k < kg; ++k) streamed = streamed && (reinterpret_cast<uintptr_t>(wptr[k]) & 15u) == 0;
-    const uint64_t full_end_all = nbytes / kWarpTile;                  // tiles [0, full_end_all) are full
-    const uint64_t full_end = streamed ? (tile_end < full_end_all ? tile_end : full_end_all) : tile_begin;
 
     // As in the dense kernel, a vector identical to the reference vector contributes the reference
     // vector's own hash terms: those are summed once per tile (ref_sum), the slots only collect the
@@ -1136,99 +1202,115 @@ __device__ __forceinline__ void ragged_stretch(const RaggedParams& p, int dt, co
         }
     };
 
-    if (full_end > tile_begin) {
-        if constexpr (FOUR) {
-            const unsigned char* src_r = ref + lane * 16;
-            const unsigned char* src_c[4];
+    if constexpr (FOUR) {
+        const unsigned char* src_r = wsrc[0] + lane * 16;
+        const unsigned char* src_c[4];
 #pragma unroll
-            for (int u = 0; u < 4; ++u) src_c[u] = wptr[u] + lane * 16;
-            auto issue_tile = [&](uint64_t tile, uint32_t half) {     // half: 0 or 1, which half of the ring / reference stage
-                if (tile < full_end) {
-                    const uint64_t off = tile * kWarpTile;
-                    cp_async16(refst_base + half * 512u, src_r + off);
+        for (int u = 0; u < 4; ++u) src_c[u] = wsrc[1 + u] + lane * 16;
+        auto issue_tile = [&](uint64_t tile, uint32_t half) {     // half: 0 or 1, which half of the ring / reference stage
+            if (tile < full_end) {
+                const uint64_t off = tile * kWarpTile;
+                cp_async16(refst_base + half * 512u, src_r + off);
 #pragma unroll
-                    for (int u = 0; u < 4; ++u) cp_async16(ring_base + (half * 4u + u) * 512u, src_c[u] + off);
-                }
-                cp_async_commit();
-            };
-            issue_tile(tile_begin, 0u);
-            issue_tile(tile_begin + 1, 1u);
-            uint32_t half = 0u;
-#pragma unroll 1
-            for (uint64_t tile = tile_begin; tile < full_end; ++tile) {
-                const uint64_t voff = tile * kWarpTile + lane * 16;     // (below 32 GiB: word indices fit 32 bits)
-                cp_async_wait<1>();                                   // this tile's group has landed
-                const uint4 r = lds128(refst_base + half * 512u);
-                uint4 c[4];
-#pragma unroll
-                for (int u = 0; u < 4; ++u) c[u] = lds128(ring_base + (half * 4u + u) * 512u);
-                issue_tile(tile + 2, half);                           // refill the stages just read
-                half ^= 1u;
-                const bool force = nan_matters && vec_has_nonfinite(dt, r);
-                const uint64_t h_ref = hash_vec_full_k32(r, static_cast<uint32_t>(voff / 8));
-                ref_sum += h_ref;
-                // one test for the common case (all four candidate vectors identical to the reference vector)
-                uint32_t any_diff = 0u;
-#pragma unroll
-                for (int u = 0; u < 4; ++u) any_diff |= (c[u].x ^ r.x) | (c[u].y ^ r.y) | (c[u].z ^ r.z) | (c[u].w ^ r.w);
-                if (__any_sync(0xFFFFFFFFu, any_diff != 0u || force)) {
-#pragma unroll
-                    for (int u = 0; u < 4; ++u) queued_visit(c[u], r, h_ref, force, voff, u);
-                }
+                for (int u = 0; u < 4; ++u) cp_async16(ring_base + (half * 4u + u) * 512u, src_c[u] + off);
             }
-        } else {
-            // The copies form one sequence: per tile the reference vector, then the kg candidate vectors.
-            // The stage a visit has just consumed is refilled at once with the copy kRing places ahead,
-            // so consumer and producer share one stage counter. src[0] is the reference, src[1 + k]
-            // candidate k (wsrc, one table per warp in shared memory).
-            const uint64_t end_off = full_end * kWarpTile;
-            uint64_t issue_off = tile_begin * kWarpTile + lane * 16;        // this lane's byte offset of the next copy
-            int issue_j = 0;
-            auto issue_one = [&](uint32_t stage_addr) {
-                if (issue_off < end_off) {
-                    cp_async16(stage_addr, wsrc[issue_j] + issue_off);
-                    const bool wrap = issue_j == kg;
-                    issue_j = wrap ? 0 : issue_j + 1;
-                    issue_off += wrap ? kWarpTile : 0;
-                }
-                cp_async_commit();
-            };
+            cp_async_commit();
+        };
+        issue_tile(tile_begin, 0u);
+        issue_tile(tile_begin + 1, 1u);
+        uint32_t half = 0u;
 #pragma unroll 1
-            for (int j = 0; j < kRing; ++j) issue_one(ring_base + j * 512u);
-            uint32_t stage = 0;
+        for (uint64_t tile = tile_begin; tile < full_end; ++tile) {
+            const uint64_t voff = tile * kWarpTile + lane * 16;     // (below 32 GiB: word indices fit 32 bits)
+            cp_async_wait<1>();                                   // this tile's group has landed
+            const uint4 r = lds128(refst_base + half * 512u);
+            uint4 c[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) c[u] = lds128(ring_base + (half * 4u + u) * 512u);
+            issue_tile(tile + 2, half);                           // refill the stages just read
+            half ^= 1u;
+            const bool force = nan_matters && vec_has_nonfinite(dt, r);
+            const uint64_t h_ref = hash_vec_full_k32(r, static_cast<uint32_t>(voff / 8));
+            ref_sum += h_ref;
+            // one test for the common case (all four candidate vectors identical to the reference vector)
+            uint32_t any_diff = 0u;
+#pragma unroll
+            for (int u = 0; u < 4; ++u) any_diff |= (c[u].x ^ r.x) | (c[u].y ^ r.y) | (c[u].z ^ r.z) | (c[u].w ^ r.w);
+            if (__any_sync(0xFFFFFFFFu, any_diff != 0u || force)) {
+#pragma unroll
+                for (int u = 0; u < 4; ++u) queued_visit(c[u], r, h_ref, force, voff, u);
+            }
+        }
+    } else {
+        // The copies form one sequence: per tile the reference vector, then the kg candidate vectors.
+        // The stage a visit has just consumed is refilled at once with the copy kRing places ahead,
+        // so consumer and producer share one stage counter. src[0] is the reference, src[1 + k]
+        // candidate k (wsrc, one table per warp in shared memory).
+        const uint64_t end_off = full_end * kWarpTile;
+        uint64_t issue_off = tile_begin * kWarpTile + lane * 16;        // this lane's byte offset of the next copy
+        int issue_j = 0;
+        auto issue_one = [&](uint32_t stage_addr) {
+            if (issue_off < end_off) {
+                cp_async16(stage_addr, wsrc[issue_j] + issue_off);
+                const bool wrap = issue_j == kg;
+                issue_j = wrap ? 0 : issue_j + 1;
+                issue_off += wrap ? kWarpTile : 0;
+            }
+            cp_async_commit();
+        };
 #pragma unroll 1
-            for (uint64_t tile = tile_begin; tile < full_end; ++tile) {
-                const uint64_t voff = tile * kWarpTile + lane * 16;
+        for (int j = 0; j < kRing; ++j) issue_one(ring_base + j * 512u);
+        uint32_t stage = 0;
+#pragma unroll 1
+        for (uint64_t tile = tile_begin; tile < full_end; ++tile) {
+            const uint64_t voff = tile * kWarpTile + lane * 16;
+            cp_async_wait<kRing - 1>();
+            uint32_t at = ring_base + stage * 512u;
+            const uint4 r = lds128(at);
+            stage = (stage + 1u) & (kRing - 1);
+            issue_one(at);
+            const bool force = nan_matters && vec_has_nonfinite(dt, r);
+            const uint64_t h_ref = hash_vec_full_k32(r, static_cast<uint32_t>(voff / 8));
+            ref_sum += h_ref;
+#pragma unroll 1
+            for (int k = 0; k < kg; ++k) {
                 cp_async_wait<kRing - 1>();
-                uint32_t at = ring_base + stage * 512u;
-                const uint4 r = lds128(at);
+                at = ring_base + stage * 512u;
+                const uint4 c = lds128(at);
                 stage = (stage + 1u) & (kRing - 1);
                 issue_one(at);
-                const bool force = nan_matters && vec_has_nonfinite(dt, r);
-                const uint64_t h_ref = hash_vec_full_k32(r, static_cast<uint32_t>(voff / 8));
-                ref_sum += h_ref;
-#pragma unroll 1
-                for (int k = 0; k < kg; ++k) {
-                    cp_async_wait<kRing - 1>();
-                    at = ring_base + stage * 512u;
-                    const uint4 c = lds128(at);
-                    stage = (stage + 1u) & (kRing - 1);
-                    issue_one(at);
-                    queued_visit(c, r, h_ref, force, voff, k);
-                }
+                queued_visit(c, r, h_ref, force, voff, k);
             }
         }
-        cp_async_wait<0>();
-        if (qcount) {                                   // the tensor's accumulators close: drain the queue
-            __syncwarp();
-            ragged_batch(dt, qbase, qhead, qcount, slots, wacc, tol);
-            __syncwarp();
-        }
     }
+    cp_async_wait<0>();
+    if (qcount) {                                   // the tensor's accumulators close: drain the queue
+        __syncwarp();
+        ragged_batch(dt, qbase, qhead, qcount, slots, wacc, tol);
+        __syncwarp();
+    }
+    return ref_sum;
+}
 
-    // ---- synchronous part: the tail tile, or every tile of a tensor that is not streamed (out of line: cold
-    // code whose registers the streaming loops should not pay for) ----
-    if (full_end < tile_end) ref_sum += ragged_tail(dt, ref, nbytes, full_end, tile_end, kg, slots, wacc, wptr, tol, nan_matters);
+template <bool FOUR>
+__device__ __forceinline__ void ragged_stretch(const RaggedParams& p, int dt, const unsigned char* ref, uint64_t n,
+                                               uint64_t tile_begin, uint64_t tile_end, int kg, uint2* slots,
+                                               CtaAcc* wacc, const unsigned char* const* wsrc, unsigned char* smem) {
+    const unsigned char* const* wptr = wsrc + 1;        // wsrc[0] = the reference, wsrc[1 + k] = candidate k
+    const int esz = elem_size(dt);
+    const uint64_t nbytes = n * esz;
+    bool streamed = (reinterpret_cast<uintptr_t>(ref) & 15u) == 0 && nbytes < (1ull << 35);
+    for (int k = 0; k < kg; ++k) streamed = streamed && (reinterpret_cast<uintptr_t>(wptr[k]) & 15u) == 0;
+    const uint64_t full_end_all = nbytes / kWarpTile;                  // tiles [0, full_end_all) are full
+    const uint64_t full_end = streamed ? (tile_end < full_end_all ? tile_end : full_end_all) : tile_begin;
+    uint64_t ref_sum = 0;
+    if (full_end > tile_begin) ref_sum = ragged_stream<FOUR>(p, dt, tile_begin, full_end, kg, smem);
+    // ---- synchronous part: the tail tile, or every tile of a tensor that is not streamed (out of line too) ----
+    if (full_end < tile_end) {
+        const TolF tol = {p.atol, p.rtol, p.equal_nan};
+        const uint32_t qbase = smem_u32(smem + RaggedSmem::kQueueOff) + (threadIdx.x >> 5) * static_cast<uint32_t>(kQueueBytes);
+        ref_sum += ragged_tail(dt, ref, nbytes, full_end, tile_end, kg, slots, wacc, wptr, tol, (dt <= GV_F16) && !p.equal_nan, qbase);
+    }
     for (int k = 0; k < kg; ++k) {
         const uint2 sl = slots[k * 32];
         const uint64_t h = pack64(sl.x, sl.y) + ref_sum;
@@ -1261,6 +1343,25 @@ struct ChunkPlan {
     }
 };
 
+// The table entries of tensor t, one per lane and all in flight together (a dependent chain of loads per
+// tensor is what made batches of tiny tensors slow): lane 0 the tensor's first unit in the work sequence,
+// lane 1 its end, lane 2 the dtype, lane 3 the element count (or the next reference offset when counts are
+// read off the offsets), lane 4 the reference offset, lanes kMetaCand.. the offsets of its first 16 candidates.
+constexpr int kMetaCand = 8;
+__device__ __forceinline__ uint64_t load_meta(const RaggedParams& p, int64_t t, int lane) {
+    uint64_t v = 0;
+    if (t < p.T) {
+        if (lane == 0) v = static_cast<uint64_t>(p.tile_prefix[t]);
+        else if (lane == 1) v = static_cast<uint64_t>(p.tile_prefix[t + 1]);
+        else if (lane == 2) v = p.dtypes[t];
+        else if (lane == 3) v = static_cast<uint64_t>(p.n_elems ? p.n_elems[t] : p.ref_off[t + 1]);
+        else if (lane == 4) v = static_cast<uint64_t>(p.ref_off[t]);
+        else if (lane >= kMetaCand && lane - kMetaCand < (p.N < kChunk ? p.N : kChunk))
+            v = static_cast<uint64_t>(p.cand_off[t * p.N + (lane - kMetaCand)]);
+    }
+    return v;
+}
+
 // One tensor's tiles [tile_begin, tile_end) against all its candidates, from pointer set-up to the publication
 // of the partial records. Out of line on purpose: the streaming loops inside get a register allocation of
 // their own, separate from the chunk bookkeeping of the kernel that calls this.
@@ -1271,25 +1372,26 @@ __device__ __noinline__ void ragged_part(const RaggedParams& p, int64_t t, uint6
     uint2* slots = reinterpret_cast<uint2*>(smem + RaggedSmem::kSlotOff) + size_t(warp) * kChunk * 32 + lane;
     CtaAcc* wacc = reinterpret_cast<CtaAcc*>(smem + RaggedSmem::kAccOff) + warp * kChunk;
     const unsigned char** wsrc = reinterpret_cast<const unsigned char**>(smem + RaggedSmem::kPtrOff) + warp * (kChunk + 2);
-    const uint32_t ring_base = smem_u32(smem + RaggedSmem::kRingOff) + (warp * kRing * 32 + lane) * 16;
-    const uint32_t qbase = smem_u32(smem + RaggedSmem::kQueueOff) + warp * static_cast<uint32_t>(kQueueBytes);
-    const uint32_t refst_base = smem_u32(smem + RaggedSmem::kRefOff) + (warp * 2 * 32 + lane) * 16;
-    const int dt = p.dtypes[t];
-    const int esz = elem_size(dt);
-    const uint64_t n = p.n_elems ? static_cast<uint64_t>(p.n_elems[t])
-                                 : static_cast<uint64_t>(p.ref_off[t + 1] - p.ref_off[t]) / esz;
-    const unsigned char* ref = p.ref_base + p.ref_off[t];
+    // the tensor's table entries, as the caller's load_meta delivered them (one per lane, now in shared memory)
+    const unsigned long long* wmeta = reinterpret_cast<const unsigned long long*>(smem + RaggedSmem::kMetaOff) + warp * 32;
+    const int dt = static_cast<int>(wmeta[2]);
+    const uint64_t n = p.n_elems ? wmeta[3] : (wmeta[3] - wmeta[4]) / static_cast<uint64_t>(elem_size(dt));
+    const unsigned char* ref = p.ref_base + wmeta[4];
     for (int c0 = 0; c0 < p.N; c0 += kChunk) {
         const int kg = FOUR ? 4 : min(kChunk, p.N - c0);
         __syncwarp();
-        if (lane < kg) {
+        // candidate pointers: the first group's offsets came with the tensor's other table entries (lanes
+        // kMetaCand .. kMetaCand + 15 of lane_meta, see load_meta), further groups are read here
+        if (c0 == 0) {
+            if (lane < kg) wsrc[1 + lane] = p.cand_base + wmeta[kMetaCand + lane];
+        } else if (lane < kg) {
             wsrc[1 + lane] = p.cand_base + p.cand_off[t * p.N + c0 + lane];
-            wacc[lane].clear();
         }
+        if (lane < kg) wacc[lane].clear();
         if (lane == 0) wsrc[0] = ref;
         for (int k = 0; k < kg; ++k) slots[k * 32] = make_uint2(0u, 0u);
         __syncwarp();
-        ragged_stretch<FOUR>(p, dt, ref, n, tile_begin, tile_end, kg, slots, wacc, wsrc, lane, ring_base, qbase, refst_base);
+        ragged_stretch<FOUR>(p, dt, ref, n, tile_begin, tile_end, kg, slots, wacc, wsrc, smem);
         __syncwarp();
         // leave the tensor (or this group of its candidates): combine and publish
         for (int k = 0; k < kg; ++k) {
@@ -1306,6 +1408,7 @@ template <bool FOUR>
 __global__ void __launch_bounds__(kThreads, 2) ragged_kernel(const __grid_constant__ RaggedParams p) {
     extern __shared__ __align__(128) unsigned char smem[];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    unsigned long long* wmeta = reinterpret_cast<unsigned long long*>(smem + RaggedSmem::kMetaOff) + warp * 32;
     const uint64_t gw = static_cast<uint64_t>(blockIdx.x) * kWarps + warp;
     const uint64_t GW = static_cast<uint64_t>(gridDim.x) * kWarps;
     const ChunkPlan plan(static_cast<uint64_t>(p.tile_prefix[p.T]), GW);
@@ -1329,16 +1432,30 @@ __global__ void __launch_bounds__(kThreads, 2) ragged_kernel(const __grid_consta
             hi = nlo + stride < hi ? nlo + stride : hi;
             lo = nlo;
         }
+        // Walk the tensors of the chunk. A tensor occupies kPartCost + tiles units of the sequence: the first
+        // kPartCost stand for the fixed cost of handling it (so chunks of many tiny tensors are not far
+        // costlier than chunks of few large ones), the rest are its tiles.
         int64_t t = lo;
         uint64_t item = begin;
+        uint64_t meta = load_meta(p, t, lane);
         while (item < end && t < p.T) {         // (t < T always holds for a consistent prefix table; the guard keeps a corrupted one from walking off its end)
-            const uint64_t t_first = static_cast<uint64_t>(p.tile_prefix[t]);
-            const uint64_t t_last = static_cast<uint64_t>(p.tile_prefix[t + 1]);
-            if (t_last > item) {                                    // (else: empty or already finished tensor)
-                const uint64_t tile_end = (t_last < end ? t_last : end) - t_first;
-                ragged_part<FOUR>(p, t, item - t_first, tile_end, smem);
-                item = t_first + tile_end;
+            const uint64_t meta_next = load_meta(p, t + 1, lane);       // in flight while tensor t is processed
+            const uint64_t t_first = __shfl_sync(0xFFFFFFFFu, meta, 0);
+            const uint64_t t_last = __shfl_sync(0xFFFFFFFFu, meta, 1);
+            if (t_last > item) {                                    // (else: empty or rejected tensor, no units)
+                const uint64_t tiles0 = t_first + kPartCost;        // where the tensor's tiles begin in the sequence
+                const uint64_t stop = t_last < end ? t_last : end;
+                const uint64_t tile_begin = item > tiles0 ? item - tiles0 : 0;
+                const uint64_t tile_end = stop > tiles0 ? stop - tiles0 : 0;
+                if (tile_end > tile_begin) {
+                    __syncwarp();
+                    wmeta[lane] = meta;
+                    __syncwarp();
+                    ragged_part<FOUR>(p, t, tile_begin, tile_end, smem);
+                }
+                item = stop;
             }
+            meta = meta_next;
             ++t;
         }
         chunk = GW + __shfl_sync(0xFFFFFFFFu, next, 0);

@@ -230,3 +230,47 @@ def test_bf16_tensor_beyond_32_gib_uses_64_bit_word_indices(oracle):
     got = _big_case(oracle, torch.bfloat16, [1.0, -2.0, 0.5, 3.0], lambda n: [3, (1 << 34) + 6, n - 2], lambda v: v + 0.5)
     assert got["max_abs_err"] == np.float32(0.5) and int(got["max_abs_diff_int"]) == 0
     assert got["max_rel_err"] == np.float32(1.0)            # 0.5 -> 1.0 at two of the places; 3.0 -> 3.5 at the third
+
+
+def test_ragged_tensor_beyond_32_gib(oracle):
+    """Maximum sizes, ragged path: one 34 GiB int32 tensor (it takes the unstreamed path with 64-bit word
+    indices) next to a small one, one candidate each. The giant's hash is pinned by the patterned-buffer closed
+    form evaluated by the oracle block by block; the changed places are known by construction; the small
+    tensor's records are compared with the oracle directly."""
+    n_words = (34 << 30) // 8 + 1
+    n_big = n_words * 2
+    n_small = 1000
+    free, _ = torch.cuda.mem_get_info()
+    need = 2 * (n_big + n_small) * 4 + (6 << 30)
+    if free < need:
+        pytest.skip(f"needs {need >> 30} GiB of free device memory")
+    pat = torch.tensor([0x0BADF00D, -12345], dtype=torch.int32, device=DEV)
+    word = int.from_bytes(host_bytes(pat).tobytes(), "little")
+    g = torch.Generator(device=DEV).manual_seed(7)
+    small = torch.randint(-100, 100, (n_small,), generator=g, device=DEV, dtype=torch.int32)
+    ref = torch.cat([pat.repeat(n_words), small])
+    cand = ref.clone()
+    places = [1, (1 << 33) + 2, n_big - 1]
+    for p in places:
+        cand[p] += 5
+    cand[n_big + 17] -= 1
+    ref_off = torch.tensor([0, n_big * 4, (n_big + n_small) * 4], dtype=torch.int64, device=DEV)
+    cand_off = torch.tensor([0, n_big * 4], dtype=torch.int64, device=DEV)
+    dtypes = torch.full((2,), 3, dtype=torch.uint8, device=DEV)
+    ws = torch.empty(gv.gv_workspace_bytes(2, 1), dtype=torch.uint8, device=DEV)
+    res = gv.gv_verify_ragged(ref.view(torch.uint8), ref_off, cand.view(torch.uint8), cand_off, dtypes, 1, 0.0, 0.0, False,
+                              workspace=ws)
+    torch.cuda.synchronize()
+    assert gv.gv_check(ws) == gv.GV_OK
+    got = gv.results_to_numpy(res)
+    M64 = (1 << 64) - 1
+    want = _patterned_hash(oracle, n_words, word)
+    for k in sorted({p // 2 for p in places}):
+        w_new = int.from_bytes(host_bytes(cand[2 * k:2 * k + 2]).tobytes(), "little")
+        want = (want - oracle.splitmix64(k ^ word) + oracle.splitmix64(k ^ w_new)) & M64
+    assert int(got[0]["hash"]) == want
+    assert int(got[0]["n_mismatch"]) == 3 and int(got[0]["first_mismatch"]) == 1 and int(got[0]["max_abs_diff_int"]) == 5
+    w_small = oracle.verify(host_bytes(small), host_bytes(cand[n_big:]), oracle.I32)
+    assert got[1].tobytes() == w_small.tobytes()
+    del ref, cand
+    torch.cuda.empty_cache()

@@ -212,3 +212,33 @@ def test_ragged_four_candidates_with_nan_and_inf_in_the_references(oracle, equal
         assert got[i].tobytes() == want[i].tobytes(), (i, got[i], want[i])
     n_nan = int(torch.isnan(refs[0]).sum())
     assert int(got[0]["n_mismatch"]) == (0 if equal_nan else n_nan)      # fp32 tensor, exact copy: only its NaNs can mismatch
+
+
+@pytest.mark.parametrize("order", ["ascending", "descending", "small_last"])
+def test_ragged_records_do_not_depend_on_the_order_of_the_tensors(oracle, order):
+    """The ragged kernel hands out work in chunks of the tensor sequence; with the tensors sorted by size a
+    chunk holds hundreds of tiny tensors or a slice of one large tensor. Same tensors, tables permuted on the
+    host (the data stay where they are): every tensor's records must equal the oracle's for the original order."""
+    wl = W.config5(DEV, T=2500, max_log2=17.0, seed=31)
+    N = wl.N
+    ne = wl.n_elems
+    if order == "ascending":
+        perm = sorted(range(wl.T), key=lambda t: ne[t])
+    elif order == "descending":
+        perm = sorted(range(wl.T), key=lambda t: -ne[t])
+    else:
+        perm = [t for t in range(wl.T) if ne[t] >= 2048] + [t for t in range(wl.T) if ne[t] < 2048]
+    idx = torch.tensor(perm, device=DEV)
+    ro = torch.cat([wl.ref_off[idx], wl.ref_off[-1:]])
+    co = wl.cand_off.view(wl.T, N)[idx].contiguous().view(-1)
+    ws = torch.empty(gv.gv_workspace_bytes(wl.T, N), dtype=torch.uint8, device=DEV)
+    res = gv.gv_verify_ragged(wl.ref_buf, ro, wl.cand_buf, co, wl.dtypes[idx].contiguous(), N, wl.atol, wl.rtol,
+                              wl.equal_nan, n_elems=wl.n_elems_t[idx].contiguous(), workspace=ws)
+    torch.cuda.synchronize()
+    assert gv.gv_check(ws) == gv.GV_OK
+    got = gv.results_to_numpy(res).reshape(wl.T, N)
+    want = oracle.verify_ragged(wl.ref_buf.cpu().numpy(), wl.ref_off.cpu().numpy(), wl.cand_buf.cpu().numpy(),
+                                wl.cand_off.cpu().numpy(), wl.dtypes.cpu().numpy(), N, wl.atol, wl.rtol, wl.equal_nan,
+                                n_elems=wl.n_elems_t.cpu().numpy()).reshape(wl.T, N)
+    for pos, t in enumerate(perm):
+        assert got[pos].tobytes() == want[t].tobytes(), (order, pos, t, ne[t])

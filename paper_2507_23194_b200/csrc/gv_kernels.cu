@@ -912,15 +912,24 @@ __global__ void __launch_bounds__(1024) ragged_prepass_kernel(RaggedParams p) {
 // partials of the current tensor live in per-(candidate, lane) shared-memory slots and the other
 // statistics in per-warp shared accumulators, all flushed with integer atomics when the warp leaves
 // the tensor. No barrier is used anywhere: warps never share a tensor's accumulators.
+// FOUR: the instance for exactly four candidates per tensor keeps slots, accumulators and pointers for four
+// candidates only (79 KB per CTA instead of 109). Both instances run 8 warps per CTA and 2 CTAs per SM: more
+// warps would need fewer registers than the compare code wants (10 warps at 96 registers: no gain; 11 at
+// 80, or 3 CTAs of 7 warps: a third slower).
+template <bool FOUR>
 struct RaggedSmem {
-    static constexpr size_t kRingOff = 0;                                                  // [warp][kRing][32] uint4
-    static constexpr size_t kSlotOff = kRingOff + size_t(kWarps) * kRing * kWarpTile;      // [warp][kChunk][32] u64
-    static constexpr size_t kAccOff = kSlotOff + size_t(kWarps) * kChunk * 32 * 8;         // [warp][kChunk] CtaAcc
-    static constexpr size_t kPtrOff = kAccOff + size_t(kWarps) * kChunk * sizeof(CtaAcc);  // [warp][kChunk + 2] reference + candidate pointers
-    static constexpr size_t kQueueOff = kPtrOff + size_t(kWarps) * (kChunk + 2) * 8;       // [warp][3][kQCap] uint4
-    static constexpr size_t kRefOff = kQueueOff + size_t(kWarps) * kQueueBytes;            // [warp][2][32] uint4 (four-candidate loop)
-    static constexpr size_t kMetaOff = kRefOff + size_t(kWarps) * 2 * kWarpTile;            // [warp][32] u64: table entries of the current tensor
-    static constexpr size_t kTotal = kMetaOff + size_t(kWarps) * 32 * 8;
+    static constexpr int kWarpsPerCta = 8;
+    static constexpr int kCtasPerSm = 2;
+    static constexpr int kCtaThreads = kWarpsPerCta * 32;
+    static constexpr int kCands = FOUR ? 4 : kChunk;                                        // candidates handled at a time
+    static constexpr size_t kRingOff = 0;                                                   // [warp][kRing][32] uint4
+    static constexpr size_t kSlotOff = kRingOff + size_t(kWarpsPerCta) * kRing * kWarpTile;        // [warp][kCands][32] u64
+    static constexpr size_t kAccOff = kSlotOff + size_t(kWarpsPerCta) * kCands * 32 * 8;           // [warp][kCands] CtaAcc
+    static constexpr size_t kPtrOff = kAccOff + size_t(kWarpsPerCta) * kCands * sizeof(CtaAcc);    // [warp][kCands + 2] reference + candidate pointers
+    static constexpr size_t kQueueOff = kPtrOff + size_t(kWarpsPerCta) * (kCands + 2) * 8;         // [warp][3][kQCap] uint4
+    static constexpr size_t kRefOff = kQueueOff + size_t(kWarpsPerCta) * kQueueBytes;              // [warp][2][32] uint4 (four-candidate loop)
+    static constexpr size_t kMetaOff = kRefOff + size_t(kWarpsPerCta) * 2 * kWarpTile;             // [warp][32] u64: table entries of the current tensor
+    static constexpr size_t kTotal = kMetaOff + size_t(kWarpsPerCta) * 32 * 8;
 };
 
 // Code size matters in this kernel: the warps of an SM are in different places at the same time (the
@@ -1165,12 +1174,13 @@ __device__ __noinline__ uint64_t ragged_stream(const RaggedParams& p, int dt, ui
     // neither the tail code nor the chunk bookkeeping, can disturb. Returns the sum of the reference's hash
     // terms over the tiles it met.)
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    uint2* slots = reinterpret_cast<uint2*>(smem + RaggedSmem::kSlotOff) + size_t(warp) * kChunk * 32 + lane;
-    CtaAcc* wacc = reinterpret_cast<CtaAcc*>(smem + RaggedSmem::kAccOff) + warp * kChunk;
-    const unsigned char* const* wsrc = reinterpret_cast<const unsigned char* const*>(smem + RaggedSmem::kPtrOff) + warp * (kChunk + 2);
-    const uint32_t ring_base = smem_u32(smem + RaggedSmem::kRingOff) + (warp * kRing * 32 + lane) * 16;
-    const uint32_t qbase = smem_u32(smem + RaggedSmem::kQueueOff) + warp * static_cast<uint32_t>(kQueueBytes);
-    const uint32_t refst_base = smem_u32(smem + RaggedSmem::kRefOff) + (warp * 2 * 32 + lane) * 16;
+    using S = RaggedSmem<FOUR>;
+    uint2* slots = reinterpret_cast<uint2*>(smem + S::kSlotOff) + size_t(warp) * S::kCands * 32 + lane;
+    CtaAcc* wacc = reinterpret_cast<CtaAcc*>(smem + S::kAccOff) + warp * S::kCands;
+    const unsigned char* const* wsrc = reinterpret_cast<const unsigned char* const*>(smem + S::kPtrOff) + warp * (S::kCands + 2);
+    const uint32_t ring_base = smem_u32(smem + S::kRingOff) + (warp * kRing * 32 + lane) * 16;
+    const uint32_t qbase = smem_u32(smem + S::kQueueOff) + warp * static_cast<uint32_t>(kQueueBytes);
+    const uint32_t refst_base = smem_u32(smem + S::kRefOff) + (warp * 2 * 32 + lane) * 16;
     const TolF tol = {p.atol, p.rtol, p.equal_nan};
     const bool nan_matters = (dt <= GV_F16) && !p.equal_nan;
 
@@ -1308,7 +1318,7 @@ __device__ __forceinline__ void ragged_stretch(const RaggedParams& p, int dt, co
     // ---- synchronous part: the tail tile, or every tile of a tensor that is not streamed (out of line too) ----
     if (full_end < tile_end) {
         const TolF tol = {p.atol, p.rtol, p.equal_nan};
-        const uint32_t qbase = smem_u32(smem + RaggedSmem::kQueueOff) + (threadIdx.x >> 5) * static_cast<uint32_t>(kQueueBytes);
+        const uint32_t qbase = smem_u32(smem + RaggedSmem<FOUR>::kQueueOff) + (threadIdx.x >> 5) * static_cast<uint32_t>(kQueueBytes);
         ref_sum += ragged_tail(dt, ref, nbytes, full_end, tile_end, kg, slots, wacc, wptr, tol, (dt <= GV_F16) && !p.equal_nan, qbase);
     }
     for (int k = 0; k < kg; ++k) {
@@ -1369,16 +1379,17 @@ template <bool FOUR>
 __device__ __noinline__ void ragged_part(const RaggedParams& p, int64_t t, uint64_t tile_begin, uint64_t tile_end,
                                          unsigned char* smem) {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    uint2* slots = reinterpret_cast<uint2*>(smem + RaggedSmem::kSlotOff) + size_t(warp) * kChunk * 32 + lane;
-    CtaAcc* wacc = reinterpret_cast<CtaAcc*>(smem + RaggedSmem::kAccOff) + warp * kChunk;
-    const unsigned char** wsrc = reinterpret_cast<const unsigned char**>(smem + RaggedSmem::kPtrOff) + warp * (kChunk + 2);
+    using S = RaggedSmem<FOUR>;
+    uint2* slots = reinterpret_cast<uint2*>(smem + S::kSlotOff) + size_t(warp) * S::kCands * 32 + lane;
+    CtaAcc* wacc = reinterpret_cast<CtaAcc*>(smem + S::kAccOff) + warp * S::kCands;
+    const unsigned char** wsrc = reinterpret_cast<const unsigned char**>(smem + S::kPtrOff) + warp * (S::kCands + 2);
     // the tensor's table entries, as the caller's load_meta delivered them (one per lane, now in shared memory)
-    const unsigned long long* wmeta = reinterpret_cast<const unsigned long long*>(smem + RaggedSmem::kMetaOff) + warp * 32;
+    const unsigned long long* wmeta = reinterpret_cast<const unsigned long long*>(smem + S::kMetaOff) + warp * 32;
     const int dt = static_cast<int>(wmeta[2]);
     const uint64_t n = p.n_elems ? wmeta[3] : (wmeta[3] - wmeta[4]) / static_cast<uint64_t>(elem_size(dt));
     const unsigned char* ref = p.ref_base + wmeta[4];
-    for (int c0 = 0; c0 < p.N; c0 += kChunk) {
-        const int kg = FOUR ? 4 : min(kChunk, p.N - c0);
+    for (int c0 = 0; c0 < p.N; c0 += S::kCands) {
+        const int kg = FOUR ? 4 : min(S::kCands, p.N - c0);
         __syncwarp();
         // candidate pointers: the first group's offsets came with the tensor's other table entries (lanes
         // kMetaCand .. kMetaCand + 15 of lane_meta, see load_meta), further groups are read here
@@ -1405,12 +1416,14 @@ __device__ __noinline__ void ragged_part(const RaggedParams& p, int64_t t, uint6
 }
 
 template <bool FOUR>
-__global__ void __launch_bounds__(kThreads, 2) ragged_kernel(const __grid_constant__ RaggedParams p) {
+__global__ void __launch_bounds__(RaggedSmem<FOUR>::kCtaThreads, RaggedSmem<FOUR>::kCtasPerSm)
+ragged_kernel(const __grid_constant__ RaggedParams p) {
     extern __shared__ __align__(128) unsigned char smem[];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    unsigned long long* wmeta = reinterpret_cast<unsigned long long*>(smem + RaggedSmem::kMetaOff) + warp * 32;
-    const uint64_t gw = static_cast<uint64_t>(blockIdx.x) * kWarps + warp;
-    const uint64_t GW = static_cast<uint64_t>(gridDim.x) * kWarps;
+    using S = RaggedSmem<FOUR>;
+    unsigned long long* wmeta = reinterpret_cast<unsigned long long*>(smem + S::kMetaOff) + warp * 32;
+    const uint64_t gw = static_cast<uint64_t>(blockIdx.x) * S::kWarpsPerCta + warp;
+    const uint64_t GW = static_cast<uint64_t>(gridDim.x) * S::kWarpsPerCta;
     const ChunkPlan plan(static_cast<uint64_t>(p.tile_prefix[p.T]), GW);
     uint64_t chunk = gw;
     while (chunk < plan.n_chunks) {
@@ -1540,6 +1553,32 @@ gv_status launch_dense(gv_dtype dt, const gv::DenseParams& p, int sm_count, cuda
         case GV_I64: return bigk ? launch_dense_t<GV_I64, true>(p, sm_count, st) : launch_dense_t<GV_I64, false>(p, sm_count, st);
     }
     return GV_ERR_UNSUPPORTED;
+}
+
+// The pre-pass and the main kernel of a ragged call (shared by the two ragged entry points).
+template <bool FOUR>
+gv_status launch_ragged_t(const gv::RaggedParams& p, int sm_count, cudaStream_t st) {
+    using S = gv::RaggedSmem<FOUR>;
+    static int blocks_per_sm[64] = {0};
+    int dev = 0;
+    GV_CUDA(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) return GV_ERR_CUDA;
+    auto kern = gv::ragged_kernel<FOUR>;
+    if (blocks_per_sm[dev] == 0) {
+        GV_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(S::kTotal)));
+        int b = 0;
+        GV_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b, kern, S::kCtaThreads, S::kTotal));
+        blocks_per_sm[dev] = b > 0 ? b : 1;
+    }
+    const unsigned grid = static_cast<unsigned>(sm_count * blocks_per_sm[dev]);
+    kern<<<grid, S::kCtaThreads, S::kTotal, st>>>(p);
+    GV_CUDA(cudaGetLastError());
+    return GV_OK;
+}
+gv_status launch_ragged(const gv::RaggedParams& p, int sm_count, cudaStream_t st) {
+    gv::ragged_prepass_kernel<<<1, 1024, 0, st>>>(p);
+    GV_CUDA(cudaGetLastError());
+    return p.N == 4 ? launch_ragged_t<true>(p, sm_count, st) : launch_ragged_t<false>(p, sm_count, st);
 }
 
 }  // namespace
@@ -1711,24 +1750,7 @@ gv_status gv_verify_ragged(const void* ref_base, const int64_t* ref_off, const v
     p.atol = static_cast<float>(tol->atol);
     p.rtol = static_cast<float>(tol->rtol);
     p.equal_nan = tol->equal_nan != 0;
-    gv::ragged_prepass_kernel<<<1, 1024, 0, st>>>(p);
-    GV_CUDA(cudaGetLastError());
-
-    static int blocks_per_sm[64] = {0};
-    int dev = 0;
-    GV_CUDA(cudaGetDevice(&dev));
-    if (blocks_per_sm[dev] == 0) {
-        for (auto kern : {gv::ragged_kernel<false>, gv::ragged_kernel<true>})
-            GV_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(gv::RaggedSmem::kTotal)));
-        int b = 0;
-        GV_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b, gv::ragged_kernel<false>, gv::kThreads, gv::RaggedSmem::kTotal));
-        blocks_per_sm[dev] = b > 0 ? b : 1;
-    }
-    const unsigned grid = static_cast<unsigned>(sm_count * blocks_per_sm[dev]);
-    if (N == 4) gv::ragged_kernel<true><<<grid, gv::kThreads, gv::RaggedSmem::kTotal, st>>>(p);
-    else gv::ragged_kernel<false><<<grid, gv::kThreads, gv::RaggedSmem::kTotal, st>>>(p);
-    GV_CUDA(cudaGetLastError());
-    return GV_OK;
+    return launch_ragged(p, sm_count, st);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -1804,22 +1826,7 @@ gv_status gv_verify_ragged_noalloc(const void* ref_base, const int64_t* ref_off,
     p.atol = static_cast<float>(tol->atol);
     p.rtol = static_cast<float>(tol->rtol);
     p.equal_nan = tol->equal_nan != 0;
-    gv::ragged_prepass_kernel<<<1, 1024, 0, st>>>(p);
-    GV_CUDA(cudaGetLastError());
-
-    static int blocks_per_sm[64] = {0};
-    if (blocks_per_sm[dev] == 0) {
-        for (auto kern : {gv::ragged_kernel<false>, gv::ragged_kernel<true>})
-            GV_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(gv::RaggedSmem::kTotal)));
-        int b = 0;
-        GV_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b, gv::ragged_kernel<false>, gv::kThreads, gv::RaggedSmem::kTotal));
-        blocks_per_sm[dev] = b > 0 ? b : 1;
-    }
-    const unsigned grid = static_cast<unsigned>(sm_count * blocks_per_sm[dev]);
-    if (N == 4) gv::ragged_kernel<true><<<grid, gv::kThreads, gv::RaggedSmem::kTotal, st>>>(p);
-    else gv::ragged_kernel<false><<<grid, gv::kThreads, gv::RaggedSmem::kTotal, st>>>(p);
-    GV_CUDA(cudaGetLastError());
-    return GV_OK;
+    return launch_ragged(p, sm_count, st);
 }
 
 gv_status gv_hash(const void* buf, uint64_t nbytes, uint64_t* out, void* cuda_stream) {

@@ -442,7 +442,11 @@ def main():
     wl = build_workload(args.workload, device, args.cands, args.tensors)
     ragged = isinstance(wl, W.RaggedWorkload)
     if args.only_class and not ragged:
-        keep = [j for j, f in enumerate(wl.facts) if f["class"] == args.only_class]
+        # a recipe class ("noise"), or a class with its parameter as the recipe records it ("rel_noise0.005", "swaps1e-05")
+        keep = [j for j, f in enumerate(wl.facts)
+                if args.only_class in (f["class"], f["class"] + str(f.get("sigma", "")) + str(f.get("frac", "")))]
+        if not keep:
+            raise SystemExit(f"no candidate of class {args.only_class!r} in {wl.name}")
         wl.cands = [wl.cands[j] for j in keep]
         wl.facts = [wl.facts[j] for j in keep]
         wl.name += ":" + args.only_class

@@ -217,6 +217,45 @@ template <> struct Widen<GV_F16> {
     }
 };
 
+// |fl32(c_e - r_e)| for the elements of a candidate vector against an already widened reference vector.
+// For the 16-bit types the subtraction takes the candidate element as it is: sm_100's mixed-precision
+// subtract (sub.rn.f32.f16 / .bf16: the 16-bit operand is converted exactly, then one correctly rounded
+// binary32 subtraction, subnormals kept) does in one instruction what "widen, then subtract" does in two
+// or three -- the same value, bit for bit.
+template <int DT> struct AbsDiff;
+template <> struct AbsDiff<GV_F32> {
+    static __device__ __forceinline__ void run(const uint4& c, const float (&rf)[4], float (&ad)[4]) {
+        ad[0] = fabsf(__fsub_rn(__uint_as_float(c.x), rf[0])); ad[1] = fabsf(__fsub_rn(__uint_as_float(c.y), rf[1]));
+        ad[2] = fabsf(__fsub_rn(__uint_as_float(c.z), rf[2])); ad[3] = fabsf(__fsub_rn(__uint_as_float(c.w), rf[3]));
+    }
+};
+template <> struct AbsDiff<GV_BF16> {
+    static __device__ __forceinline__ void run(const uint4& c, const float (&rf)[8], float (&ad)[8]) {
+        const uint32_t w[4] = {c.x, c.y, c.z, c.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            float d0, d1;
+            asm("{ .reg .b16 lo, hi;\n\t mov.b32 {lo, hi}, %2;\n\t sub.rn.f32.bf16 %0, lo, %3;\n\t sub.rn.f32.bf16 %1, hi, %4; }"
+                : "=f"(d0), "=f"(d1) : "r"(w[i]), "f"(rf[2 * i]), "f"(rf[2 * i + 1]));
+            ad[2 * i] = fabsf(d0);
+            ad[2 * i + 1] = fabsf(d1);
+        }
+    }
+};
+template <> struct AbsDiff<GV_F16> {
+    static __device__ __forceinline__ void run(const uint4& c, const float (&rf)[8], float (&ad)[8]) {
+        const uint32_t w[4] = {c.x, c.y, c.z, c.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            float d0, d1;
+            asm("{ .reg .b16 lo, hi;\n\t mov.b32 {lo, hi}, %2;\n\t sub.rn.f32.f16 %0, lo, %3;\n\t sub.rn.f32.f16 %1, hi, %4; }"
+                : "=f"(d0), "=f"(d1) : "r"(w[i]), "f"(rf[2 * i]), "f"(rf[2 * i + 1]));
+            ad[2 * i] = fabsf(d0);
+            ad[2 * i + 1] = fabsf(d1);
+        }
+    }
+};
+
 // ------------------------------------------------------------------------------------------
 // per-thread partial statistics of one candidate visit
 // ------------------------------------------------------------------------------------------
@@ -426,13 +465,10 @@ __device__ __forceinline__ bool vec_fast_float(const uint4& c, const RefVec<16 /
     // running maxima of this (CTA, candidate): max|d| bits, max relative error bits, filter threshold
     const uint4 run = lds128(smem_u32(&s->maxabs));
     const float nT = -__uint_as_float(run.z);
-    float cf[EPV], ad[EPV], w[EPV];
-    Widen<DT>::run(c, cf);
+    float ad[EPV], w[EPV];
+    AbsDiff<DT>::run(c, r.rf, ad);
 #pragma unroll
-    for (int e = 0; e < EPV; ++e) {
-        ad[e] = fabsf(__fsub_rn(cf[e], r.rf[e]));
-        w[e] = __fmaf_rn(nT, fabsf(r.rf[e]), ad[e]);         // > 0  <=  the quotient could exceed M
-    }
+    for (int e = 0; e < EPV; ++e) w[e] = __fmaf_rn(nT, fabsf(r.rf[e]), ad[e]);         // > 0  <=  the quotient could exceed M
     float va, vw;       // va propagates NaN: a NaN anywhere (candidate or reference) must not be skipped
     if (EPV == 8) {
         va = max2_nan(max3_nan(ad[0], ad[1], ad[2]), max3_nan(max3_nan(ad[3], ad[4], ad[5]), ad[6], ad[7]));

@@ -416,6 +416,17 @@ __device__ __forceinline__ uint32_t rel_threshold_bits(uint32_t m_bits) {
     return __float_as_uint(__fmul_rd(__uint_as_float(m_bits), __uint_as_float(0x3F7FFFF0u)));   // 1 - 2^-20
 }
 
+// Add a 32-bit count to a 64-bit counter in shared memory. A 64-bit shared-memory atomic add is a
+// compare-and-swap loop, and the lanes of a warp that add to the same counter (a batch of entries of one
+// candidate that mismatch everywhere) then retry against each other; the 32-bit add is one instruction
+// that resolves the conflict in hardware. The carry into the upper word is added separately (exact:
+// the sum wraps mod 2^64, and nothing reads the counter before the CTA's final barrier).
+__device__ __forceinline__ void add_count(unsigned long long* counter, uint32_t v) {
+    uint32_t* w = reinterpret_cast<uint32_t*>(counter);
+    const uint32_t old = atomicAdd(w, v);
+    if (old + v < old) atomicAdd(w + 1, 1u);
+}
+
 // Raise the CTA's running maxima (bit patterns of non-negative floats).
 __device__ __forceinline__ void raise_maxabs(CtaAcc* s, uint32_t bits) {
     if (bits > *reinterpret_cast<volatile unsigned int*>(&s->maxabs)) {
@@ -495,7 +506,7 @@ __device__ __forceinline__ bool vec_fast_float(const uint4& c, const RefVec<16 /
             if (ad[e] > tolc_of(fabsf(r.rf[e]), t)) { cnt += 1u; first_e = e; }
         }
         if (cnt) {
-            if (ADD_NOW) atomicAdd(&s->cnt, static_cast<unsigned long long>(cnt));
+            if (ADD_NOW) add_count(&s->cnt, cnt);
             else n_not_close += cnt;
             const unsigned long long idx = elem0 + first_e;
             if (idx < *reinterpret_cast<volatile unsigned long long*>(&s->first)) atomicMin(&s->first, idx);
@@ -652,7 +663,7 @@ __device__ __forceinline__ uint64_t warp_max_u64(uint64_t v) {
 // Merge per-lane mismatch counts at a point where all 32 lanes of the warp are converged.
 __device__ __forceinline__ void merge_counts_converged(CtaAcc* s, uint32_t lane_cnt) {
     const uint32_t total = __reduce_add_sync(0xFFFFFFFFu, lane_cnt);
-    if (total && (threadIdx.x & 31) == 0) atomicAdd(&s->cnt, static_cast<unsigned long long>(total));
+    if (total && (threadIdx.x & 31) == 0) add_count(&s->cnt, total);
 }
 
 // Rare-path partials of one thread's visit -> CTA accumulators.
@@ -661,8 +672,8 @@ __device__ __forceinline__ void merge_counts_converged(CtaAcc* s, uint32_t lane_
 __device__ __forceinline__ void push_rare(CtaAcc* s, const Acc& a) {
     if (a.cnt && a.first < *reinterpret_cast<volatile unsigned long long*>(&s->first))
         atomicMin(&s->first, static_cast<unsigned long long>(a.first));
-    if (a.nan) atomicAdd(&s->nan, static_cast<unsigned long long>(a.nan));
-    if (a.inf) atomicAdd(&s->inf, static_cast<unsigned long long>(a.inf));
+    if (a.nan) add_count(&s->nan, a.nan);
+    if (a.inf) add_count(&s->inf, a.inf);
     if (a.maxint > *reinterpret_cast<volatile unsigned long long*>(&s->maxint))
         atomicMax(&s->maxint, static_cast<unsigned long long>(a.maxint));
     raise_maxrel(s, a.maxrel);

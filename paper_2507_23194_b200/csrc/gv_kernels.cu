@@ -232,7 +232,7 @@ __device__ __noinline__ void settle_vector_exact(uint4 c, RefVec<16 / Traits<DT>
     const uint32_t thr = *reinterpret_cast<volatile unsigned int*>(&s->thr);
     vec_exact_float<DT>(c, r, elem0, t, thr, a);
     push_rare(s, a);
-    if (a.cnt) atomicAdd(&s->cnt, static_cast<unsigned long long>(a.cnt));
+    if (a.cnt) add_count(&s->cnt, a.cnt);
     raise_maxabs(s, a.maxabs);
 }
 template <int DT>
@@ -241,7 +241,7 @@ __device__ __noinline__ void settle_vector_int(uint4 c, uint4 r, uint64_t elem0,
     a.clear();
     vec_int<DT>(c, r, elem0, 16 / Traits<DT>::ESZ, a);
     push_rare(s, a);
-    if (a.cnt) atomicAdd(&s->cnt, static_cast<unsigned long long>(a.cnt));
+    if (a.cnt) add_count(&s->cnt, a.cnt);
 }
 
 // Compare the n (<= 32) oldest entries of the warp's queue, one per lane; called with the warp
@@ -270,8 +270,8 @@ __device__ __forceinline__ void batch_entries(uint32_t qbase, uint32_t head, uin
         const uint64_t hs = pack64(sl.x, sl.y) + (h - h_ref);
         slots[k * 32] = make_uint2(static_cast<uint32_t>(hs), static_cast<uint32_t>(hs >> 32));
         CtaAcc* s = &acc[k];
-        // (mismatch counts: one shared atomic per lane that found some -- these do not stall the warp, and a
-        // vote plus a match over the candidate slots measured slower even when every entry mismatches)
+        // (mismatch counts: one 32-bit shared atomic per lane that found some, add_count -- a vote plus a
+        // match over the candidate slots measured slower even when every entry mismatches)
         if constexpr (Traits<DT>::IS_FLOAT) {
             RefVec<16 / ESZ> rv;
             uint32_t rflags = 0u, unused = 0u;
@@ -282,7 +282,7 @@ __device__ __forceinline__ void batch_entries(uint32_t qbase, uint32_t head, uin
             a.clear();
             vec_int<DT>(c, r, voff / ESZ, 16 / ESZ, a);
             push_rare(s, a);
-            if (a.cnt) atomicAdd(&s->cnt, static_cast<unsigned long long>(a.cnt));
+            if (a.cnt) add_count(&s->cnt, a.cnt);
         }
     }
 }
@@ -788,7 +788,7 @@ dense_kernel(const __grid_constant__ DenseParams p) {
                     const uint64_t h = pack64(sl.x, sl.y) + a.hash;
                     slots[k * 32] = make_uint2(static_cast<uint32_t>(h), static_cast<uint32_t>(h >> 32));
                     push_rare(&cacc[k], a);
-                    if (a.cnt) atomicAdd(&cacc[k].cnt, static_cast<unsigned long long>(a.cnt));
+                    if (a.cnt) add_count(&cacc[k].cnt, a.cnt);
                     raise_maxabs(&cacc[k], a.maxabs);
                 }
             }
@@ -953,7 +953,7 @@ __device__ __forceinline__ void ragged_entry(const uint4& c, const uint4& r, uin
         a.clear();
         vec_int<DT>(c, r, voff / ESZ, 16 / ESZ, a);
         push_rare(s, a);
-        if (a.cnt) atomicAdd(&s->cnt, static_cast<unsigned long long>(a.cnt));
+        if (a.cnt) add_count(&s->cnt, a.cnt);
     }
 }
 __device__ __noinline__ void ragged_batch(int dt, uint32_t qbase, uint32_t head, uint32_t n, uint2* slots, CtaAcc* wacc,
@@ -1020,7 +1020,7 @@ __device__ __noinline__ void ragged_elements(int dt, uint4 c, uint4 r, uint64_t 
     const uint64_t h = pack64(sl.x, sl.y) + a.hash;
     *slot = make_uint2(static_cast<uint32_t>(h), static_cast<uint32_t>(h >> 32));
     push_rare(s, a);
-    if (a.cnt) atomicAdd(&s->cnt, static_cast<unsigned long long>(a.cnt));
+    if (a.cnt) add_count(&s->cnt, a.cnt);
     raise_maxabs(s, a.maxabs);
 }
 // A 16-byte vector at byte_off of a tensor of nbytes bytes: one 128-bit load when it is complete and

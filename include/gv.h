@@ -56,7 +56,7 @@ typedef enum gv_dtype { GV_F32 = 0, GV_BF16 = 1, GV_F16 = 2, GV_I32 = 3, GV_I64 
 
 typedef enum gv_status {
     GV_OK = 0,
-    GV_ERR_INVALID_ARG = 1,    /* null pointer, negative count, non-finite or negative tolerance */
+    GV_ERR_INVALID_ARG = 1,    /* null pointer, negative count, negative tolerance or one above FLT_MAX */
     GV_ERR_UNSUPPORTED = 2,    /* dtype code out of range                                       */
     GV_ERR_MISALIGNED = 3,     /* a base address is not a multiple of the element size          */
     GV_ERR_WORKSPACE = 4,      /* workspace missing, misaligned or smaller than gv_workspace_bytes */
@@ -82,8 +82,8 @@ typedef struct gv_result {
 
 /* Tolerances of the comparison (Section 3.1 names them without values; callers choose). */
 typedef struct gv_tol {
-    double atol;       /* finite, >= 0 */
-    double rtol;       /* finite, >= 0 */
+    double atol;       /* >= 0 and at most FLT_MAX: it is used as a finite binary32 value */
+    double rtol;       /* the same */
     int32_t equal_nan; /* nonzero: NaN in both c and r counts as close */
     int32_t reserved;  /* 0 */
 } gv_tol;

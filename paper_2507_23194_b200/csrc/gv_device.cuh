@@ -299,12 +299,12 @@ __device__ __forceinline__ bool is_finite_bits(uint32_t b) { return (b & 0x7F800
 
 // The per-element rule, written out once, exactly as the header states it. Used for every
 // element on the general path and for the elements of vectors the fast path cannot settle.
-// 2^-64 as binary32 bits: below this magnitude a reference element (or a running maximum) is "tiny"
+// 2^-50 as binary32 bits: below this magnitude a reference element (or a running maximum) is "tiny"
 // and the cheap relative-error filter is not trusted (see rel_threshold_bits).
-constexpr uint32_t kTinyBits = 0x1F800000u;
+constexpr uint32_t kTinyBits = 0x26800000u;
 
 // GUARDED: the exact quotient is only needed when it can exceed the running maximum M. Callers that
-// hold a threshold from rel_threshold_bits (T <= M (1 - 2^-20), or 0 while M is tiny) pass it, and the
+// hold a threshold from rel_threshold_bits (T = M, or 0 while M is tiny) pass it, and the
 // division is skipped for elements with |d| <= T |r| (sign of one fused multiply-add).
 template <bool GUARDED>
 __device__ __forceinline__ void element_rule(float c, float r, const TolF& t, uint64_t idx, Acc& a,
@@ -376,7 +376,7 @@ __device__ __forceinline__ float tolc_of(float abs_r, const TolF& t) {
     return fminf(__fadd_rn(t.atol, __fmul_rn(t.rtol, abs_r)), __uint_as_float(0x7F7FFFFFu));
 }
 
-// flags: bit 1 = the vector holds a nonzero element below 2^-64 (relative filter not trusted)
+// flags: bit 1 = the vector holds a nonzero element below 2^-50 (relative filter not trusted)
 template <int DT>
 __device__ __forceinline__ void hoist_ref(const uint4& raw, const TolF& t, RefVec<16 / Traits<DT>::ESZ>& o,
                                           uint32_t& flags) {
@@ -388,7 +388,7 @@ __device__ __forceinline__ void hoist_ref(const uint4& raw, const TolF& t, RefVe
 #pragma unroll
     for (int e = 0; e < EPV; ++e) amin = fminf(amin, fabsf(o.rf[e]));
     o.tolmin = tolc_of(amin, t);
-    // A nonzero element below 2^-64 can only exist when the smallest |r| is below 2^-64 (it may be a
+    // A nonzero element below 2^-50 can only exist when the smallest |r| is below 2^-50 (it may be a
     // zero, so look at the elements then; f16 has no nonzero value that small).
     flags = 0u;
     if (DT != GV_F16 && __float_as_uint(amin) < kTinyBits) {
@@ -402,18 +402,19 @@ __device__ __forceinline__ void hoist_ref(const uint4& raw, const TolF& t, RefVe
     }
 }
 
-// Relative-error filter of one (CTA, candidate). M = largest exact quotient recorded so far;
-// T = M (1 - 2^-20) rounded down, or 0 while M < 2^-64. An element can raise M only if
-// fl(|d| / |r|) > M, which implies |d| / |r| > M (1 - 2^-24), hence |d| - T |r| > |r| M 2^-21 > 0; the
-// fused multiply-add w = fma(-T, |r|, |d|) delivers that difference correctly rounded, so w > 0
-// whenever |r| M 2^-21 is not below the subnormal range -- guaranteed for |r| >= 2^-64 and
-// M >= 2^-64. Vectors holding a nonzero |r| < 2^-64 skip the filter (flag from hoist_ref), and while
-// T == 0 every nonzero |d| passes (w = |d|). When T |r| overflows, |d| / |r| < M and nothing is missed.
-// Elements with r == 0 pass the filter whenever |d| != 0 and are dropped afterwards (no relative error).
+// Relative-error filter of one (CTA, candidate). M = largest quotient fl(|d| / |r|) recorded so far; the
+// threshold T is M itself, or 0 while M < 2^-50. Rounding is monotone and M is a binary32 value, so an
+// element can raise M only if the real quotient exceeds M, i.e. x = |d| - M |r| > 0. The fused
+// multiply-add w = fma(-T, |r|, |d|) rounds that exact x once, which keeps its sign unless a nonzero x
+// rounds to zero; with M >= 2^-50 and |r| >= 2^-50 the product M |r| is a multiple of 2^-146 and |d| one
+// of 2^-149, so a positive x is at least 2^-149 and stays positive: w > 0 exactly when the quotient
+// exceeds M. Elements whose quotient only ties with M -- every element of a candidate of zeros, of a
+// negated or a scaled one, and the usual case in quantised noise -- therefore stop at the filter.
+// Vectors holding a nonzero |r| < 2^-50 skip the filter (flag from hoist_ref), and while T == 0 every
+// nonzero |d| passes (w = |d|). When M |r| overflows the quotient is below M and w is -Inf. Elements
+// with r == 0 pass whenever |d| != 0 and are dropped afterwards (no relative error).
 __device__ __forceinline__ uint32_t rel_threshold_bits(uint32_t m_bits) {
-    if (m_bits < kTinyBits) return 0u;
-    if (m_bits >= 0x7F800000u) return 0x7F800000u;                        // M = +Inf: nothing can exceed it
-    return __float_as_uint(__fmul_rd(__uint_as_float(m_bits), __uint_as_float(0x3F7FFFF0u)));   // 1 - 2^-20
+    return m_bits < kTinyBits ? 0u : m_bits;
 }
 
 // Add a 32-bit count to a 64-bit counter in shared memory. A 64-bit shared-memory atomic add is a
@@ -499,16 +500,17 @@ __device__ __forceinline__ bool vec_fast_float(const uint4& c, const RefVec<16 /
         // the caller runs the exact rule. Otherwise every pair is finite and an element is close
         // exactly when |d| <= its own tolc.
         if (va != va || vab >= 0x7F800000u) return false;
-        uint32_t cnt = 0u;
-        int first_e = EPV;
+        // (every |d| is finite here, so the clamp of tolc_of is not needed: |d| > tol is false for tol = +Inf)
+        uint32_t bad = 0u;
 #pragma unroll
-        for (int e = EPV - 1; e >= 0; --e) {
-            if (ad[e] > tolc_of(fabsf(r.rf[e]), t)) { cnt += 1u; first_e = e; }
+        for (int e = 0; e < EPV; ++e) {
+            if (ad[e] > __fadd_rn(t.atol, __fmul_rn(t.rtol, fabsf(r.rf[e])))) bad |= 1u << e;
         }
-        if (cnt) {
+        if (bad) {
+            const uint32_t cnt = static_cast<uint32_t>(__popc(bad));
             if (ADD_NOW) add_count(&s->cnt, cnt);
             else n_not_close += cnt;
-            const unsigned long long idx = elem0 + first_e;
+            const unsigned long long idx = elem0 + static_cast<uint32_t>(__ffs(bad) - 1);
             if (idx < *reinterpret_cast<volatile unsigned long long*>(&s->first)) atomicMin(&s->first, idx);
         }
     }
@@ -517,12 +519,36 @@ __device__ __forceinline__ bool vec_fast_float(const uint4& c, const RefVec<16 /
         // some element may raise the relative maximum M: each one that passes the filter is examined
         const float M = __uint_as_float(run.y);
         uint32_t best = 0u;
+        // A quotient above M still rounds to M unless it reaches M + half an ulp, i.e. |d| - M |r| >= half |r|
+        // (w is monotone in that difference and half |r| is exact). Without this test the elements of a
+        // quantised candidate whose quotient lies just above the maximum it rounds to would divide every time.
+        const float half = (run.z != 0u && run.z < 0x7F800000u) ? __uint_as_float(((run.z >> 23) - 24u) << 23) : 0.0f;
+        if constexpr (ADD_NOW) {
+        // (callers with one lane per entry: one call site for all elements keeps the batch function short)
+        uint32_t pass = 0u;
 #pragma unroll
         for (int e = 0; e < EPV; ++e) {
-            if ((w[e] > 0.0f) || ((flags & 2u) && ad[e] != 0.0f)) {
+            if ((w[e] > 0.0f && w[e] >= __fmul_rn(half, fabsf(r.rf[e]))) || ((flags & 2u) && ad[e] != 0.0f)) pass |= 1u << e;
+        }
+        while (pass) {                                  // one call site for all elements
+            const int e = __ffs(pass) - 1;
+            pass &= pass - 1u;
+            float ade = ad[0], are = r.rf[0];
+#pragma unroll
+            for (int k = 1; k < EPV; ++k) {
+                if (e == k) { ade = ad[k]; are = r.rf[k]; }
+            }
+            const uint32_t qe = rel_candidate_bits(ade, fabsf(are), M, run.z);
+            best = qe > best ? qe : best;
+        }
+        } else {
+#pragma unroll
+        for (int e = 0; e < EPV; ++e) {
+            if ((w[e] > 0.0f && w[e] >= __fmul_rn(half, fabsf(r.rf[e]))) || ((flags & 2u) && ad[e] != 0.0f)) {
                 const uint32_t qe = rel_candidate_bits(ad[e], fabsf(r.rf[e]), M, run.z);
                 best = qe > best ? qe : best;
             }
+        }
         }
         if (best > run.y) raise_maxrel(s, best);
     }

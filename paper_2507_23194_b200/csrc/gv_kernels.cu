@@ -1515,7 +1515,10 @@ gv_status device_info(int* sm_count) {
 }
 
 bool tol_valid(const gv_tol* t) {
-    return t && isfinite(t->atol) && isfinite(t->rtol) && t->atol >= 0.0 && t->rtol >= 0.0;
+    // (written so that a NaN fails; above FLT_MAX the binary32 tolerance would be infinite and
+    // tol = atol + rtol * |r| a NaN for r = 0)
+    const double top = 3.4028234663852886e38;
+    return t && t->atol >= 0.0 && t->atol <= top && t->rtol >= 0.0 && t->rtol <= top;
 }
 
 template <int DT, bool BIGK>

@@ -63,6 +63,8 @@ def test_dense_argument_errors_return_before_any_launch(gvlib):
     assert _call_batch(gv, atol=float("nan")) == gv.GV_ERR_INVALID_ARG
     assert _call_batch(gv, rtol=-1.0) == gv.GV_ERR_INVALID_ARG
     assert _call_batch(gv, atol=float("inf")) == gv.GV_ERR_INVALID_ARG
+    assert _call_batch(gv, atol=3.5e38) == gv.GV_ERR_INVALID_ARG          # not a finite binary32 value
+    assert _call_batch(gv, rtol=1e300) == gv.GV_ERR_INVALID_ARG
     assert _call_batch(gv, tol_null=True) == gv.GV_ERR_INVALID_ARG
     assert _call_batch(gv, ws=None) == gv.GV_ERR_WORKSPACE
     assert _call_batch(gv, ws_bytes=8) == gv.GV_ERR_WORKSPACE

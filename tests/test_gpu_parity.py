@@ -700,3 +700,72 @@ def test_hash2_sizes_and_offsets(oracle):
     z, o = torch.zeros(2, dtype=torch.int64, device=DEV), torch.ones(2, dtype=torch.int64, device=DEV)
     assert int(gv.gv_hash(z).cpu()[0]) == int(gv.gv_hash(o).cpu()[0])          # the first lane's collision pair
     assert int(gv.gv_hash2(z).cpu()[0]) != int(gv.gv_hash2(o).cpu()[0])
+
+
+def _tie_candidates(r: torch.Tensor):
+    """Candidates whose relative errors tie, or nearly tie, with the running maximum in every element."""
+    f = r.float()
+    return [torch.zeros_like(r),                                  # |d| / |r| = 1 everywhere
+            -r,                                                   # 2 everywhere
+            (f * 3).to(r.dtype),                                  # 2 up to the rounding of 3r and of c - r
+            (f * 1.5).to(r.dtype),                                # 0.5 up to rounding
+            (f * (1 + 2.0 ** -7)).to(r.dtype),                    # a few quantised quotients
+            torch.where(torch.arange(r.numel()) % 5 == 0, (f * 3).to(r.dtype), r)]
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("code", [0, 1, 2])
+def test_relative_maximum_under_ties(oracle, code):
+    """The filter in front of the exact relative error lets an element through only when its quotient
+    exceeds the running maximum. Here nearly every element ties with that maximum or misses it by one
+    rounding, on the queueing path (small call) and the in-place path (a call large enough for the
+    sampling pass, every vector differing)."""
+    for n, scale in [(70001, 1.0), ((1 << 24) + 37 if code == 0 else (1 << 25) + 37, 0.05)]:
+        g = torch.Generator().manual_seed(900 + code)
+        r = (torch.randn(n, generator=g) * scale).to(TDT[code])
+        cands = _tie_candidates(r)
+        for atol, rtol in [(1e-2, 1e-2), (0.0, 0.0)]:
+            got, _ = run_dense(r.to(DEV), [c.to(DEV) for c in cands], atol, rtol, False)
+            want = oracle.verify_batch(host_bytes(r), [host_bytes(c) for c in cands], code, atol, rtol, False)
+            assert_records_equal(got, want, f"ties dtype {code} n {n} tol {atol}")
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("code", [0, 1])
+def test_relative_maximum_with_tiny_references(oracle, code):
+    """Reference magnitudes from 2^-20 down to the subnormals (the relative-error filter trusts its
+    multiply-add only above 2^-50 and must hand smaller elements to the exact path), mixed with ordinary
+    values so that a running maximum exists, candidates tying with it."""
+    rng = np.random.default_rng(77 + code)
+    n = 40003
+    expo = rng.integers(-149 if code == 0 else -133, -20, n)
+    mant = 1.0 + rng.integers(0, 1 << 7, n) / 128.0
+    vals = np.ldexp(mant, expo) * rng.choice([-1.0, 1.0], n)
+    ordinary = rng.random(n) < 0.3
+    vals[ordinary] = rng.standard_normal(int(ordinary.sum()))
+    vals[rng.integers(0, n, 50)] = 0.0
+    r = torch.from_numpy(vals.astype(np.float32)).to(TDT[code])
+    cands = _tie_candidates(r)
+    for atol, rtol in [(0.0, 0.0), (1e-30, 1e-3), (1e-2, 1e-2)]:
+        got, _ = run_dense(r.to(DEV), [c.to(DEV) for c in cands], atol, rtol, False)
+        want = oracle.verify_batch(host_bytes(r), [host_bytes(c) for c in cands], code, atol, rtol, False)
+        assert_records_equal(got, want, f"tiny references dtype {code} tol {atol}")
+    # the ragged kernel runs the same filter from its own loops: the same data as one ragged tensor
+    nb = n * ESZ[code]
+    stride = (nb + 15) // 16 * 16
+    N = len(cands)
+    cand_buf = torch.zeros(stride * N, dtype=torch.uint8)
+    for j, c in enumerate(cands):
+        cand_buf[j * stride:j * stride + nb] = c.view(torch.uint8)
+    ref_buf = r.view(torch.uint8).clone()
+    ref_off, cand_off = torch.tensor([0, nb]), torch.tensor([j * stride for j in range(N)])
+    dtypes_t, n_el = torch.tensor([code], dtype=torch.uint8), torch.tensor([n])
+    for atol, rtol in [(0.0, 0.0), (1e-2, 1e-2)]:
+        ws = torch.empty(gv.gv_workspace_bytes(1, N), dtype=torch.uint8, device=DEV)
+        res = gv.gv_verify_ragged(ref_buf.to(DEV), ref_off.to(DEV), cand_buf.to(DEV), cand_off.to(DEV), dtypes_t.to(DEV),
+                                  N, atol, rtol, False, n_elems=n_el.to(DEV), workspace=ws)
+        torch.cuda.synchronize()
+        assert gv.gv_check(ws) == gv.GV_OK
+        want = oracle.verify_ragged(ref_buf.numpy(), ref_off.numpy(), cand_buf.numpy(), cand_off.numpy(), dtypes_t.numpy(),
+                                    N, atol, rtol, False, n_elems=n_el.numpy())
+        assert_records_equal(gv.results_to_numpy(res), want, f"ragged tiny references dtype {code} tol {atol}")

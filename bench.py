@@ -59,11 +59,11 @@ def _scaled(measured, ref_bytes, cap_cands, full_cands, cap_chunks=None, full_ch
 
 
 NCU_TRAFFIC_BYTES = {
-    "cfg2": _scaled(2.182e9 + 4.4e6, 33554432, 64, 256, cap_chunks=1, full_chunks=1),   # profiles/dense_kernel_bf16_cfg2.md (reference stays in L2)
-    "cfg3": _scaled(5.100e9 + 4.8e6, 268435456, 16, 32, cap_chunks=3, full_chunks=2),   # profiles/dense_kernel_f16_cfg3.md
+    "cfg2": _scaled(2.181e9 + 3.8e6, 33554432, 64, 256, cap_chunks=1, full_chunks=1),   # profiles/dense_kernel_bf16_cfg2.md (reference stays in L2)
+    "cfg3": _scaled(5.100e9 + 5.1e6, 268435456, 16, 32, cap_chunks=3, full_chunks=2),   # profiles/dense_kernel_f16_cfg3.md
     "cfg4": _scaled(4.563e9 + 4.1e6, 268435456, 16, 64),      # profiles/dense_kernel_i32_cfg4.md
     "cfg4w": _scaled(4.832e9 + 3.8e6, 536870912, 8, 64, cap_chunks=1, full_chunks=4),   # profiles/dense_kernel_i64_cfg4w.md
-    "cfg5": (2.299e9 + 45.1e6) * 10000 / 2000,                # profiles/ragged_kernel_cfg5.md (2000 of 10000 tensors)
+    "cfg5": (2.300e9 + 45.4e6) * 10000 / 2000,                # profiles/ragged_kernel_cfg5.md (2000 of 10000 tensors)
 }
 
 

@@ -769,3 +769,83 @@ def test_relative_maximum_with_tiny_references(oracle, code):
         want = oracle.verify_ragged(ref_buf.numpy(), ref_off.numpy(), cand_buf.numpy(), cand_off.numpy(), dtypes_t.numpy(),
                                     N, atol, rtol, False, n_elems=n_el.numpy())
         assert_records_equal(gv.results_to_numpy(res), want, f"ragged tiny references dtype {code} tol {atol}")
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("code", [0, 1, 2])
+def test_relative_tolerance_regime(oracle, code):
+    """Tolerances that are relative in effect (atol far below rtol |r|): the fast path may then declare a
+    vector close because no quotient |d| / |r| exceeds a running maximum that is itself below rtol. Noise
+    inside, across and exactly at the edge of rtol, the margin around rtol (1 - 2^-22) bracketed, a single
+    far-off element that switches the shortcut off, zeros and tiny elements in the reference."""
+    g = torch.Generator().manual_seed(4100 + code)
+    # large enough that every warp sees many tiles of each candidate (the shortcut works on a per-CTA running
+    # maximum), small enough that the whole call stays on the queueing path (below the sampling pass)
+    n = 6000004 // ESZ[code] + 1
+    r = torch.randn(n, generator=g)
+    r[torch.randint(0, n, (40,), generator=g)] = 0.0
+    r[torch.randint(0, n, (40,), generator=g)] = 2.0 ** -60 if code != 2 else 2.0 ** -20
+    r = r.to(TDT[code])
+    rf = r.double()
+    u = torch.rand(n, generator=g, dtype=torch.float64) * 2 - 1
+    sign = torch.where(torch.rand(n, generator=g) < 0.5, -1.0, 1.0).double()
+    for rtol in [2.0 ** -7, 1e-2, 1.6e-2]:
+        cands = [(rf * (1 + u * rtol * 0.9)).to(TDT[code]),
+                 (rf * (1 + u * rtol * 1.1)).to(TDT[code]),
+                 (rf * (1 + sign * rtol)).to(TDT[code]),
+                 (rf * (1 + sign * rtol * (1 - 2.0 ** -22))).to(TDT[code]),
+                 (rf * (1 + sign * rtol * (1 - 2.0 ** -21))).to(TDT[code]),
+                 (rf * (1 + sign * rtol * (1 - 2.0 ** -23))).to(TDT[code])]
+        far = (rf * (1 + u * rtol * 0.5)).to(TDT[code])
+        far[n // 2] = far[n // 2] * 3 + 1
+        cands.append(far)
+        nz = r.clone()
+        nz[r == 0] = 2.0 ** -24
+        cands.append(nz)
+        withnan = cands[0].clone()
+        withnan[torch.randint(0, n, (9,), generator=g)] = float("nan")
+        withnan[torch.randint(0, n, (9,), generator=g)] = float("inf")
+        cands.append(withnan)
+        for atol in [0.0, 1e-8, 1e-5]:
+            got, _ = run_dense(r.to(DEV), [c.to(DEV) for c in cands], atol, rtol, False)
+            want = oracle.verify_batch(host_bytes(r), [host_bytes(c) for c in cands], code, atol, rtol, False)
+            assert_records_equal(got, want, f"relative regime dtype {code} rtol {rtol} atol {atol}")
+        # the same through the ragged kernel: one tensor, all candidates
+        nb = n * ESZ[code]
+        stride = (nb + 15) // 16 * 16
+        N = len(cands)
+        cand_buf = torch.zeros(stride * N, dtype=torch.uint8)
+        for j, c in enumerate(cands):
+            cand_buf[j * stride:j * stride + nb] = c.view(torch.uint8)
+        ref_buf = r.view(torch.uint8).clone()
+        ref_off, cand_off = torch.tensor([0, nb]), torch.tensor([j * stride for j in range(N)])
+        dtypes_t, n_el = torch.tensor([code], dtype=torch.uint8), torch.tensor([n])
+        ws = torch.empty(gv.gv_workspace_bytes(1, N), dtype=torch.uint8, device=DEV)
+        res = gv.gv_verify_ragged(ref_buf.to(DEV), ref_off.to(DEV), cand_buf.to(DEV), cand_off.to(DEV), dtypes_t.to(DEV),
+                                  N, 1e-8, rtol, True, n_elems=n_el.to(DEV), workspace=ws)
+        torch.cuda.synchronize()
+        assert gv.gv_check(ws) == gv.GV_OK
+        want = oracle.verify_ragged(ref_buf.numpy(), ref_off.numpy(), cand_buf.numpy(), cand_off.numpy(), dtypes_t.numpy(),
+                                    N, 1e-8, rtol, True, n_elems=n_el.numpy())
+        assert_records_equal(gv.results_to_numpy(res), want, f"ragged relative regime dtype {code} rtol {rtol}")
+
+
+@pytest.mark.gpu
+def test_relative_tolerance_edge_band(oracle):
+    """fp32 elements whose quotient |d| / |r| is rtol exactly (close: |d| = tol) or one step of 2^-23 above
+    it (not close), with atol = 0: the running maximum first settles at rtol through the ties, and the
+    elements one step above must still be counted -- a shortcut that trusted a maximum slightly above rtol
+    would call them close."""
+    rng = np.random.default_rng(5)
+    n = (1 << 22) + 3                                 # ~27 tiles per warp, so the per-CTA maximum settles
+    rtol = 0.25
+    sign = rng.choice([-1.0, 1.0], n)
+    r = (sign * 2.0 ** 20).astype(np.float32)
+    step = rng.choice([0, 0, 0, 1, 2], n).astype(np.float64)
+    c = (sign * (2.0 ** 20 * 1.25 + step * 2.0 ** -3)).astype(np.float32)
+    assert np.all(np.abs(c.astype(np.float64) - r) == 2.0 ** 18 + step * 2.0 ** -3)
+    rt, ct = torch.from_numpy(r), torch.from_numpy(c)
+    got, _ = run_dense(rt.to(DEV), [ct.to(DEV), ct.to(DEV).flip(0).flip(0)], 0.0, rtol, False)
+    want = oracle.verify_batch(host_bytes(rt), [host_bytes(ct)] * 2, oracle.F32, 0.0, rtol, False)
+    assert int(want[0]["n_mismatch"]) == int((step > 0).sum())          # by construction
+    assert_records_equal(got, want, "edge band")

@@ -470,7 +470,7 @@ __device__ __noinline__ uint32_t rel_candidate_bits(float ad, float ar, float M,
 // atomic per warp) -- inside this function the set of lanes present is not known reliably.
 // ADD_NOW: add the count to the accumulator at once (callers whose lanes each work for their own
 // candidate) instead of returning it in n_not_close.
-template <int DT, bool ADD_NOW = false>
+template <int DT, bool ADD_NOW = false, bool REL_OK = ADD_NOW>
 __device__ __forceinline__ bool vec_fast_float(const uint4& c, const RefVec<16 / Traits<DT>::ESZ>& r, uint32_t flags,
                                                const TolF& t, CtaAcc* s, uint64_t elem0, uint32_t& n_not_close) {
     constexpr int EPV = 16 / Traits<DT>::ESZ;
@@ -497,10 +497,10 @@ __device__ __forceinline__ bool vec_fast_float(const uint4& c, const RefVec<16 /
     // and |d| a binary32 value. So when no element of the vector exceeds M (vw <= 0) and all |d| are
     // finite, every element is close whatever the smallest tolerance of the vector says: with an
     // essentially relative tolerance (atol << rtol |r|) the vector's largest |d| sits on a large element
-    // and exceeds the tolerance of its smallest one all the time. (Used by the callers with one lane per
-    // entry; in the in-place loop of the dense kernel the two extra instructions cost 3-4 % on data that
-    // does not need them.)
-    const float lim = (ADD_NOW && run.z <= __float_as_uint(t.rtol)) ? __uint_as_float(0x7F7FFFFFu) : r.tolmin;
+    // and exceeds the tolerance of its smallest one all the time. (REL_OK: the callers with one lane per
+    // entry always; the in-place loop of the dense kernel, where the two extra instructions cost 3-4 % on
+    // data that does not need them, in the instance the host picks when atol is far below rtol.)
+    const float lim = (REL_OK && run.z <= __float_as_uint(t.rtol)) ? __uint_as_float(0x7F7FFFFFu) : r.tolmin;
     const bool raise_abs = vab > run.x;
     const bool maybe_rel = vw > 0.0f || ((flags & 2u) && vab != 0u);
     if (va <= lim && !(raise_abs || maybe_rel)) return true;

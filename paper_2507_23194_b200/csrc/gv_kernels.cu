@@ -159,6 +159,7 @@ struct DenseParams {
     int equal_nan;
     int N;                      // candidates in this launch (<= kMaxPtrs)
     int all_aligned;            // reference and every candidate base are 16-byte aligned
+    int rel_regime;             // float dtypes: atol is far below rtol (the tolerance is relative in effect): REL kernel
     const unsigned char* flags; // device, one byte per candidate of this launch: 1 = differs from the reference nearly everywhere
     const unsigned char* cands[kMaxPtrs];
 };
@@ -319,7 +320,9 @@ __global__ void __launch_bounds__(kThreads) classify_kernel(const __grid_constan
 }
 
 // BIGK: word indices of the hash need more than 32 bits (tensors of 32 GiB and more).
-template <int DT, bool BIGK>
+// REL: float dtypes, the in-place loop with the fast path's second way to "all close" (the host picks it
+// when atol is far below rtol; a kernel of its own so that the other one pays nothing for it).
+template <int DT, bool BIGK, bool REL>
 __global__ void __launch_bounds__(DenseShape<DT>::kWarpsPerCta * 32, DenseShape<DT>::kCtasPerSm)
 dense_kernel(const __grid_constant__ DenseParams p) {
     constexpr int kWarps = DenseShape<DT>::kWarpsPerCta;      // (shadows the 8-warp default of the other kernels)
@@ -438,7 +441,9 @@ dense_kernel(const __grid_constant__ DenseParams p) {
         // ================= fast loop: full warp-tiles, every base 16-byte aligned =================
         // Two instances of the same loop: MODE 0 queues every differing vector (candidates that mostly
         // agree with the reference), MODE 1 compares every differing vector in place against values
-        // hoisted per tile (candidates that differ nearly everywhere). Both are correct for any data.
+        // hoisted per tile (candidates that differ nearly everywhere), MODE 2 (the REL kernel's) is MODE 1 with
+        // the fast path's second way to "all close" for tolerances that are relative in effect. All are correct
+        // for any data.
         auto fast_loop = [&](auto mode_tag) {
             constexpr int MODE = decltype(mode_tag)::value;
             const uint32_t my_tiles = static_cast<uint32_t>(min((full_tiles - gw + GW - 1) / GW, uint64_t(0xFFFFFFFFu)));
@@ -494,7 +499,7 @@ dense_kernel(const __grid_constant__ DenseParams p) {
                 if constexpr (!IS_FLOAT) {
                     settle_vector_int<DT>(c, r, voff / ESZ, &cacc[k]);
                 } else {
-                    if (!vec_fast_float<DT>(c, rv, rflags, tol, &cacc[k], voff / ESZ, lane_cnt))
+                    if (!vec_fast_float<DT, false, MODE == 2>(c, rv, rflags, tol, &cacc[k], voff / ESZ, lane_cnt))
                         settle_vector_exact<DT>(c, rv, voff / ESZ, tol, &cacc[k]);
                 }
             };
@@ -508,7 +513,7 @@ dense_kernel(const __grid_constant__ DenseParams p) {
             // Float chunks of flagged candidates in the block loop: when nearly every vector differs, the identity
             // test decides nothing (a warp runs the compare whenever one of its lanes needs it), so every vector
             // is hashed and compared outright and the slots collect whole hashes, not corrections.
-            constexpr bool kEveryVector = MODE == 1 && IS_FLOAT;
+            constexpr bool kEveryVector = MODE != 0 && IS_FLOAT;
             const bool want_ref_hash = g == 0 && p.ref_hash != nullptr;
             uint64_t ref_only = 0;     // the reference's own terms where the slots do not need them
             auto hash_of = [&](const uint4& v) -> uint64_t {
@@ -545,7 +550,7 @@ dense_kernel(const __grid_constant__ DenseParams p) {
                 const bool differs = (c.x != r.x) || (c.y != r.y) || (c.z != r.z) || (c.w != r.w);
                 if (__any_sync(0xFFFFFFFFu, differs) || tile_forced) {
                     const bool want = differs || force != 0u;
-                    if constexpr (MODE == 1) {
+                    if constexpr (MODE != 0) {
                         ensure_hoisted(r);
                         uint32_t lane_cnt = 0u;
                         if (differs) correct_slot(c, k);
@@ -764,8 +769,11 @@ dense_kernel(const __grid_constant__ DenseParams p) {
             }
         };
         if (gw < full_tiles && !timed_out) {
-            if (chunk_dense) fast_loop(std::integral_constant<int, 1>{});
-            else fast_loop(std::integral_constant<int, 0>{});
+            if (!chunk_dense) {
+                fast_loop(std::integral_constant<int, 0>{});
+            } else {
+                fast_loop(std::integral_constant<int, (IS_FLOAT && REL) ? 2 : 1>{});
+            }
         }
 
         // ================= general loop: ragged tail, or some base not 16-byte aligned =================
@@ -1521,14 +1529,15 @@ bool tol_valid(const gv_tol* t) {
     return t && t->atol >= 0.0 && t->atol <= top && t->rtol >= 0.0 && t->rtol <= top;
 }
 
-template <int DT, bool BIGK>
+template <int DT, bool BIGK, bool REL = false>
 gv_status launch_dense_t(const gv::DenseParams& p, int sm_count, cudaStream_t st) {
     constexpr int kWarpsCta = gv::DenseShape<DT>::kWarpsPerCta;
     using S = gv::DenseSmem<kWarpsCta>;
     static int blocks_per_sm[64] = {0};
     int dev = 0;
     GV_CUDA(cudaGetDevice(&dev));
-    auto kern = gv::dense_kernel<DT, BIGK>;
+    if (dev < 0 || dev >= 64) return GV_ERR_CUDA;
+    auto kern = gv::dense_kernel<DT, BIGK, REL>;
     if (blocks_per_sm[dev] == 0) {
         GV_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(S::kTotal)));
         int b = 0;
@@ -1548,6 +1557,14 @@ gv_status launch_dense_t(const gv::DenseParams& p, int sm_count, cudaStream_t st
 
 gv_status launch_dense(gv_dtype dt, const gv::DenseParams& p, int sm_count, cudaStream_t st) {
     const bool bigk = p.n * static_cast<uint64_t>(gv::elem_size(dt)) >= (1ull << 35);
+    if (!bigk && p.rel_regime) {
+        switch (dt) {
+            case GV_F32: return launch_dense_t<GV_F32, false, true>(p, sm_count, st);
+            case GV_BF16: return launch_dense_t<GV_BF16, false, true>(p, sm_count, st);
+            case GV_F16: return launch_dense_t<GV_F16, false, true>(p, sm_count, st);
+            default: break;
+        }
+    }
     switch (dt) {
         case GV_F32: return bigk ? launch_dense_t<GV_F32, true>(p, sm_count, st) : launch_dense_t<GV_F32, false>(p, sm_count, st);
         case GV_BF16: return bigk ? launch_dense_t<GV_BF16, true>(p, sm_count, st) : launch_dense_t<GV_BF16, false>(p, sm_count, st);
@@ -1687,6 +1704,7 @@ gv_status gv_verify_batch(const void* ref, const void* const* cands, int32_t N, 
         p.atol = is_float ? static_cast<float>(tol->atol) : 0.0f;
         p.rtol = is_float ? static_cast<float>(tol->rtol) : 0.0f;
         p.equal_nan = is_float ? (tol->equal_nan != 0) : 0;
+        p.rel_regime = is_float && p.atol < p.rtol * 0.0625f;
         p.N = (N - j0) < gv::kMaxPtrs ? (N - j0) : gv::kMaxPtrs;
         uintptr_t all_bits = reinterpret_cast<uintptr_t>(ref);
         for (int k = 0; k < gv::kMaxPtrs; ++k) {

@@ -183,7 +183,9 @@ struct DenseParams {
 //     candidates, cuts them into chunks and runs one of two instances of its loop per chunk: one
 //     queues differing vectors per warp and compares them 32 at a time, one per lane (candidates
 //     that mostly agree with the reference); the other compares every differing vector in place
-//     against values derived from the reference once per tile (chunks of flagged candidates).
+//     against values derived from the reference once per tile (chunks of flagged candidates). A
+//     second compilation of the kernel (REL), launched when atol is far below rtol, lets that loop
+//     settle vectors by the running maximum of the relative error as well.
 //   * Accumulators: max |d|, max relative error, counts and the first index go to per-CTA shared
 //     accumulators only when they can change them. One block combine and one set of global
 //     integer atomics per (CTA, candidate).
@@ -439,7 +441,7 @@ dense_kernel(const __grid_constant__ DenseParams p) {
         for (int k = 0; k < kg; ++k) slots[k * 32] = make_uint2(0u, 0u);
 
         // ================= fast loop: full warp-tiles, every base 16-byte aligned =================
-        // Two instances of the same loop: MODE 0 queues every differing vector (candidates that mostly
+        // Instances of the same loop: MODE 0 queues every differing vector (candidates that mostly
         // agree with the reference), MODE 1 compares every differing vector in place against values
         // hoisted per tile (candidates that differ nearly everywhere), MODE 2 (the REL kernel's) is MODE 1 with
         // the fast path's second way to "all close" for tolerances that are relative in effect. All are correct

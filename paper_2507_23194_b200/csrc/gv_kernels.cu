@@ -726,8 +726,37 @@ dense_kernel(const __grid_constant__ DenseParams p) {
                 };
                 for (uint32_t t = 0; t < depth; ++t) issue_tile(t, t);
                 uint32_t slot = 0u;
+                uint32_t i = 0u;
+                if (kg == 1) {
+                    // One candidate: a warp's iteration is a chain of dependent instructions (the reference's
+                    // hash, two votes, the identity test) with nothing to overlap it, so two tiles are taken
+                    // per iteration and their reference hashes computed side by side.
 #pragma unroll 1
-                for (uint32_t i = 0; i < my_tiles; ++i) {
+                    for (; i + 2u <= my_tiles; i += 2u) {
+                        cp_async_wait<2>();                            // the two oldest tiles have landed
+                        const uint32_t at0 = ring_base + slot * 1024u, at1 = at0 + 1024u;     // slot is 0 or 2 here
+                        const uint4 r0 = lds128(at0), c0 = lds128(at0 + 512u);
+                        const uint4 r1 = lds128(at1), c1 = lds128(at1 + 512u);
+                        issue_tile(i + 4u, slot);
+                        issue_tile(i + 5u, slot + 1u);
+                        slot ^= 2u;
+                        const uint64_t h0 = hash_of(r0);
+                        voff += tile_stride;
+                        const uint64_t h1 = hash_of(r1);
+                        voff -= tile_stride;
+                        ref_sum += h0 + h1;
+                        h_ref = h0;
+                        new_tile(r0);
+                        visit(c0, r0, 0);
+                        voff += tile_stride;
+                        h_ref = h1;
+                        new_tile(r1);
+                        visit(c1, r1, 0);
+                        voff += tile_stride;
+                    }
+                }
+#pragma unroll 1
+                for (; i < my_tiles; ++i) {
                     if (depth == 4u) cp_async_wait<3>(); else cp_async_wait<1>();
                     const uint32_t at = ring_base + slot * per * 512u;
                     const uint4 r = lds128(at);

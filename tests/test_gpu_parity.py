@@ -852,3 +852,29 @@ def test_relative_tolerance_edge_band(oracle):
     want = oracle.verify_batch(host_bytes(rt), [host_bytes(ct)] * 2, oracle.F32, 0.0, rtol, False)
     assert int(want[0]["n_mismatch"]) == int((step > 0).sum())          # by construction
     assert_records_equal(got, want, "edge band")
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("code", [0, 1, 2, 3, 4])
+def test_single_candidate_tile_pairs(oracle, code):
+    """One candidate per call at sizes where the warps of the grid get two to five 512-byte tiles each, an
+    odd or an even number and not the same for every warp: the loop for a single candidate takes its
+    tiles two at a time and finishes with a single one."""
+    g = torch.Generator().manual_seed(600 + code)
+    warps = 148 * 2 * 8
+    for tiles in [2 * warps, 2 * warps + 1, 3 * warps + 777, 4 * warps - 1, 5 * warps + 5]:
+        n = tiles * 512 // ESZ[code] + 3
+        if code >= 3:
+            r = torch.randint(-(1 << 20), 1 << 20, (n,), generator=g, dtype=TDT[code])
+            c = torch.where(torch.rand(n, generator=g) < 1e-3, r + 7, r)
+            d = torch.where(torch.rand(n, generator=g) < 0.7, r - 1, r)
+        else:
+            r = torch.randn(n, generator=g).to(TDT[code])
+            r[torch.randint(0, n, (5,), generator=g)] = float("nan")
+            c = torch.where(torch.rand(n, generator=g) < 1e-3, (r.float() + 1).to(TDT[code]), r)
+            d = (r.float() * (1 + 3e-3 * torch.randn(n, generator=g))).to(TDT[code])
+        for cand in (r.clone(), c, d):
+            got, rh = run_dense(r.to(DEV), [cand.to(DEV)], 1e-2, 1e-2, code == 1)
+            want = oracle.verify_batch(host_bytes(r), [host_bytes(cand)], code, 1e-2, 1e-2, code == 1)
+            assert_records_equal(got, want, f"single candidate dtype {code} tiles {tiles}")
+            assert rh == oracle.hash_bytes(host_bytes(r))

@@ -238,6 +238,22 @@ __device__ __noinline__ void settle_vector_exact(uint4 c, RefVec<16 / Traits<DT>
     if (a.cnt) add_count(&s->cnt, a.cnt);
     raise_maxabs(s, a.maxabs);
 }
+// Two vectors of one flagged float candidate (two tiles of a single-candidate chunk), each against its own
+// reference vector: derived values, fast path, exact rule where needed, counts merged for both.
+template <int DT, bool REL_OK>
+__device__ __noinline__ void compare_pair_float(uint4 c0, uint4 r0, uint4 c1, uint4 r1, TolF tol, CtaAcc* s, uint64_t elem0,
+                                                uint64_t elem1) {
+    if constexpr (Traits<DT>::IS_FLOAT) {
+        constexpr int EPV = 16 / Traits<DT>::ESZ;
+        RefVec<EPV> rva, rvb;
+        uint32_t fa = 0u, fb = 0u, n0 = 0u, n1 = 0u;
+        hoist_ref<DT>(r0, tol, rva, fa);
+        hoist_ref<DT>(r1, tol, rvb, fb);
+        if (!vec_fast_float<DT, false, REL_OK>(c0, rva, fa, tol, s, elem0, n0)) settle_vector_exact<DT>(c0, rva, elem0, tol, s);
+        if (!vec_fast_float<DT, false, REL_OK>(c1, rvb, fb, tol, s, elem1, n1)) settle_vector_exact<DT>(c1, rvb, elem1, tol, s);
+        if (__any_sync(0xFFFFFFFFu, (n0 | n1) != 0u)) merge_counts_converged(s, n0 + n1);
+    }
+}
 template <int DT>
 __device__ __noinline__ void settle_vector_int(uint4 c, uint4 r, uint64_t elem0, CtaAcc* s) {
     Acc a;
@@ -740,19 +756,34 @@ dense_kernel(const __grid_constant__ DenseParams p) {
                         issue_tile(i + 4u, slot);
                         issue_tile(i + 5u, slot + 1u);
                         slot ^= 2u;
-                        const uint64_t h0 = hash_of(r0);
-                        voff += tile_stride;
-                        const uint64_t h1 = hash_of(r1);
-                        voff -= tile_stride;
-                        ref_sum += h0 + h1;
-                        h_ref = h0;
-                        new_tile(r0);
-                        visit(c0, r0, 0);
-                        voff += tile_stride;
-                        h_ref = h1;
-                        new_tile(r1);
-                        visit(c1, r1, 0);
-                        voff += tile_stride;
+                        if constexpr (kEveryVector) {
+                            // a flagged float candidate: both vectors hashed and compared outright, as in the
+                            // block loop (whole hashes in the slot, the reference's terms only for ref_hash)
+                            uint64_t hc = hash_of(c0);
+                            if (want_ref_hash) ref_only += hash_of(r0);
+                            voff += tile_stride;
+                            hc += hash_of(c1);
+                            if (want_ref_hash) ref_only += hash_of(r1);
+                            const uint2 sl = slots[0];
+                            const uint64_t hs = pack64(sl.x, sl.y) + hc;
+                            slots[0] = make_uint2(static_cast<uint32_t>(hs), static_cast<uint32_t>(hs >> 32));
+                            compare_pair_float<DT, MODE == 2>(c0, r0, c1, r1, tol, &cacc[0], (voff - tile_stride) / ESZ, voff / ESZ);
+                            voff += tile_stride;
+                        } else {
+                            const uint64_t h0 = hash_of(r0);
+                            voff += tile_stride;
+                            const uint64_t h1 = hash_of(r1);
+                            voff -= tile_stride;
+                            ref_sum += h0 + h1;
+                            h_ref = h0;
+                            new_tile(r0);
+                            visit(c0, r0, 0);
+                            voff += tile_stride;
+                            h_ref = h1;
+                            new_tile(r1);
+                            visit(c1, r1, 0);
+                            voff += tile_stride;
+                        }
                     }
                 }
 #pragma unroll 1

@@ -862,7 +862,9 @@ def test_single_candidate_tile_pairs(oracle, code):
     tiles two at a time and finishes with a single one."""
     g = torch.Generator().manual_seed(600 + code)
     warps = 148 * 2 * 8
-    for tiles in [2 * warps, 2 * warps + 1, 3 * warps + 777, 4 * warps - 1, 5 * warps + 5]:
+    # (the last size is past 64 MB, where the sampling pass runs: the candidate that differs everywhere is then
+    # flagged and takes the in-place form of the loop)
+    for tiles in [2 * warps, 2 * warps + 1, 3 * warps + 777, 4 * warps - 1, 5 * warps + 5, (64 << 20) // 512 + warps + 1]:
         n = tiles * 512 // ESZ[code] + 3
         if code >= 3:
             r = torch.randint(-(1 << 20), 1 << 20, (n,), generator=g, dtype=TDT[code])
@@ -874,6 +876,8 @@ def test_single_candidate_tile_pairs(oracle, code):
             c = torch.where(torch.rand(n, generator=g) < 1e-3, (r.float() + 1).to(TDT[code]), r)
             d = (r.float() * (1 + 3e-3 * torch.randn(n, generator=g))).to(TDT[code])
         for cand in (r.clone(), c, d):
+            if tiles > 6 * warps and cand is c:
+                continue
             got, rh = run_dense(r.to(DEV), [cand.to(DEV)], 1e-2, 1e-2, code == 1)
             want = oracle.verify_batch(host_bytes(r), [host_bytes(cand)], code, 1e-2, 1e-2, code == 1)
             assert_records_equal(got, want, f"single candidate dtype {code} tiles {tiles}")

@@ -254,6 +254,26 @@ __device__ __noinline__ void compare_pair_float(uint4 c0, uint4 r0, uint4 c1, ui
         if (__any_sync(0xFFFFFFFFu, (n0 | n1) != 0u)) merge_counts_converged(s, n0 + n1);
     }
 }
+// One tile of a chunk of one to three flagged float candidates: the reference vector's derived values
+// once, then each candidate's vector against them.
+template <int DT, bool REL_OK>
+__device__ __noinline__ void compare_few_float(uint4 c0, uint4 c1, uint4 c2, uint4 r, int kg, TolF tol, CtaAcc* acc, uint64_t elem0) {
+    if constexpr (Traits<DT>::IS_FLOAT) {
+        constexpr int EPV = 16 / Traits<DT>::ESZ;
+        RefVec<EPV> rv;
+        uint32_t flags = 0u;
+        hoist_ref<DT>(r, tol, rv, flags);
+        const uint4 c[3] = {c0, c1, c2};
+#pragma unroll
+        for (int u = 0; u < 3; ++u) {
+            if (u < kg) {
+                uint32_t n = 0u;
+                if (!vec_fast_float<DT, false, REL_OK>(c[u], rv, flags, tol, &acc[u], elem0, n)) settle_vector_exact<DT>(c[u], rv, elem0, tol, &acc[u]);
+                if (__any_sync(0xFFFFFFFFu, n != 0u)) merge_counts_converged(&acc[u], n);
+            }
+        }
+    }
+}
 template <int DT>
 __device__ __noinline__ void settle_vector_int(uint4 c, uint4 r, uint64_t elem0, CtaAcc* s) {
     Acc a;
@@ -796,12 +816,26 @@ dense_kernel(const __grid_constant__ DenseParams p) {
                     for (int u = 0; u < 3; ++u) c[u] = u < kg ? lds128(at + (1u + u) * 512u) : r;
                     issue_tile(i + depth, slot);                       // refill the stages just read
                     slot = slot + 1u == depth ? 0u : slot + 1u;
-                    h_ref = hash_of(r);
-                    ref_sum += h_ref;
-                    new_tile(r);
+                    if constexpr (kEveryVector) {
+                        // flagged float candidates: every vector hashed and compared outright (see the block loop)
+                        if (want_ref_hash) ref_only += hash_of(r);
 #pragma unroll
-                    for (int u = 0; u < 3; ++u)
-                        if (u < kg) visit(c[u], r, u);
+                        for (int u = 0; u < 3; ++u) {
+                            if (u < kg) {
+                                const uint2 sl = slots[u * 32];
+                                const uint64_t hs = pack64(sl.x, sl.y) + hash_of(c[u]);
+                                slots[u * 32] = make_uint2(static_cast<uint32_t>(hs), static_cast<uint32_t>(hs >> 32));
+                            }
+                        }
+                        compare_few_float<DT, MODE == 2>(c[0], c[1], c[2], r, kg, tol, cacc, voff / ESZ);
+                    } else {
+                        h_ref = hash_of(r);
+                        ref_sum += h_ref;
+                        new_tile(r);
+#pragma unroll
+                        for (int u = 0; u < 3; ++u)
+                            if (u < kg) visit(c[u], r, u);
+                    }
                     voff += tile_stride;
                 }
             }

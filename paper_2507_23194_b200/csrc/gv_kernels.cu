@@ -1375,8 +1375,33 @@ __device__ __noinline__ uint64_t ragged_stream(const RaggedParams& p, int dt, ui
 #pragma unroll 1
         for (int j = 0; j < kRing; ++j) issue_one(ring_base + j * 512u);
         uint32_t stage = 0;
+        uint64_t tile = tile_begin;
+        if (kg == 1) {
+            // One candidate per tensor: two tiles per iteration (four copies of the sequence), the two
+            // reference hashes side by side -- a single tile's chain of dependent instructions is too short
+            // of parallelism for 16 warps per SM to hide.
 #pragma unroll 1
-        for (uint64_t tile = tile_begin; tile < full_end; ++tile) {
+            for (; tile + 2 <= full_end; tile += 2) {
+                const uint64_t voff0 = tile * kWarpTile + lane * 16, voff1 = voff0 + kWarpTile;
+                cp_async_wait<kRing - 4>();
+                const uint32_t at0 = ring_base + stage * 512u, at1 = ring_base + ((stage + 1u) & (kRing - 1)) * 512u;
+                const uint32_t at2 = ring_base + ((stage + 2u) & (kRing - 1)) * 512u, at3 = ring_base + ((stage + 3u) & (kRing - 1)) * 512u;
+                const uint4 r0 = lds128(at0), c0 = lds128(at1), r1 = lds128(at2), c1 = lds128(at3);
+                stage = (stage + 4u) & (kRing - 1);
+                issue_one(at0);
+                issue_one(at1);
+                issue_one(at2);
+                issue_one(at3);
+                const bool force0 = nan_matters && vec_has_nonfinite(dt, r0), force1 = nan_matters && vec_has_nonfinite(dt, r1);
+                const uint64_t h0 = hash_vec_full_k32(r0, static_cast<uint32_t>(voff0 / 8));
+                const uint64_t h1 = hash_vec_full_k32(r1, static_cast<uint32_t>(voff1 / 8));
+                ref_sum += h0 + h1;
+                queued_visit(c0, r0, h0, force0, voff0, 0);
+                queued_visit(c1, r1, h1, force1, voff1, 0);
+            }
+        }
+#pragma unroll 1
+        for (; tile < full_end; ++tile) {
             const uint64_t voff = tile * kWarpTile + lane * 16;
             cp_async_wait<kRing - 1>();
             uint32_t at = ring_base + stage * 512u;

@@ -882,3 +882,50 @@ def test_single_candidate_tile_pairs(oracle, code):
             want = oracle.verify_batch(host_bytes(r), [host_bytes(cand)], code, 1e-2, 1e-2, code == 1)
             assert_records_equal(got, want, f"single candidate dtype {code} tiles {tiles}")
             assert rh == oracle.hash_bytes(host_bytes(r))
+
+
+@pytest.mark.gpu
+def test_ragged_single_candidate_streams(oracle):
+    """One candidate per tensor, tensors of hundreds to thousands of tiles of every dtype: the ragged kernel's
+    loop for any candidate count takes a single candidate's tiles two at a time (and an odd one last)."""
+    g = torch.Generator().manual_seed(888)
+    sizes = [(1 << 20) + 77, (1 << 19) + 5, 999999, 3 * (1 << 18), 40000, (1 << 20) - 3, 128 * 7 + 1]
+    codes = [0, 1, 2, 3, 4, 1, 0]
+    T = len(sizes)
+    refs, cands = [], []
+    for t in range(T):
+        code, n = codes[t], sizes[t]
+        if code >= 3:
+            r = torch.randint(-(1 << 20), 1 << 20, (n,), generator=g, dtype=TDT[code])
+            c = torch.where(torch.rand(n, generator=g) < 0.01, r + 3, r)
+        else:
+            r = torch.randn(n, generator=g).to(TDT[code])
+            r[torch.randint(0, n, (7,), generator=g)] = float("nan")
+            c = torch.where(torch.rand(n, generator=g) < (0.01 if t % 2 else 1.0),
+                            (r.float() * (1 + 2e-3 * torch.randn(n, generator=g))).to(TDT[code]), r)
+        refs.append(r)
+        cands.append(c)
+    ref_off, cand_off, rc = [], [], 0
+    for t in range(T):
+        rc = (rc + 15) // 16 * 16
+        ref_off.append(rc)
+        cand_off.append(rc)
+        rc += sizes[t] * ESZ[codes[t]]
+    ref_off.append(rc)
+    ref_buf = torch.zeros(rc, dtype=torch.uint8)
+    cand_buf = torch.zeros(rc, dtype=torch.uint8)
+    for t in range(T):
+        nb = sizes[t] * ESZ[codes[t]]
+        ref_buf[ref_off[t]:ref_off[t] + nb] = refs[t].view(torch.uint8)
+        cand_buf[cand_off[t]:cand_off[t] + nb] = cands[t].view(torch.uint8)
+    ro, co = torch.tensor(ref_off), torch.tensor(cand_off)
+    dt, ne = torch.tensor(codes, dtype=torch.uint8), torch.tensor(sizes)
+    for en in (False, True):
+        ws = torch.empty(gv.gv_workspace_bytes(T, 1), dtype=torch.uint8, device=DEV)
+        res = gv.gv_verify_ragged(ref_buf.to(DEV), ro.to(DEV), cand_buf.to(DEV), co.to(DEV), dt.to(DEV), 1, 1e-2, 1e-2, en,
+                                  n_elems=ne.to(DEV), workspace=ws)
+        torch.cuda.synchronize()
+        assert gv.gv_check(ws) == gv.GV_OK
+        want = oracle.verify_ragged(ref_buf.numpy(), ro.numpy(), cand_buf.numpy(), co.numpy(), dt.numpy(), 1, 1e-2, 1e-2, en,
+                                    n_elems=ne.numpy())
+        assert_records_equal(gv.results_to_numpy(res), want, f"ragged single candidate equal_nan {en}")

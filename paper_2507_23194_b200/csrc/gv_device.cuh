@@ -417,10 +417,10 @@ __device__ __forceinline__ uint32_t rel_threshold_bits(uint32_t m_bits) {
     return m_bits < kTinyBits ? 0u : m_bits;
 }
 
-// Add a 32-bit count to a 64-bit counter in shared memory. A 64-bit shared-memory atomic add is a
-// compare-and-swap loop, and the lanes of a warp that add to the same counter (a batch of entries of one
-// candidate that mismatch everywhere) then retry against each other; the 32-bit add is one instruction
-// that resolves the conflict in hardware. The carry into the upper word is added separately (exact:
+// Add a 32-bit count to a 64-bit counter in shared memory. A 64-bit atomic add on shared memory behaves
+// like a compare-and-swap loop: when the lanes of a warp add to the same counter (a batch of entries of
+// one candidate that mismatch everywhere) its cost grows with the number of lanes that collide (measured:
+// shared-memory stalls dominated such launches); the 32-bit add resolves the conflict in hardware. The carry into the upper word is added separately (exact:
 // the sum wraps mod 2^64, and nothing reads the counter before the CTA's final barrier).
 __device__ __forceinline__ void add_count(unsigned long long* counter, uint32_t v) {
     uint32_t* w = reinterpret_cast<uint32_t*>(counter);
